@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the CoCoD-SGD parameter engine on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A "step" is one communication round of Algorithm 1 over all K workers: comm_begin (stored copy +
+averaging on the side stream), k local momentum-SGD steps, comm_end (merge).  The metric is
+worker-parameter updates per second = K * P * k * rounds / time, whole job over all ranks.
+Prints ONE JSON line (rank 0).
+
+N > 1 (torchrun): the path shards by parameter index with no exchange at all, so every rank
+runs the same per-GPU workload on its own column range (weak scaling); time is the max over
+ranks of the device-timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "worker-param updates/sec (K*P*steps/s)"
+UNIT = "updates/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20, help="timed rounds")
+    ap.add_argument("--warmup", type=int, default=3, help="untimed rounds (>= 3)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18", choices=["tiny", "resnet18", "vgg16"])
+    ap.add_argument("--snapshot", default="flip", choices=["flip", "copy"])
+    ap.add_argument("--ring", type=int, default=4, help="distinct gradient buffers cycled through")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-cols", type=int, default=1 << 20)
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(index), "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle leg
+def time_oracle(wl, cols: int, steps: int, warmup: int):
+    """The oracle as it stands (ref mode, all host cores) on a column sample of the workload:
+    rounds of Algorithm 1 over K workers x `cols` columns.  Gradient generation is outside the
+    timed region.  Returns (updates/s, seconds per round, cores)."""
+    import numpy as np
+    from oracle import cocod_oracle as O
+    from paper_1906_12043_b200 import inputs as I
+    cores = O.max_threads()
+    O.set_threads(cores)
+    K, k = wl.K, wl.k
+    col_idx = np.arange(cols, dtype=np.uint64)
+    eng = O.OracleEngine(K, cols, wl.lr, wl.mu, wl.wd, mode="ref")
+    eng.set_params(I.initial_point(wl.P, wl.sigma_x0, cols=col_idx))
+    ring = [I.gradients(K, wl.P, t, wl.sigma_g, cols=col_idx) for t in range(max(2, k))]
+
+    def one_round(r):
+        eng.comm_begin()
+        for s in range(k):
+            eng.local_step(ring[(r * k + s) % len(ring)])
+        eng.comm_end()
+
+    for r in range(warmup):
+        one_round(r)
+    t0 = time.perf_counter()
+    for r in range(steps):
+        one_round(warmup + r)
+    dt = time.perf_counter() - t0
+    O.set_threads(1)
+    return K * cols * k * steps / dt, dt / steps, cores
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cols = min(args.cpu_sample_cols, wl.P)
+    value, s_per_round, cores = time_oracle(wl, cols, args.steps, args.warmup)
+    sample = (f"{wl.K} workers x first {cols} of {wl.P} columns, {args.steps} rounds of k={wl.k} local steps "
+              f"(ref-mode oracle, OpenMP over columns); gradients pre-generated")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": s_per_round * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": wl.name, "K": wl.K, "P": wl.P, "k": wl.k, "lr": wl.lr, "mu": wl.mu, "wd": wl.wd,
+                   "sampled_columns": cols},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ---------------------------------------------------------------------------------------------- our arm
+def summarize_profile(recs, names):
+    by = {}
+    for kind, a, b in recs:
+        by.setdefault(names[kind], []).append((a, b))
+    return by
+
+
+def overlap_fraction(by):
+    """Share of the mean kernels' lifetime that lies inside some local-step kernel's lifetime."""
+    steps = sorted(by.get("local_step", []))
+    tot = cov = 0.0
+    for a, b in by.get("mean", []):
+        tot += b - a
+        for c, d in steps:
+            lo, hi = max(a, c), min(b, d)
+            if hi > lo:
+                cov += hi - lo
+    return cov / tot if tot > 0 else None
+
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_1906_12043_b200 import build, engine as E, inputs as I, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the engine has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    E.load()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K, P, k = wl.K, wl.P, wl.k
+    p0 = rank * P                                       # this rank's columns of the global vector
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
+
+    eng = E.Engine(K, P, wl.lr, wl.mu, wl.wd)
+    eng.set_option(E.OPT_SNAPSHOT, E.SNAPSHOT_FLIP if args.snapshot == "flip" else E.SNAPSHOT_COPY)
+    x0 = torch.empty(P, dtype=torch.float32, device="cuda")
+    I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, p0, wl.sigma_x0)
+    eng.set_params(x0)
+    ring = []
+    for t in range(max(1, args.ring)):
+        g = torch.empty((K, P), dtype=torch.float32, device="cuda")
+        I.device_gradients_into(g, t, wl.sigma_g, p0=p0)
+        ring.append(g)
+    side = torch.cuda.Stream(priority=-1)
+    compute = torch.cuda.current_stream()
+    step_no = [0]
+
+    def one_round(side_stream):
+        eng.comm_begin(side_stream)
+        for _ in range(k):
+            eng.local_step(ring[step_no[0] % len(ring)])
+            step_no[0] += 1
+        eng.comm_end()
+
+    # ---- device-resident timed region
+    for _ in range(max(3, args.warmup)):
+        one_round(side)
+    eng.set_option(E.OPT_PROFILE, 1)
+    eng.profile_reset()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = eng.launch_count
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(compute)
+    for _ in range(args.steps):
+        one_round(side)
+    ev1.record(compute)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    ms = ev0.elapsed_time(ev1)
+    launches = eng.launch_count - launches0
+    by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+    eng.set_option(E.OPT_PROFILE, 0)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * K * P * k * args.steps / (ms * 1e-3)
+
+    alg_bytes = {"local_step": W.BYTES_LOCAL_STEP * K * P, "snapshot": W.BYTES_SNAPSHOT * K * P,
+                 "mean": W.bytes_mean(K) * K * P, "merge": W.bytes_merge(K) * K * P}
+
+    def kernel_table(by_kind):
+        out = {}
+        for name, iv in by_kind.items():
+            avg_ms = sum(b - a for a, b in iv) / len(iv)
+            gbs = alg_bytes[name] / (avg_ms * 1e-3) / 1e9
+            out[name] = {"launches": len(iv), "avg_ms": round(avg_ms, 5), "gbs": round(gbs, 1),
+                         "frac_of_peak": round(gbs / hbm_peak, 4)}
+        return out
+
+    in_loop = kernel_table(by)
+    overlap = overlap_fraction(by)
+
+    # ---- the same rounds with the mean on the compute stream: isolated kernel times, serial round time
+    eng.set_option(E.OPT_PROFILE, 1)
+    eng.profile_reset()
+    torch.cuda.synchronize()
+    n_ser = min(args.steps, 10)
+    ev0.record(compute)
+    for _ in range(n_ser):
+        one_round(compute)
+    ev1.record(compute)
+    torch.cuda.synchronize()
+    ms_serial = ev0.elapsed_time(ev1) / n_ser
+    isolated = kernel_table(summarize_profile(eng.profile_records(), E.KERNEL_NAMES))
+    eng.set_option(E.OPT_PROFILE, 0)
+
+    dom = "local_step"
+    traffic = None
+    try:
+        tj = json.load(open(os.path.join(ROOT, "profiles", "ncu_traffic.json")))
+        ent = tj.get(dom, {})
+        if ent.get("dram_bytes_per_element") is not None:
+            traffic = ent["dram_bytes_per_element"] * K * P
+    except (OSError, ValueError):
+        pass
+    dom_tab = in_loop.get(dom, {})
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": dom_tab.get("gbs"), "peak": hbm_peak,
+                "unit": "GB/s", "frac": dom_tab.get("frac_of_peak"), "traffic": traffic,
+                "peak_kind": peak_kind, "algorithmic_bytes_per_launch": alg_bytes[dom],
+                "avg_launch_ms": dom_tab.get("avg_ms"), "isolated": isolated.get(dom)}
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        host_ring = []
+        for t in range(2):
+            hbuf = torch.empty((K, P), dtype=torch.float32, pin_memory=True)
+            hbuf.copy_(ring[t % len(ring)])
+            host_ring.append(hbuf)
+        mean_out = torch.empty(P, dtype=torch.float32, pin_memory=True)
+        hs = [0]
+
+        def one_round_host():
+            eng.comm_begin(side)
+            for _ in range(k):
+                eng.local_step_host(host_ring[hs[0] % 2])
+                hs[0] += 1
+            eng.comm_end()
+            eng.get_mean(mean_out)                      # device -> host read of the round's result
+
+        n_e2e = max(1, min(args.steps, 10))
+        for _ in range(2):
+            one_round_host()
+        barrier()
+        t0 = time.perf_counter()
+        ev0.record(compute)
+        for _ in range(n_e2e):
+            one_round_host()
+        ev1.record(compute)
+        barrier()
+        wall = time.perf_counter() - t0
+        ms_e2e = max(ev0.elapsed_time(ev1), 0.0)
+        if world > 1:
+            t = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": world * K * P * k * n_e2e / (ms_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": k * K * P * 4, "d2h_bytes_per_step": P * 4,
+               "rounds": n_e2e, "ms_per_step": ms_e2e / n_e2e, "wall_ms_per_step": wall * 1e3 / n_e2e}
+
+    # ---- CPU oracle beside it (rank 0, N = 1 only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cols = min(args.cpu_sample_cols, P)
+        target_s = 12.0
+        probe, s_per_round, cores = time_oracle(wl, cols, 2, 1)
+        n_rounds = max(2, min(200, int(target_s / max(s_per_round, 1e-6))))
+        v, s_per_round, cores = time_oracle(wl, cols, n_rounds, 1)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"{K} workers x first {cols} of {P} columns, {n_rounds} rounds of k={k} "
+                                  f"(ref-mode oracle, OpenMP over columns, gradients pre-generated)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "K": K, "P": P, "k": k, "lr": wl.lr, "mu": wl.mu, "wd": wl.wd,
+                       "snapshot": args.snapshot, "gradient_ring": len(ring),
+                       "l2": "inputs larger than L2 (each K x P buffer is %.0f MB, L2 is 126 MB)" % (K * P * 4 / 1e6)
+                             if K * P * 4 > 126e6 else "L2-resident workload: not an HBM number",
+                       "sharding": "columns, no exchange" if world > 1 else "single GPU"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "kernels_in_loop": in_loop, "kernels_isolated": isolated,
+            "overlap_fraction": overlap, "ms_per_round_overlapped": ms / args.steps,
+            "ms_per_round_serial": ms_serial,
+            "hbm_gbs_whole_round": wl.bytes_per_round(args.snapshot == "copy") / (ms / args.steps * 1e-3) / 1e9,
+        }
+        print(json.dumps(line))
+    eng.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse()
+    from paper_1906_12043_b200.workloads import WORKLOADS
+    wl = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,174 @@
+/*
+ * cocod.h -- C boundary of the B200 CoCoD-SGD parameter engine (libcocod.so).
+ *
+ * The engine holds K simulated workers (the paper's N) as replicas in one GPU's HBM and runs
+ * the per-round parameter path of Algorithm 1 ("CoCoD-SGD") of arxiv 1906.12043:
+ *
+ *     cocod_comm_begin   Step I   store x_t^i, start averaging the stored copies (side stream)
+ *     cocod_local_step   Step II  one local update of every worker (compute stream), k times
+ *     cocod_comm_end     line 6   x^i <- x_hat_t + (x^i - x_t^i)
+ *
+ * Conventions
+ *   - Plain C, opaque handle, every call returns an int: 0 = COCOD_OK, negative = error.
+ *     Nothing throws or aborts.  cocod_strerror() names a code.
+ *   - Layout: every K x P matrix is worker-major row-major fp32 with row stride P
+ *     (row i = worker i's flattened model of P parameters, the paper's d).
+ *   - Ownership: the engine owns x, the momentum v, the stored copies and the average model;
+ *     the caller owns gradient buffers and CUDA streams and must keep a gradient buffer valid
+ *     and unmodified until the compute stream has passed the call that reads it.
+ *   - "device" pointers are CUDA device pointers on the device that was current at
+ *     cocod_create; "host" pointers are ordinary (preferably pinned) host memory.
+ *   - Streams are passed as void* holding a cudaStream_t (NULL = the legacy default stream).
+ *   - All device work is stream-ordered and asynchronous; no call blocks the host except
+ *     cocod_sync, cocod_comm_wait, cocod_destroy and the transfers that name host memory.
+ *   - One host thread per handle (not thread-safe).  The device that was current at
+ *     cocod_create must be current for every later call on the handle.
+ *   - There is no CPU fallback: without a CUDA device every call fails with COCOD_ERR_CUDA.
+ */
+#ifndef COCOD_H
+#define COCOD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cocod_engine cocod_handle;
+typedef void *cocod_stream_t; /* a cudaStream_t */
+
+enum {
+    COCOD_OK = 0,
+    COCOD_ERR_INVALID = -1, /* bad argument (NULL, K < 1, P < 1, non-finite hyper-parameter, ...) */
+    COCOD_ERR_OOM = -2,     /* device or pinned-host allocation failed; nothing is leaked */
+    COCOD_ERR_STATE = -3,   /* call not legal now (comm_end without comm_begin, double begin) */
+    COCOD_ERR_CUDA = -4,    /* a CUDA call or kernel failed; sticky, see cocod_last_cuda_error */
+    COCOD_ERR_TIMEOUT = -5  /* cocod_comm_wait ran out of time; the engine is still usable */
+};
+
+/* Options for cocod_set_option. */
+enum {
+    /* How Step I "stores x_t^i".  COPY: a copy kernel writes the stored copies (8 B per
+     * worker-parameter per round).  FLIP (default): the buffer holding x becomes the stored
+     * copy and the first local step of the round writes x into the spare buffer (0 B); the
+     * values are identical. */
+    COCOD_OPT_SNAPSHOT = 1,
+    /* Record CUDA events around every kernel (cocod_profile_*). 0 = off (default). */
+    COCOD_OPT_PROFILE = 2
+};
+enum { COCOD_SNAPSHOT_COPY = 0, COCOD_SNAPSHOT_FLIP = 1 };
+
+/* Kernel kinds reported by cocod_profile_get. */
+enum { COCOD_KERNEL_LOCAL_STEP = 0, COCOD_KERNEL_SNAPSHOT = 1, COCOD_KERNEL_MEAN = 2, COCOD_KERNEL_MERGE = 3 };
+
+/* ---------------------------------------------------------------------------------------------
+ * Algorithm 1, "Input" / "Initialize": K workers, model size P, learning rate gamma = lr, and
+ * the optimizer constants of Section 5.1 (momentum mu, weight decay wd).  Allocates x, v, the
+ * stored copies (K x P fp32 each) and the average model (P) on the current device, zero-fills
+ * x and v, uses equal mini-batch sizes, the legacy default stream as compute stream, and the
+ * FLIP snapshot.  *out is written only on success.
+ * Errors: INVALID (out NULL, K < 1 or > 1024, P < 1, K*P*4 overflows, lr/mu/wd not finite),
+ * OOM, CUDA. */
+int cocod_create(cocod_handle **out, int K, int64_t P, float lr, float mu, float wd);
+
+/* Waits for the engine's pending device work, frees everything.  NULL is a no-op. */
+int cocod_destroy(cocod_handle *h);
+
+/* Algorithm 1, Step II body, one iteration tau for every worker, with the optimizer of the
+ * paper's experiments (Section 5.1; PyTorch SGD form, v starts at 0):
+ *     d = g + wd * x ;  v = mu * v + d ;  x = x - lr * v
+ * (mu = wd = 0 is Algorithm 1's x <- x - gamma G literally.)  grads: device, K x P, borrowed.
+ * Asynchronous on the compute stream.  Legal with or without a communication in flight. */
+int cocod_local_step(cocod_handle *h, const float *grads);
+
+/* Same update with the gradients in HOST memory (K x P): the engine stages them to the device
+ * in chunks on an internal copy stream, overlapping the copies with the update kernel.  The
+ * host buffer must stay valid until cocod_sync (or a later blocking call) returns. */
+int cocod_local_step_host(cocod_handle *h, const float *host_grads);
+
+/* Algorithm 1, Step I: store x_t^i and start computing the weighted mean of the stored copies
+ * x_hat_t = sum_i (M_i / sum_j M_j) x_t^i, "in parallel" with Step II: the mean kernel runs on
+ * `side`, ordered after the compute stream's work so far.  side == compute stream is allowed
+ * (then it simply runs in order).  Errors: STATE if a communication is already in flight. */
+int cocod_comm_begin(cocod_handle *h, cocod_stream_t side);
+
+/* Algorithm 1, line 6: once the mean is complete (stream-ordered wait, the host does not
+ * block), x^i <- x_hat_t + (x^i - x_t^i) for every worker.  Errors: STATE without a begin. */
+int cocod_comm_end(cocod_handle *h);
+
+/* ---------------------------------------------------------------------------------------------
+ * Additions the five calls above need around them (initial point, results, schedule).      */
+
+/* Stream for local steps, stored copies and merges (borrowed).  Not while a communication is
+ * in flight (STATE). */
+int cocod_set_stream(cocod_handle *h, cocod_stream_t compute);
+
+/* "Initialize: x_i^0 = x_hat_0": broadcast P values to all K workers.  on_host selects what
+ * kind of pointer x0 is.  Stream-ordered on the compute stream (host sources are copied
+ * synchronously first).  Not while a communication is in flight (STATE). */
+int cocod_set_params(cocod_handle *h, const float *x0, int on_host);
+
+/* Set / get all K x P models, the momentum, and the last average model (P values).  The get
+ * calls with on_host = 1 block until the data is in `out`; with on_host = 0 they are ordered on
+ * the compute stream.  set_* are not legal while a communication is in flight (STATE). */
+int cocod_set_params_all(cocod_handle *h, const float *x, int on_host);
+int cocod_set_momentum(cocod_handle *h, const float *v, int on_host);
+int cocod_get_params(cocod_handle *h, float *out, int on_host);
+int cocod_get_momentum(cocod_handle *h, float *out, int on_host);
+int cocod_get_mean(cocod_handle *h, float *out, int on_host);
+
+/* The paper changes gamma during a run (warm-up, decay at epoch 81; Section 5.1). */
+int cocod_set_lr(cocod_handle *h, float lr);
+
+/* Mini-batch sizes M_1..M_K of Algorithm 1 ("proportionally sampling", Section 3.2): the mean
+ * uses weights M_i / sum_j M_j.  M: host, K positive finite values; NULL = all equal. */
+int cocod_set_batch_sizes(cocod_handle *h, const double *M);
+
+int cocod_set_option(cocod_handle *h, int option, int value);
+
+/* Block the host until all of the engine's device work is done.  Returns the sticky error. */
+int cocod_sync(cocod_handle *h);
+
+/* Poll (no device-side waiting) until the mean started by comm_begin is complete or
+ * timeout_ms has passed: OK, TIMEOUT, or STATE if nothing is in flight. */
+int cocod_comm_wait(cocod_handle *h, int timeout_ms);
+
+/* Number of local steps taken so far (the paper's iteration counter t). */
+int64_t cocod_step_count(const cocod_handle *h);
+
+/* The cudaError_t of the first failed CUDA call on this handle (0 if none). */
+int cocod_last_cuda_error(const cocod_handle *h);
+
+const char *cocod_strerror(int code);
+
+/* ---------------------------------------------------------------------------------------------
+ * Profiling (COCOD_OPT_PROFILE = 1): the engine brackets each of its kernels with CUDA events.
+ * cocod_profile_count syncs the device and returns how many records exist (at most 4096 since
+ * the last reset); cocod_profile_get returns record i: the kernel kind and its start/end in
+ * milliseconds relative to the first record's start.  Used to report per-kernel bandwidth and
+ * how much of the mean kernel's lifetime overlaps local steps. */
+int cocod_profile_reset(cocod_handle *h);
+int cocod_profile_count(cocod_handle *h);
+int cocod_profile_get(cocod_handle *h, int i, int *kind, float *start_ms, float *end_ms);
+
+/* Number of kernels this handle has launched since creation (all kinds). */
+int64_t cocod_launch_count(const cocod_handle *h);
+
+/* ---------------------------------------------------------------------------------------------
+ * The four kernels on caller-owned device buffers (no handle, no state): the same code the
+ * engine launches, exposed for per-kernel measurement and tests.  All pointers: device, fp32.
+ *   local_step: n = number of elements; x_out may equal x_in (in place).
+ *   mean:       w = K device weights, or NULL for the plain mean.
+ *   merge:      x (K x P) updated in place from snap (K x P) and mean (P).              */
+int cocod_kernel_local_step(const float *x_in, float *x_out, float *v, const float *g, int64_t n,
+                            float lr, float mu, float wd, cocod_stream_t stream);
+int cocod_kernel_snapshot(const float *x, float *snap, int64_t n, cocod_stream_t stream);
+int cocod_kernel_mean(const float *snap, int K, int64_t P, const float *w, float *mean,
+                      cocod_stream_t stream);
+int cocod_kernel_merge(float *x, const float *snap, const float *mean, int K, int64_t P,
+                       cocod_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COCOD_H */

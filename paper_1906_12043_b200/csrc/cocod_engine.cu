@@ -1,0 +1,620 @@
+// libcocod.so: host side of the CoCoD-SGD parameter engine -- state machine, stream/event
+// plumbing and kernel launches behind the C boundary declared in include/cocod.h.
+//
+// One round of Algorithm 1 (arxiv 1906.12043) maps to
+//   comm_begin : [compute] stored copy (copy kernel, or buffer flip) -> ev_snap
+//                [side]    wait ev_snap -> mean kernel -> ev_mean
+//   local_step : [compute] fused momentum-SGD kernel over the flat K*P vector, k times
+//   comm_end   : [compute] wait ev_mean -> merge kernel
+// Ordering is by stream events only; no kernel spins on another and the host never blocks
+// inside a round.
+#include "cocod.h"
+#include "cocod_kernels.cuh"
+
+#include <algorithm>
+#include <chrono>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <thread>
+#include <vector>
+
+namespace {
+
+constexpr int kMaxWorkers = 1024;
+constexpr int kMaxProfile = 4096;
+constexpr int64_t kHostChunk = int64_t(1) << 24;   // elements per staged host->device chunk (64 MiB)
+constexpr int kHostSlots = 2;
+
+enum State { IDLE = 0, IN_FLIGHT = 1 };
+
+struct ProfileRec {
+    int kind;
+    cudaEvent_t a, b;
+};
+
+}  // namespace
+
+struct cocod_engine {
+    int K = 0;
+    int64_t P = 0, n = 0;
+    float lr = 0, mu = 0, wd = 0;
+    int device = 0;
+    // buf[cur] holds x; buf[1 - cur] holds the stored copies (or is spare between rounds)
+    float *buf[2] = {nullptr, nullptr};
+    int cur = 0;
+    float *v = nullptr, *mean = nullptr, *w = nullptr;
+    bool weighted = false;
+    const float *snap = nullptr;       // where this round's stored copies live
+    bool pending_flip = false;          // FLIP mode: x still lives in the stored-copy buffer
+    bool mean_valid = false;
+    int state = IDLE;
+    int snapshot_mode = COCOD_SNAPSHOT_FLIP;
+    cudaStream_t compute = nullptr, side = nullptr, copy = nullptr;
+    cudaEvent_t ev_snap = nullptr, ev_mean = nullptr, ev_tmp = nullptr;
+    // staging for host gradients
+    float *stage[kHostSlots] = {nullptr, nullptr};
+    cudaEvent_t ev_copied[kHostSlots] = {nullptr, nullptr}, ev_consumed[kHostSlots] = {nullptr, nullptr};
+    bool slot_used[kHostSlots] = {false, false};
+    // bookkeeping
+    int64_t steps = 0, launches = 0;
+    int cuda_error = 0;
+    bool profile = false;
+    std::vector<ProfileRec> prof;
+    std::vector<cudaEvent_t> ev_pool;
+};
+
+namespace {
+
+inline bool fail(cocod_engine *h, cudaError_t e)
+{
+    if (e == cudaSuccess) return false;
+    if (h && h->cuda_error == 0) h->cuda_error = (int)e;
+    return true;
+}
+#define CK(h, call) do { if (fail((h), (call))) return COCOD_ERR_CUDA; } while (0)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline unsigned grid_for(int64_t items, int per_block)
+{
+    return (unsigned)((items + per_block - 1) / per_block);
+}
+
+// ---------------------------------------------------------------- launchers (shared with the stateless entry points)
+cudaError_t launch_local_step(const float *x_in, float *x_out, float *v, const float *g, int64_t n,
+                              float lr, float mu, float wd, cudaStream_t s, int *n_launch)
+{
+    using namespace cocod;
+    if (n <= 0) return cudaSuccess;
+    constexpr int UNROLL = 4;
+    int64_t done = 0;
+    if (aligned16(x_in) && aligned16(x_out) && aligned16(v) && aligned16(g) && n >= 4) {
+        const int64_t nvec = n / 4;
+        local_step_vec4<UNROLL><<<grid_for(nvec, kThreads * UNROLL), kThreads, 0, s>>>(
+            reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
+            reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd);
+        done = nvec * 4;
+        if (n_launch) ++*n_launch;
+    }
+    if (done < n) {
+        const int64_t rest = n - done;
+        const unsigned grid = (unsigned)std::min<int64_t>((rest + kThreads - 1) / kThreads, 148 * 8);
+        local_step_scalar<<<grid, kThreads, 0, s>>>(x_in, x_out, v, g, done, rest, lr, mu, wd);
+        if (n_launch) ++*n_launch;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_snapshot(const float *x, float *snap, int64_t n, cudaStream_t s, int *n_launch)
+{
+    using namespace cocod;
+    if (n <= 0) return cudaSuccess;
+    constexpr int UNROLL = 4;
+    int64_t done = 0;
+    if (aligned16(x) && aligned16(snap) && n >= 4) {
+        const int64_t nvec = n / 4;
+        snapshot_vec4<UNROLL><<<grid_for(nvec, kThreads * UNROLL), kThreads, 0, s>>>(
+            reinterpret_cast<const float4 *>(x), reinterpret_cast<float4 *>(snap), nvec);
+        done = nvec * 4;
+        if (n_launch) ++*n_launch;
+    }
+    if (done < n) {
+        const int64_t rest = n - done;
+        const unsigned grid = (unsigned)std::min<int64_t>((rest + kThreads - 1) / kThreads, 148 * 8);
+        snapshot_scalar<<<grid, kThreads, 0, s>>>(x, snap, done, rest);
+        if (n_launch) ++*n_launch;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, float *mean, cudaStream_t s,
+                        int *n_launch)
+{
+    using namespace cocod;
+    const float inv_k = 1.0f / (float)K;
+    if ((P % 4) == 0 && aligned16(snap) && aligned16(mean)) {
+        const int64_t pvec = P / 4;
+        mean_vec4<8><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
+            reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k);
+    } else {
+        mean_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
+    }
+    if (n_launch) ++*n_launch;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, int64_t P, cudaStream_t s,
+                         int *n_launch)
+{
+    using namespace cocod;
+    if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean)) {
+        const int64_t pvec = P / 4;
+        merge_vec4<4><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
+            reinterpret_cast<float4 *>(x), reinterpret_cast<const float4 *>(snap),
+            reinterpret_cast<const float4 *>(mean), K, pvec);
+    } else {
+        merge_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(x, snap, mean, K, P);
+    }
+    if (n_launch) ++*n_launch;
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- profiling brackets
+struct Bracket {
+    cocod_engine *h;
+    cudaStream_t s;
+    int kind;
+    cudaEvent_t a = nullptr, b = nullptr;
+    bool on = false;
+    Bracket(cocod_engine *h_, cudaStream_t s_, int kind_) : h(h_), s(s_), kind(kind_)
+    {
+        if (!h->profile || (int)h->prof.size() >= kMaxProfile) return;
+        if (cudaEventCreate(&a) != cudaSuccess) { a = nullptr; return; }
+        if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); a = b = nullptr; return; }
+        on = true;
+        cudaEventRecord(a, s);
+    }
+    ~Bracket()
+    {
+        if (!on) return;
+        cudaEventRecord(b, s);
+        h->prof.push_back({kind, a, b});
+    }
+};
+
+void profile_clear(cocod_engine *h)
+{
+    for (auto &r : h->prof) {
+        cudaEventDestroy(r.a);
+        cudaEventDestroy(r.b);
+    }
+    h->prof.clear();
+}
+
+int check_live(const cocod_engine *h)
+{
+    if (!h) return COCOD_ERR_INVALID;
+    if (h->cuda_error) return COCOD_ERR_CUDA;
+    return COCOD_OK;
+}
+
+void free_all(cocod_engine *h)
+{
+    profile_clear(h);
+    for (int i = 0; i < 2; ++i) if (h->buf[i]) cudaFree(h->buf[i]);
+    if (h->v) cudaFree(h->v);
+    if (h->mean) cudaFree(h->mean);
+    if (h->w) cudaFree(h->w);
+    for (int i = 0; i < kHostSlots; ++i) {
+        if (h->stage[i]) cudaFree(h->stage[i]);
+        if (h->ev_copied[i]) cudaEventDestroy(h->ev_copied[i]);
+        if (h->ev_consumed[i]) cudaEventDestroy(h->ev_consumed[i]);
+    }
+    if (h->ev_snap) cudaEventDestroy(h->ev_snap);
+    if (h->ev_mean) cudaEventDestroy(h->ev_mean);
+    if (h->ev_tmp) cudaEventDestroy(h->ev_tmp);
+    if (h->copy) cudaStreamDestroy(h->copy);
+    delete h;
+}
+
+// copy `bytes` into a device buffer from host or device memory, ordered on the compute stream
+int copy_in(cocod_engine *h, float *dst, const float *src, size_t bytes, int on_host)
+{
+    if (on_host) {
+        CK(h, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, h->compute));
+        CK(h, cudaStreamSynchronize(h->compute));
+    } else {
+        CK(h, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, h->compute));
+    }
+    return COCOD_OK;
+}
+
+int copy_out(cocod_engine *h, float *dst, const float *src, size_t bytes, int on_host)
+{
+    if (on_host) {
+        CK(h, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, h->compute));
+        CK(h, cudaStreamSynchronize(h->compute));
+    } else {
+        CK(h, cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, h->compute));
+    }
+    return COCOD_OK;
+}
+
+// One local step over elements [off, off + len) with gradients at g (already offset).
+int step_range(cocod_engine *h, const float *g, int64_t off, int64_t len)
+{
+    const float *x_in = h->buf[h->cur] + off;
+    float *x_out = (h->pending_flip ? h->buf[1 - h->cur] : h->buf[h->cur]) + off;
+    int nl = 0;
+    {
+        Bracket br(h, h->compute, COCOD_KERNEL_LOCAL_STEP);
+        CK(h, launch_local_step(x_in, x_out, h->v + off, g, len, h->lr, h->mu, h->wd, h->compute, &nl));
+    }
+    h->launches += nl;
+    return COCOD_OK;
+}
+
+void finish_step(cocod_engine *h)
+{
+    if (h->pending_flip) {      // x now lives in the other buffer; the old one stays as stored copy
+        h->cur = 1 - h->cur;
+        h->pending_flip = false;
+    }
+    ++h->steps;
+}
+
+}  // namespace
+
+extern "C" {
+
+int cocod_create(cocod_handle **out, int K, int64_t P, float lr, float mu, float wd)
+{
+    if (!out || K < 1 || K > kMaxWorkers || P < 1) return COCOD_ERR_INVALID;
+    if (!std::isfinite(lr) || !std::isfinite(mu) || !std::isfinite(wd)) return COCOD_ERR_INVALID;
+    if (P > (INT64_MAX / 4) / K) return COCOD_ERR_INVALID;
+    cocod_engine *h = new (std::nothrow) cocod_engine();
+    if (!h) return COCOD_ERR_OOM;
+    h->K = K; h->P = P; h->n = (int64_t)K * P;
+    h->lr = lr; h->mu = mu; h->wd = wd;
+    if (cudaGetDevice(&h->device) != cudaSuccess) { cudaGetLastError(); delete h; return COCOD_ERR_CUDA; }
+    const size_t bytes = (size_t)h->n * sizeof(float);
+    cudaError_t e = cudaSuccess;
+    auto alloc = [&](float **p, size_t b) { if (e == cudaSuccess) e = cudaMalloc((void **)p, b); };
+    alloc(&h->buf[0], bytes);
+    alloc(&h->buf[1], bytes);
+    alloc(&h->v, bytes);
+    alloc(&h->mean, (size_t)P * sizeof(float));
+    alloc(&h->w, (size_t)K * sizeof(float));
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_snap, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_mean, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_tmp, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->buf[0], 0, bytes, h->compute);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->v, 0, bytes, h->compute);
+    if (e == cudaSuccess) e = cudaMemsetAsync(h->mean, 0, (size_t)P * sizeof(float), h->compute);
+    if (e != cudaSuccess) {
+        const int rc = (e == cudaErrorMemoryAllocation) ? COCOD_ERR_OOM : COCOD_ERR_CUDA;
+        cudaGetLastError();
+        free_all(h);
+        return rc;
+    }
+    *out = h;
+    return COCOD_OK;
+}
+
+int cocod_destroy(cocod_handle *h)
+{
+    if (!h) return COCOD_OK;
+    cudaStreamSynchronize(h->compute);
+    if (h->side) cudaStreamSynchronize(h->side);
+    if (h->copy) cudaStreamSynchronize(h->copy);
+    const int rc = h->cuda_error ? COCOD_ERR_CUDA : COCOD_OK;
+    free_all(h);
+    return rc;
+}
+
+int cocod_local_step(cocod_handle *h, const float *grads)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!grads) return COCOD_ERR_INVALID;
+    if (int rc = step_range(h, grads, 0, h->n)) return rc;
+    finish_step(h);
+    return COCOD_OK;
+}
+
+int cocod_local_step_host(cocod_handle *h, const float *host_grads)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!host_grads) return COCOD_ERR_INVALID;
+    if (!h->copy) {
+        CK(h, cudaStreamCreateWithFlags(&h->copy, cudaStreamNonBlocking));
+        const int64_t cap = std::min<int64_t>(kHostChunk, h->n);
+        for (int i = 0; i < kHostSlots; ++i) {
+            cudaError_t e = cudaMalloc((void **)&h->stage[i], (size_t)cap * sizeof(float));
+            if (e != cudaSuccess) { cudaGetLastError(); return COCOD_ERR_OOM; }
+            CK(h, cudaEventCreateWithFlags(&h->ev_copied[i], cudaEventDisableTiming));
+            CK(h, cudaEventCreateWithFlags(&h->ev_consumed[i], cudaEventDisableTiming));
+        }
+    }
+    int slot = 0;
+    for (int64_t off = 0; off < h->n; off += kHostChunk, slot = (slot + 1) % kHostSlots) {
+        const int64_t len = std::min<int64_t>(kHostChunk, h->n - off);
+        if (h->slot_used[slot]) CK(h, cudaStreamWaitEvent(h->copy, h->ev_consumed[slot], 0));
+        CK(h, cudaMemcpyAsync(h->stage[slot], host_grads + off, (size_t)len * sizeof(float),
+                              cudaMemcpyHostToDevice, h->copy));
+        CK(h, cudaEventRecord(h->ev_copied[slot], h->copy));
+        CK(h, cudaStreamWaitEvent(h->compute, h->ev_copied[slot], 0));
+        if (int rc = step_range(h, h->stage[slot], off, len)) return rc;
+        CK(h, cudaEventRecord(h->ev_consumed[slot], h->compute));
+        h->slot_used[slot] = true;
+    }
+    finish_step(h);
+    return COCOD_OK;
+}
+
+int cocod_comm_begin(cocod_handle *h, cocod_stream_t side)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    h->side = (cudaStream_t)side;
+    if (h->snapshot_mode == COCOD_SNAPSHOT_FLIP) {
+        h->snap = h->buf[h->cur];
+        h->pending_flip = true;
+    } else {
+        float *dst = h->buf[1 - h->cur];
+        int nl = 0;
+        {
+            Bracket br(h, h->compute, COCOD_KERNEL_SNAPSHOT);
+            CK(h, launch_snapshot(h->buf[h->cur], dst, h->n, h->compute, &nl));
+        }
+        h->launches += nl;
+        h->snap = dst;
+        h->pending_flip = false;
+    }
+    if (h->side != h->compute) {
+        CK(h, cudaEventRecord(h->ev_snap, h->compute));
+        CK(h, cudaStreamWaitEvent(h->side, h->ev_snap, 0));
+    }
+    int nl = 0;
+    {
+        Bracket br(h, h->side, COCOD_KERNEL_MEAN);
+        CK(h, launch_mean(h->snap, h->K, h->P, h->weighted ? h->w : nullptr, h->mean, h->side, &nl));
+    }
+    h->launches += nl;
+    CK(h, cudaEventRecord(h->ev_mean, h->side));
+    h->mean_valid = true;
+    h->state = IN_FLIGHT;
+    return COCOD_OK;
+}
+
+int cocod_comm_end(cocod_handle *h)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IN_FLIGHT) return COCOD_ERR_STATE;
+    if (h->side != h->compute) CK(h, cudaStreamWaitEvent(h->compute, h->ev_mean, 0));
+    int nl = 0;
+    {
+        Bracket br(h, h->compute, COCOD_KERNEL_MERGE);
+        // with no local step since comm_begin (FLIP) x still aliases the stored copies
+        CK(h, launch_merge(h->buf[h->cur], h->snap, h->mean, h->K, h->P, h->compute, &nl));
+    }
+    h->launches += nl;
+    h->pending_flip = false;
+    h->snap = nullptr;
+    h->state = IDLE;
+    return COCOD_OK;
+}
+
+int cocod_set_stream(cocod_handle *h, cocod_stream_t compute)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    cudaStream_t s = (cudaStream_t)compute;
+    if (s != h->compute) {      // later work on the new stream stays ordered after earlier work
+        CK(h, cudaEventRecord(h->ev_tmp, h->compute));
+        CK(h, cudaStreamWaitEvent(s, h->ev_tmp, 0));
+        h->compute = s;
+    }
+    return COCOD_OK;
+}
+
+int cocod_set_params(cocod_handle *h, const float *x0, int on_host)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!x0) return COCOD_ERR_INVALID;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    const float *src = x0;
+    if (on_host) {      // stage through the (idle) average-model buffer
+        if (int rc = copy_in(h, h->mean, x0, (size_t)h->P * sizeof(float), 1)) return rc;
+        src = h->mean;
+        h->mean_valid = false;
+    }
+    cocod::broadcast_rows<<<grid_for(h->P, cocod::kThreads), cocod::kThreads, 0, h->compute>>>(
+        src, h->buf[h->cur], h->K, h->P);
+    CK(h, cudaGetLastError());
+    ++h->launches;
+    return COCOD_OK;
+}
+
+int cocod_set_params_all(cocod_handle *h, const float *x, int on_host)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!x) return COCOD_ERR_INVALID;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    return copy_in(h, h->buf[h->cur], x, (size_t)h->n * sizeof(float), on_host);
+}
+
+int cocod_set_momentum(cocod_handle *h, const float *v, int on_host)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!v) return COCOD_ERR_INVALID;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    return copy_in(h, h->v, v, (size_t)h->n * sizeof(float), on_host);
+}
+
+int cocod_get_params(cocod_handle *h, float *out, int on_host)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!out) return COCOD_ERR_INVALID;
+    return copy_out(h, out, h->buf[h->cur], (size_t)h->n * sizeof(float), on_host);
+}
+
+int cocod_get_momentum(cocod_handle *h, float *out, int on_host)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!out) return COCOD_ERR_INVALID;
+    return copy_out(h, out, h->v, (size_t)h->n * sizeof(float), on_host);
+}
+
+int cocod_get_mean(cocod_handle *h, float *out, int on_host)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!out) return COCOD_ERR_INVALID;
+    if (!h->mean_valid) return COCOD_ERR_STATE;
+    if (h->side != h->compute) CK(h, cudaStreamWaitEvent(h->compute, h->ev_mean, 0));
+    return copy_out(h, out, h->mean, (size_t)h->P * sizeof(float), on_host);
+}
+
+int cocod_set_lr(cocod_handle *h, float lr)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!std::isfinite(lr)) return COCOD_ERR_INVALID;
+    h->lr = lr;
+    return COCOD_OK;
+}
+
+int cocod_set_batch_sizes(cocod_handle *h, const double *M)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    if (!M) { h->weighted = false; return COCOD_OK; }
+    double sum = 0.0;
+    for (int i = 0; i < h->K; ++i) {
+        if (!(M[i] > 0.0) || !std::isfinite(M[i])) return COCOD_ERR_INVALID;
+        sum += M[i];
+    }
+    float w[kMaxWorkers];
+    for (int i = 0; i < h->K; ++i) w[i] = (float)(M[i] / sum);
+    CK(h, cudaMemcpyAsync(h->w, w, (size_t)h->K * sizeof(float), cudaMemcpyHostToDevice, h->compute));
+    CK(h, cudaStreamSynchronize(h->compute));      // w[] is a stack buffer
+    h->weighted = true;
+    return COCOD_OK;
+}
+
+int cocod_set_option(cocod_handle *h, int option, int value)
+{
+    if (int rc = check_live(h)) return rc;
+    switch (option) {
+    case COCOD_OPT_SNAPSHOT:
+        if (value != COCOD_SNAPSHOT_COPY && value != COCOD_SNAPSHOT_FLIP) return COCOD_ERR_INVALID;
+        if (h->state != IDLE) return COCOD_ERR_STATE;
+        h->snapshot_mode = value;
+        return COCOD_OK;
+    case COCOD_OPT_PROFILE:
+        h->profile = value != 0;
+        return COCOD_OK;
+    default:
+        return COCOD_ERR_INVALID;
+    }
+}
+
+int cocod_sync(cocod_handle *h)
+{
+    if (!h) return COCOD_ERR_INVALID;
+    fail(h, cudaStreamSynchronize(h->compute));
+    if (h->side && h->side != h->compute) fail(h, cudaStreamSynchronize(h->side));
+    if (h->copy) fail(h, cudaStreamSynchronize(h->copy));
+    return h->cuda_error ? COCOD_ERR_CUDA : COCOD_OK;
+}
+
+int cocod_comm_wait(cocod_handle *h, int timeout_ms)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IN_FLIGHT) return COCOD_ERR_STATE;
+    const auto t0 = std::chrono::steady_clock::now();
+    for (;;) {
+        cudaError_t e = cudaEventQuery(h->ev_mean);
+        if (e == cudaSuccess) return COCOD_OK;
+        if (e != cudaErrorNotReady) { fail(h, e); return COCOD_ERR_CUDA; }
+        cudaGetLastError();
+        const auto ms = std::chrono::duration_cast<std::chrono::milliseconds>(
+                            std::chrono::steady_clock::now() - t0).count();
+        if (ms >= timeout_ms) return COCOD_ERR_TIMEOUT;
+        std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+}
+
+int64_t cocod_step_count(const cocod_handle *h) { return h ? h->steps : -1; }
+
+int cocod_last_cuda_error(const cocod_handle *h) { return h ? h->cuda_error : 0; }
+
+int64_t cocod_launch_count(const cocod_handle *h) { return h ? h->launches : -1; }
+
+const char *cocod_strerror(int code)
+{
+    switch (code) {
+    case COCOD_OK: return "ok";
+    case COCOD_ERR_INVALID: return "invalid argument";
+    case COCOD_ERR_OOM: return "out of memory";
+    case COCOD_ERR_STATE: return "call not legal in the engine's current state";
+    case COCOD_ERR_CUDA: return "CUDA error";
+    case COCOD_ERR_TIMEOUT: return "timed out";
+    default: return "unknown error code";
+    }
+}
+
+int cocod_profile_reset(cocod_handle *h)
+{
+    if (int rc = check_live(h)) return rc;
+    if (int rc = cocod_sync(h)) return rc;
+    profile_clear(h);
+    return COCOD_OK;
+}
+
+int cocod_profile_count(cocod_handle *h)
+{
+    if (int rc = check_live(h)) return rc;
+    if (int rc = cocod_sync(h)) return rc;
+    return (int)h->prof.size();
+}
+
+int cocod_profile_get(cocod_handle *h, int i, int *kind, float *start_ms, float *end_ms)
+{
+    if (int rc = check_live(h)) return rc;
+    if (i < 0 || i >= (int)h->prof.size() || !kind || !start_ms || !end_ms) return COCOD_ERR_INVALID;
+    const ProfileRec &r = h->prof[i];
+    *kind = r.kind;
+    CK(h, cudaEventElapsedTime(start_ms, h->prof[0].a, r.a));
+    CK(h, cudaEventElapsedTime(end_ms, h->prof[0].a, r.b));
+    return COCOD_OK;
+}
+
+// ------------------------------------------------------------------ stateless kernel entry points
+int cocod_kernel_local_step(const float *x_in, float *x_out, float *v, const float *g, int64_t n,
+                            float lr, float mu, float wd, cocod_stream_t stream)
+{
+    if (!x_in || !x_out || !v || !g || n < 0) return COCOD_ERR_INVALID;
+    return launch_local_step(x_in, x_out, v, g, n, lr, mu, wd, (cudaStream_t)stream, nullptr) == cudaSuccess
+               ? COCOD_OK : COCOD_ERR_CUDA;
+}
+
+int cocod_kernel_snapshot(const float *x, float *snap, int64_t n, cocod_stream_t stream)
+{
+    if (!x || !snap || n < 0) return COCOD_ERR_INVALID;
+    return launch_snapshot(x, snap, n, (cudaStream_t)stream, nullptr) == cudaSuccess ? COCOD_OK : COCOD_ERR_CUDA;
+}
+
+int cocod_kernel_mean(const float *snap, int K, int64_t P, const float *w, float *mean, cocod_stream_t stream)
+{
+    if (!snap || !mean || K < 1 || P < 1) return COCOD_ERR_INVALID;
+    return launch_mean(snap, K, P, w, mean, (cudaStream_t)stream, nullptr) == cudaSuccess ? COCOD_OK : COCOD_ERR_CUDA;
+}
+
+int cocod_kernel_merge(float *x, const float *snap, const float *mean, int K, int64_t P, cocod_stream_t stream)
+{
+    if (!x || !snap || !mean || K < 1 || P < 1) return COCOD_ERR_INVALID;
+    return launch_merge(x, snap, mean, K, P, (cudaStream_t)stream, nullptr) == cudaSuccess ? COCOD_OK : COCOD_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,243 @@
+// Device kernels of the CoCoD-SGD parameter path (Algorithm 1 of arxiv 1906.12043) for sm_100a.
+//
+// All four are HBM-bandwidth-bound streaming kernels (0.2-0.3 flop per byte): the design
+// goal is full-width coalesced 128-bit accesses, enough independent loads in flight per SM to
+// cover HBM latency, and no byte moved twice.  K x P matrices are worker-major row-major fp32
+// with row stride P.
+//
+// Arithmetic order is fixed (and mirrored by the test oracle's fp32 mode, so results can be
+// compared bit for bit):
+//   local step : d = fma(wd, x, g) ; v = fma(mu, v, d) ; x = fma(-lr, v, x)
+//   mean       : uniform  s = snap_0 ; s = s + snap_i (i = 1..K-1) ; mean = s * (1/K)
+//                weighted s = w_0 * snap_0 ; s = fma(w_i, snap_i, s)
+//   merge      : x = mean + (x - snap)
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cocod {
+
+constexpr int kThreads = 256;
+
+// ------------------------------------------------------------------------------------------ loads / stores
+// g is read exactly once per step: stream it past L1 and mark it evict-first in L2.
+__device__ __forceinline__ float4 ld_stream(const float4 *p)
+{
+    return __ldcs(p);
+}
+__device__ __forceinline__ float4 ld_plain(const float4 *p) { return *p; }
+__device__ __forceinline__ void st_plain(float4 *p, float4 v) { *p = v; }
+
+__device__ __forceinline__ void sgd_update(float4 &x, float4 &v, const float4 &g, float lr, float mu, float wd)
+{
+    float d;
+    d = __fmaf_rn(wd, x.x, g.x); v.x = __fmaf_rn(mu, v.x, d); x.x = __fmaf_rn(-lr, v.x, x.x);
+    d = __fmaf_rn(wd, x.y, g.y); v.y = __fmaf_rn(mu, v.y, d); x.y = __fmaf_rn(-lr, v.y, x.y);
+    d = __fmaf_rn(wd, x.z, g.z); v.z = __fmaf_rn(mu, v.z, d); x.z = __fmaf_rn(-lr, v.z, x.z);
+    d = __fmaf_rn(wd, x.w, g.w); v.w = __fmaf_rn(mu, v.w, d); x.w = __fmaf_rn(-lr, v.w, x.w);
+}
+
+// ------------------------------------------------------------------------------------------ local step (Step II)
+// One CTA owns a contiguous tile of kThreads * UNROLL float4 of the flat K*P vector: all
+// 3 * UNROLL loads of a thread are issued before the first use.  x_in may equal x_out.
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__restrict__ g,
+                int64_t nvec, float lr, float mu, float wd)
+{
+    const int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
+    float4 xr[UNROLL], vr[UNROLL], gr[UNROLL];
+    if (base + (int64_t)(UNROLL - 1) * kThreads < nvec) {       // full tile: no predicates
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int64_t i = base + (int64_t)u * kThreads;
+            gr[u] = ld_stream(g + i);
+            xr[u] = ld_plain(x_in + i);
+            vr[u] = ld_plain(v + i);
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int64_t i = base + (int64_t)u * kThreads;
+            sgd_update(xr[u], vr[u], gr[u], lr, mu, wd);
+            st_plain(v + i, vr[u]);
+            st_plain(x_out + i, xr[u]);
+        }
+    } else {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int64_t i = base + (int64_t)u * kThreads;
+            if (i < nvec) {
+                float4 xx = ld_plain(x_in + i), vv = ld_plain(v + i), gg = ld_stream(g + i);
+                sgd_update(xx, vv, gg, lr, mu, wd);
+                st_plain(v + i, vv);
+                st_plain(x_out + i, xx);
+            }
+        }
+    }
+}
+
+// Scalar path: misaligned pointers and the n mod 4 tail.  Elements [first, first + count).
+__global__ void __launch_bounds__(kThreads)
+local_step_scalar(const float *x_in, float *x_out, float *v, const float *__restrict__ g,
+                  int64_t first, int64_t count, float lr, float mu, float wd)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += stride) {
+        const int64_t e = first + j;
+        const float d = __fmaf_rn(wd, x_in[e], g[e]);
+        const float vn = __fmaf_rn(mu, v[e], d);
+        v[e] = vn;
+        x_out[e] = __fmaf_rn(-lr, vn, x_in[e]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------ stored copy (Step I)
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+snapshot_vec4(const float4 *__restrict__ x, float4 *__restrict__ snap, int64_t nvec)
+{
+    const int64_t base = (int64_t)blockIdx.x * (kThreads * UNROLL) + threadIdx.x;
+    float4 r[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        const int64_t i = base + (int64_t)u * kThreads;
+        if (i < nvec) r[u] = ld_plain(x + i);
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        const int64_t i = base + (int64_t)u * kThreads;
+        if (i < nvec) st_plain(snap + i, r[u]);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+snapshot_scalar(const float *__restrict__ x, float *__restrict__ snap, int64_t first, int64_t count)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += stride)
+        snap[first + j] = x[first + j];
+}
+
+// ------------------------------------------------------------------------------------------ average model (Step I)
+// One thread owns one float4 of columns and walks the K rows in order, RC row loads in flight
+// at a time (RC * 16 B per thread).  Needs P mod 4 == 0 and 16-byte aligned bases.
+template <int RC>
+__global__ void __launch_bounds__(kThreads)
+mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__restrict__ w,
+          float4 *__restrict__ mean, float inv_k)
+{
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= pvec) return;
+    const float4 *col = snap + c;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i0 = 0; i0 < K; i0 += RC) {
+        float4 r[RC];
+#pragma unroll
+        for (int j = 0; j < RC; ++j)
+            if (i0 + j < K) r[j] = ld_stream(col + (int64_t)(i0 + j) * pvec);
+#pragma unroll
+        for (int j = 0; j < RC; ++j) {
+            const int i = i0 + j;
+            if (i < K) {
+                if (w != nullptr) {
+                    const float wi = __ldg(w + i);
+                    if (i == 0) {
+                        s.x = __fmul_rn(wi, r[j].x); s.y = __fmul_rn(wi, r[j].y);
+                        s.z = __fmul_rn(wi, r[j].z); s.w = __fmul_rn(wi, r[j].w);
+                    } else {
+                        s.x = __fmaf_rn(wi, r[j].x, s.x); s.y = __fmaf_rn(wi, r[j].y, s.y);
+                        s.z = __fmaf_rn(wi, r[j].z, s.z); s.w = __fmaf_rn(wi, r[j].w, s.w);
+                    }
+                } else {
+                    if (i == 0) s = r[j];
+                    else {
+                        s.x = __fadd_rn(s.x, r[j].x); s.y = __fadd_rn(s.y, r[j].y);
+                        s.z = __fadd_rn(s.z, r[j].z); s.w = __fadd_rn(s.w, r[j].w);
+                    }
+                }
+            }
+        }
+    }
+    if (w == nullptr) {
+        s.x = __fmul_rn(s.x, inv_k); s.y = __fmul_rn(s.y, inv_k);
+        s.z = __fmul_rn(s.z, inv_k); s.w = __fmul_rn(s.w, inv_k);
+    }
+    mean[c] = s;
+}
+
+// Any P / alignment: one thread per column, same row order.
+__global__ void __launch_bounds__(kThreads)
+mean_scalar(const float *__restrict__ snap, int K, int64_t P, const float *__restrict__ w,
+            float *__restrict__ mean, float inv_k)
+{
+    const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (p >= P) return;
+    float s;
+    if (w != nullptr) {
+        s = __fmul_rn(__ldg(w), snap[p]);
+        for (int i = 1; i < K; ++i) s = __fmaf_rn(__ldg(w + i), snap[(int64_t)i * P + p], s);
+    } else {
+        s = snap[p];
+        for (int i = 1; i < K; ++i) s = __fadd_rn(s, snap[(int64_t)i * P + p]);
+        s = __fmul_rn(s, inv_k);
+    }
+    mean[p] = s;
+}
+
+// ------------------------------------------------------------------------------------------ merge (line 6)
+// Same column ownership: the average is read once per column (4/K B per worker-parameter) and
+// reused for all K rows; RC rows (2 * RC loads) in flight per thread.  x may alias snap (a
+// merge with no local step in between): every element is read before it is written.
+template <int RC>
+__global__ void __launch_bounds__(kThreads)
+merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K, int64_t pvec)
+{
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= pvec) return;
+    const float4 m = mean[c];
+    for (int i0 = 0; i0 < K; i0 += RC) {
+        float4 xr[RC], sr[RC];
+#pragma unroll
+        for (int j = 0; j < RC; ++j)
+            if (i0 + j < K) {
+                const int64_t e = (int64_t)(i0 + j) * pvec + c;
+                xr[j] = ld_plain(x + e);
+                sr[j] = ld_stream(snap + e);
+            }
+#pragma unroll
+        for (int j = 0; j < RC; ++j)
+            if (i0 + j < K) {
+                const int64_t e = (int64_t)(i0 + j) * pvec + c;
+                float4 o;
+                o.x = __fadd_rn(m.x, __fsub_rn(xr[j].x, sr[j].x));
+                o.y = __fadd_rn(m.y, __fsub_rn(xr[j].y, sr[j].y));
+                o.z = __fadd_rn(m.z, __fsub_rn(xr[j].z, sr[j].z));
+                o.w = __fadd_rn(m.w, __fsub_rn(xr[j].w, sr[j].w));
+                st_plain(x + e, o);
+            }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+merge_scalar(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P)
+{
+    const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (p >= P) return;
+    const float m = mean[p];
+    for (int i = 0; i < K; ++i) {
+        const int64_t e = (int64_t)i * P + p;
+        x[e] = __fadd_rn(m, __fsub_rn(x[e], snap[e]));
+    }
+}
+
+// Broadcast P values to K rows ("Initialize: x_i^0 = x_hat_0").
+__global__ void __launch_bounds__(kThreads)
+broadcast_rows(const float *__restrict__ x0, float *__restrict__ x, int K, int64_t P)
+{
+    const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (p >= P) return;
+    const float a = x0[p];
+    for (int i = 0; i < K; ++i) x[(int64_t)i * P + p] = a;
+}
+
+}  // namespace cocod

@@ -1,0 +1,116 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times (buffer
+flip, high-priority side stream, device-resident gradients): sampled columns against the
+oracle (every column of the K x P state is an independent problem, so the oracle can compute
+any subset exactly), plus properties that hold at any size."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle.cocod_oracle import OracleEngine
+from paper_1906_12043_b200 import inputs as I
+from paper_1906_12043_b200.workloads import WORKLOADS
+from test_gpu_parity import assert_bit_equal, assert_close_scaled, cpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_1906_12043_b200 import build, engine
+    build.build()
+    engine.load()
+    return engine
+
+
+def sample_columns(K, P, n_random, seed):
+    rng = np.random.default_rng(seed)
+    cols = set(range(0, 64)) | set(range(P - 64, P)) | set(int(c) for c in rng.integers(0, P, n_random))
+    for tile in (1024, 4096, 1 << 16, 1 << 24):          # tile edges of any plausible kernel shape
+        for m in (1, 2, 7):
+            for d in range(-4, 4):
+                c = tile * m + d
+                if 0 <= c < P:
+                    cols.add(c)
+    for flat in (1 << 31, 1 << 32):                        # flat index i * P + p crossing 2^31 / 2^32
+        for i in range(K):
+            for d in range(-8, 8):
+                p = flat + d - i * P
+                if 0 <= p < P:
+                    cols.add(int(p))
+    return np.array(sorted(cols), dtype=np.int64)
+
+
+def run_fullsize(E, wl, rounds, n_random, check_first_round=True):
+    K, P, k = wl.K, wl.P, wl.k
+    cols = sample_columns(K, P, n_random, seed=5)
+    cols_d = torch.from_numpy(cols).cuda()
+    eng = E.Engine(K, P, wl.lr, wl.mu, wl.wd)
+    x0 = torch.empty(P, dtype=torch.float32, device="cuda")
+    I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, 0, wl.sigma_x0)
+    eng.set_params(x0)
+    ref = OracleEngine(K, len(cols), wl.lr, wl.mu, wl.wd, mode="ref")
+    mir = OracleEngine(K, len(cols), wl.lr, wl.mu, wl.wd, mode="mirror")
+    x0_cols = I.initial_point(P, wl.sigma_x0, cols=cols)
+    assert_bit_equal(cpu(x0[cols_d]), x0_cols, "device x0 vs host recipe")
+    ref.set_params(x0_cols)
+    mir.set_params(x0_cols)
+    side = torch.cuda.Stream(priority=-1)
+    g = torch.empty((K, P), dtype=torch.float32, device="cuda")
+    scratch = torch.empty((K, P), dtype=torch.float32, device="cuda")
+
+    def gpu_cols(getter):
+        getter(scratch)
+        return cpu(scratch[:, cols_d])
+
+    for r in range(rounds):
+        eng.comm_begin(side)
+        ref.comm_begin()
+        mir.comm_begin()
+        for s in range(k):
+            t = r * k + s
+            eng.sync()                       # g is reused: the previous step must have consumed it
+            I.device_gradients_into(g, t, wl.sigma_g)
+            gc = I.gradients(K, P, t, wl.sigma_g, cols=cols)
+            if t == 0:
+                assert_bit_equal(cpu(g[:, cols_d]), gc, "device gradients vs host recipe")
+            eng.local_step(g)
+            ref.local_step(gc)
+            mir.local_step(gc)
+        pre = None
+        if r == rounds - 1:                  # invariant at full size: line 6 keeps mean_i x_i
+            pre = eng.get_params(scratch).double().mean(0)
+        eng.comm_end()
+        ref.comm_end()
+        mir.comm_end()
+        if r == 0 and check_first_round:
+            assert_close_scaled(gpu_cols(eng.get_params), ref.x, 1e-6, "x after round 1")
+            assert_close_scaled(gpu_cols(eng.get_momentum), ref.v, 1e-6, "v after round 1")
+        if pre is not None:
+            post = eng.get_params(scratch).double().mean(0)
+            assert float((post - pre).abs().max()) < 2e-7
+    xs, vs = gpu_cols(eng.get_params), gpu_cols(eng.get_momentum)
+    ex = assert_close_scaled(xs, ref.x, 1e-5, "x after the run")
+    ev = assert_close_scaled(vs, ref.v, 1e-5, "v after the run")
+    assert_bit_equal(xs, mir.x, "x vs mirror")
+    assert_bit_equal(vs, mir.v, "v vs mirror")
+    assert_bit_equal(cpu(eng.get_mean()[cols_d]), mir.mean, "average model vs mirror")
+    assert torch.isfinite(eng.get_params(scratch)).all()
+    print(f"{wl.name}: {len(cols)} sampled columns x {K} workers, {rounds} rounds: "
+          f"max scaled err x {ex:.2e}, v {ev:.2e}")
+    eng.destroy()
+
+
+def test_resnet18_sized_full_run_sampled_columns(E):
+    """K=16, P=11,689,512, k=2, 50 rounds (the benchmark workload)."""
+    wl = WORKLOADS["resnet18"]
+    run_fullsize(E, wl, wl.rounds, n_random=4096)
+
+
+def test_vgg16_sized_sampled_columns_cross_the_2_31_flat_index(E):
+    """K=16, P=138,357,544 (K*P > 2^31): 64-bit indexing.  Needs about 45 GB of HBM."""
+    wl = WORKLOADS["vgg16"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 80e9:
+        pytest.skip("not enough free HBM for the VGG16-sized state")
+    run_fullsize(E, wl, rounds=5, n_random=2048)

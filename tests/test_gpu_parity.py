@@ -1,0 +1,418 @@
+"""GPU parity: the CUDA engine, called through the C boundary, against the CPU oracle on the
+same seeded inputs.
+
+Bars (fp32 path):
+  * against the oracle's "ref" mode (fp32-stored, fp64-evaluated): per element
+        |gpu - ref| <= rtol * max(|ref|, rms(ref))
+    with rtol 1e-6 after one round and 1e-5 after a full run, on x and on the momentum v;
+  * against the oracle's "mirror" mode (same fp32 operation order): bit for bit.
+"""
+import os
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle.cocod_oracle import OracleEngine
+from paper_1906_12043_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+@pytest.fixture(scope="module")
+def E():
+    from paper_1906_12043_b200 import build, engine
+    build.build()
+    engine.load()
+    return engine
+
+
+def assert_close_scaled(got, ref, rtol, what=""):
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    scale = np.maximum(np.abs(ref), np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(got - ref) / np.maximum(scale, 1e-300)
+    worst = float(err.max()) if err.size else 0.0
+    assert worst <= rtol, f"{what}: max scaled error {worst:.3e} > {rtol:.1e}"
+    return worst
+
+
+def assert_bit_equal(got, ref, what=""):
+    got = np.ascontiguousarray(got, np.float32).view(np.uint32)
+    ref = np.ascontiguousarray(ref, np.float32).view(np.uint32)
+    bad = np.nonzero(got != ref)
+    assert bad[0].size == 0, f"{what}: {bad[0].size} elements differ, first at {[b[0] for b in bad]}"
+
+
+def cpu(t):
+    return t.detach().cpu().numpy()
+
+
+def run_both(E, K, P, lr, mu, wd, k, rounds, x0, grad_fn, M=None, snapshot=None, side="own",
+             check_round=None):
+    """Drive the engine and both oracle modes with the same bytes; returns (eng, ref, mirror)."""
+    eng = E.Engine(K, P, lr, mu, wd)
+    if snapshot is not None:
+        eng.set_option(E.OPT_SNAPSHOT, snapshot)
+    if M is not None:
+        eng.set_batch_sizes(M)
+    eng.set_params(torch.from_numpy(x0).cuda())
+    side_stream = {"own": torch.cuda.Stream(), "same": None,
+                   "high": torch.cuda.Stream(priority=-1)}[side]
+    ref = OracleEngine(K, P, lr, mu, wd, mode="ref", batch_sizes=M)
+    mir = OracleEngine(K, P, lr, mu, wd, mode="mirror", batch_sizes=M)
+    ref.set_params(x0)
+    mir.set_params(x0)
+    keep = []
+    for r in range(rounds):
+        eng.comm_begin(side_stream if side_stream is not None else torch.cuda.current_stream())
+        ref.comm_begin()
+        mir.comm_begin()
+        for s in range(k):
+            g = np.ascontiguousarray(grad_fn(r * k + s), np.float32)
+            gd = torch.from_numpy(g).cuda()
+            keep.append(gd)
+            eng.local_step(gd)
+            ref.local_step(g)
+            mir.local_step(g)
+        eng.comm_end()
+        ref.comm_end()
+        mir.comm_end()
+        if check_round is not None:
+            check_round(r, eng, ref, mir)
+    eng.sync()
+    return eng, ref, mir
+
+
+# ----------------------------------------------------------------------------- inputs: device == host
+def test_device_generator_matches_host_bits(E):
+    n = 200_003
+    for (seed, stream, w, t, p0, sigma) in [(0, I.STREAM_X0, 0, 0, 0, 0.01), (1234, I.STREAM_GRAD, 5, 17, 0, 0.01),
+                                            (1234, I.STREAM_GRAD, 15, 99, 2 ** 33 + 5, 1.0)]:
+        out = torch.empty(n, dtype=torch.float32, device="cuda")
+        I.device_gaussian_into(out, seed, stream, w, t, p0, sigma)
+        assert_bit_equal(cpu(out), I.gaussian(seed, stream, w, t, p0, n, sigma), f"stream {stream}")
+    g = torch.empty((3, 1001), dtype=torch.float32, device="cuda")
+    I.device_gradients_into(g, step=4)
+    assert_bit_equal(cpu(g), I.gradients(3, 1001, 4))
+
+
+# ----------------------------------------------------------------------------- hand-computed rounds
+@pytest.mark.parametrize("snapshot", [0, 1])
+@pytest.mark.parametrize("name", ["algorithm1_k2_p8.txt", "algorithm1_weight_decay_k1.txt",
+                                  "algorithm1_weighted_mean.txt"])
+def test_golden_rounds_through_the_c_boundary(E, name, snapshot):
+    from test_oracle_pins import load_fixture
+    fx = load_fixture(name)
+    K, P, k = fx["K"], fx["P"], fx["k"]
+    eng = E.Engine(K, P, fx["lr"], fx["mu"], fx["wd"])
+    eng.set_option(E.OPT_SNAPSHOT, snapshot)
+    if fx["batch_sizes"] is not None:
+        eng.set_batch_sizes(fx["batch_sizes"])
+    eng.set_params(fx["x0"].astype(np.float32))
+    side = torch.cuda.Stream()
+    for r in range(fx["rounds"]):
+        eng.comm_begin(side)
+        np.testing.assert_array_equal(cpu(eng.get_mean()).astype(float), fx["expect_mean"][r])
+        for s in range(k):
+            g = np.stack([fx["grad"][(r * k + s, w)] for w in range(K)]).astype(np.float32)
+            eng.local_step(torch.from_numpy(g).cuda())
+        eng.comm_end()
+        x = cpu(eng.get_params()).astype(float)
+        for w in range(K):
+            np.testing.assert_array_equal(x[w], fx["expect_x"][(r, w)])
+    v = cpu(eng.get_momentum()).astype(float)
+    for w in range(K):
+        np.testing.assert_array_equal(v[w], fx["expect_v"][w])
+    assert eng.step_count == k * fx["rounds"]
+
+
+# ----------------------------------------------------------------------------- config 1, element by element
+@pytest.mark.parametrize("snapshot", [0, 1])
+def test_config1_full_vector_parity(E, snapshot):
+    """K=4, P=100,000, lr 0.1, mu 0.9, wd 5e-4, k=4, 10 rounds; x0 and gradients from the
+    seeded recipe.  1e-6 after round one, 1e-5 after the run; mirror mode bit for bit."""
+    K, P, k, rounds = 4, 100_000, 4, 10
+    lr, mu, wd = 0.1, 0.9, 5e-4
+    x0 = I.initial_point(P)
+    worst = {}
+
+    def check(r, eng, ref, mir):
+        if r in (0, rounds - 1):
+            rtol = 1e-6 if r == 0 else 1e-5
+            x, v = cpu(eng.get_params()), cpu(eng.get_momentum())
+            worst[r] = (assert_close_scaled(x, ref.x, rtol, f"x after round {r + 1}"),
+                        assert_close_scaled(v, ref.v, rtol, f"v after round {r + 1}"))
+            assert_bit_equal(x, mir.x, f"x vs mirror after round {r + 1}")
+            assert_bit_equal(v, mir.v, f"v vs mirror after round {r + 1}")
+
+    eng, ref, mir = run_both(E, K, P, lr, mu, wd, k, rounds, x0, lambda t: I.gradients(K, P, t),
+                             snapshot=snapshot, check_round=check)
+    assert_bit_equal(cpu(eng.get_mean()), mir.mean, "last average model")
+    print("config1 worst scaled errors (x, v) by round:", worst)
+
+
+# ----------------------------------------------------------------------------- shapes: tiles, ragged tails, misaligned rows
+@pytest.mark.parametrize("K,P", [(1, 1), (1, 4099), (2, 8), (3, 7), (5, 1001), (2, 3), (16, 4096 + 4),
+                                 (64, 1028), (7, 262_144 + 12), (33, 515), (128, 260)])
+@pytest.mark.parametrize("snapshot", [0, 1])
+def test_shapes_spanning_tiles_and_ragged_tails(E, K, P, snapshot):
+    rng = np.random.default_rng(K * 1000 + P)
+    k, rounds = 2, 3
+    lr, mu, wd = 0.1, 0.9, 5e-4
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    G = (rng.standard_normal((k * rounds, K, P)) * 0.01).astype(np.float32)
+    eng, ref, mir = run_both(E, K, P, lr, mu, wd, k, rounds, x0, lambda t: G[t], snapshot=snapshot)
+    x, v = cpu(eng.get_params()), cpu(eng.get_momentum())
+    assert_bit_equal(x, mir.x, "x vs mirror")
+    assert_bit_equal(v, mir.v, "v vs mirror")
+    assert_close_scaled(x, ref.x, 1e-5, "x vs ref")
+    assert_close_scaled(v, ref.v, 1e-5, "v vs ref")
+
+
+@pytest.mark.parametrize("side", ["own", "same", "high"])
+@pytest.mark.parametrize("weighted", [False, True])
+def test_side_stream_choices_and_weighted_mean(E, side, weighted):
+    rng = np.random.default_rng(11)
+    K, P, k, rounds = 6, 50_000, 3, 4
+    M = rng.integers(1, 9, K).astype(float) if weighted else None
+    x0 = I.initial_point(P)
+    eng, ref, mir = run_both(E, K, P, 0.05, 0.9, 5e-4, k, rounds, x0, lambda t: I.gradients(K, P, t),
+                             M=M, side=side)
+    x = cpu(eng.get_params())
+    assert_bit_equal(x, mir.x, "x vs mirror")
+    assert_close_scaled(x, ref.x, 1e-5, "x vs ref")
+    assert_close_scaled(cpu(eng.get_mean()), ref.mean, 1e-6, "mean vs ref")
+    # line 6 preserves the weighted mean over workers
+    w = np.full(K, 1 / K) if M is None else M / M.sum()
+    np.testing.assert_allclose(w @ x.astype(float), w @ ref.x.astype(float), rtol=0, atol=2e-7)
+
+
+def test_misaligned_gradient_pointer_takes_the_scalar_path(E):
+    rng = np.random.default_rng(12)
+    K, P = 3, 10_001
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    g = (rng.standard_normal(K * P + 1) * 0.01).astype(np.float32)
+    gd = torch.from_numpy(g).cuda()
+    view = gd[1:].view(K, P)                      # 4-byte aligned only
+    assert view.data_ptr() % 16 != 0
+    eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
+    eng.set_params(x0)
+    eng.local_step(view)
+    mir = OracleEngine(K, P, 0.1, 0.9, 5e-4, mode="mirror")
+    mir.set_params(x0)
+    mir.local_step(g[1:].reshape(K, P))
+    assert_bit_equal(cpu(eng.get_params()), mir.x)
+    assert_bit_equal(cpu(eng.get_momentum()), mir.v)
+
+
+# ----------------------------------------------------------------------------- degenerate cases of the method
+@pytest.mark.parametrize("snapshot", [0, 1])
+def test_merge_without_local_steps_is_plain_model_averaging(E, snapshot):
+    rng = np.random.default_rng(13)
+    K, P = 5, 3000
+    X = (rng.standard_normal((K, P)) * 0.1).astype(np.float32)
+    eng = E.Engine(K, P, 0.1, 0.9, 0.0)
+    eng.set_option(E.OPT_SNAPSHOT, snapshot)
+    eng.set_params_all(torch.from_numpy(X).cuda())
+    eng.comm_begin(torch.cuda.Stream())
+    eng.comm_end()
+    x, m = cpu(eng.get_params()), cpu(eng.get_mean())
+    for i in range(K):
+        assert_bit_equal(x[i], m, f"row {i}")
+    np.testing.assert_allclose(m, X.astype(float).mean(0), rtol=0, atol=3e-8)
+
+
+def test_single_worker_merge_is_identity_to_rounding(E):
+    rng = np.random.default_rng(14)
+    P = 5000
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    G = (rng.standard_normal((6, 1, P)) * 0.01).astype(np.float32)
+    eng, ref, mir = run_both(E, 1, P, 0.1, 0.9, 5e-4, 3, 2, x0, lambda t: G[t])
+    # equals plain single-worker momentum SGD
+    x, v = x0.astype(float), np.zeros(P)
+    for t in range(6):
+        v = np.float32(0.9) * v + G[t, 0] + np.float32(5e-4) * x
+        x = x - np.float32(0.1) * v
+    assert_close_scaled(cpu(eng.get_params())[0], x, 1e-5)
+    assert_bit_equal(cpu(eng.get_params()), mir.x)
+
+
+def test_pure_local_sgd_without_any_communication(E):
+    rng = np.random.default_rng(15)
+    K, P = 2, 777
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    eng = E.Engine(K, P, 0.1, 0.0, 0.0)             # mu = wd = 0: Algorithm 1's update literally
+    eng.set_params(x0)
+    g = (rng.standard_normal((K, P)) * 0.01).astype(np.float32)
+    eng.local_step(torch.from_numpy(g).cuda())
+    want = np.float32(x0[None, :]) - np.float32(0.1) * g.astype(np.float64)
+    assert_close_scaled(cpu(eng.get_params()), want, 1e-6)
+
+
+# ----------------------------------------------------------------------------- boundary behaviour
+def test_state_machine_and_argument_errors(E):
+    eng = E.Engine(2, 16, 0.1, 0.9, 0.0)
+    with pytest.raises(E.CocodError) as e:
+        eng.comm_end()
+    assert e.value.code == E.ERR_STATE
+    with pytest.raises(E.CocodError):
+        eng.get_mean()                              # no average model exists yet
+    s = torch.cuda.Stream()
+    eng.comm_begin(s)
+    with pytest.raises(E.CocodError) as e:
+        eng.comm_begin(s)
+    assert e.value.code == E.ERR_STATE
+    with pytest.raises(E.CocodError) as e:
+        eng.set_params(np.zeros(16, np.float32))
+    assert e.value.code == E.ERR_STATE
+    with pytest.raises(E.CocodError):
+        eng.set_option(E.OPT_SNAPSHOT, 0)
+    assert eng.comm_wait(2000) == E.OK
+    eng.comm_end()
+    with pytest.raises(E.CocodError) as e:
+        eng.comm_wait(1)
+    assert e.value.code == E.ERR_STATE
+    with pytest.raises(E.CocodError) as e:
+        eng.set_batch_sizes([1.0, -1.0])
+    assert e.value.code == E.ERR_INVALID
+    with pytest.raises(E.CocodError):
+        eng.set_option(99, 0)
+    with pytest.raises(ValueError):
+        eng.local_step(torch.zeros(2, 15, device="cuda"))
+    with pytest.raises(ValueError):
+        eng.local_step(torch.zeros(2, 16))          # host tensor on the device entry point
+    eng.sync()
+    eng.destroy()
+    eng.destroy()                                   # idempotent
+
+
+def test_host_gradient_entry_point_matches_device_entry_point(E):
+    K, P = 4, 300_000
+    x0 = I.initial_point(P)
+    a, b = E.Engine(K, P, 0.1, 0.9, 5e-4), E.Engine(K, P, 0.1, 0.9, 5e-4)
+    side = torch.cuda.Stream()
+    for eng in (a, b):
+        eng.set_params(x0)
+    for r in range(2):
+        a.comm_begin(side)
+        b.comm_begin(side)
+        for s in range(2):
+            g = I.gradients(K, P, r * 2 + s)
+            a.local_step(torch.from_numpy(g).cuda())
+            b.local_step_host(torch.from_numpy(g).pin_memory())
+            b.sync()
+        a.comm_end()
+        b.comm_end()
+    assert_bit_equal(cpu(a.get_params()), cpu(b.get_params()))
+    assert_bit_equal(cpu(a.get_momentum()), cpu(b.get_momentum()))
+    host_out = np.empty((K, P), np.float32)
+    b.get_params(host_out)
+    assert_bit_equal(host_out, cpu(a.get_params()))
+
+
+def test_save_restore_resumes_bit_exactly(E):
+    K, P, k = 3, 20_000, 2
+    x0 = I.initial_point(P)
+    side = torch.cuda.Stream()
+
+    def rounds(eng, r0, r1):
+        for r in range(r0, r1):
+            eng.comm_begin(side)
+            for s in range(k):
+                eng.local_step(torch.from_numpy(I.gradients(K, P, r * k + s)).cuda())
+            eng.comm_end()
+
+    a = E.Engine(K, P, 0.1, 0.9, 5e-4)
+    a.set_params(x0)
+    rounds(a, 0, 6)
+    b = E.Engine(K, P, 0.1, 0.9, 5e-4)
+    b.set_params(x0)
+    rounds(b, 0, 3)
+    x, v = b.get_params().clone(), b.get_momentum().clone()
+    c = E.Engine(K, P, 0.1, 0.9, 5e-4)
+    c.set_params_all(x)
+    c.set_momentum(v)
+    rounds(c, 3, 6)
+    assert_bit_equal(cpu(c.get_params()), cpu(a.get_params()))
+    assert_bit_equal(cpu(c.get_momentum()), cpu(a.get_momentum()))
+
+
+def test_learning_rate_schedule_and_profile_records(E):
+    K, P = 2, 4096
+    eng = E.Engine(K, P, 0.1, 0.9, 0.0)
+    mir = OracleEngine(K, P, 0.1, 0.9, 0.0, mode="mirror")
+    x0 = I.initial_point(P)
+    eng.set_params(x0)
+    mir.set_params(x0)
+    eng.set_option(E.OPT_PROFILE, 1)
+    side = torch.cuda.Stream()
+    for r, lr in enumerate([0.1, 0.01]):
+        eng.set_lr(lr)
+        mir.set_lr(lr)
+        eng.comm_begin(side)
+        mir.comm_begin()
+        g = I.gradients(K, P, r)
+        eng.local_step(torch.from_numpy(g).cuda())
+        mir.local_step(g)
+        eng.comm_end()
+        mir.comm_end()
+    assert_bit_equal(cpu(eng.get_params()), mir.x)
+    recs = eng.profile_records()
+    kinds = [E.KERNEL_NAMES[k] for k, _, _ in recs]
+    assert kinds.count("local_step") == 2 and kinds.count("mean") == 2 and kinds.count("merge") == 2
+    assert all(b >= a for _, a, b in recs)
+    assert eng.launch_count >= 7
+
+
+# ----------------------------------------------------------------------------- the four kernels on caller buffers
+def test_stateless_kernels_against_oracle_pieces(E):
+    rng = np.random.default_rng(16)
+    K, P = 9, 12_345 * 4
+    X = (rng.standard_normal((K, P)) * 0.1).astype(np.float32)
+    S = (rng.standard_normal((K, P)) * 0.1).astype(np.float32)
+    V = (rng.standard_normal((K, P)) * 0.02).astype(np.float32)
+    G = (rng.standard_normal((K, P)) * 0.01).astype(np.float32)
+    mir = OracleEngine(K, P, 0.1, 0.9, 5e-4, mode="mirror")
+    mir.x[:], mir.v[:] = X, V
+    mir.local_step(G)
+    x, v, g = (torch.from_numpy(a).cuda() for a in (X, V, G))
+    x_out = torch.empty_like(x)
+    E.kernel_local_step(x, x_out, v, g, 0.1, 0.9, 5e-4)
+    assert_bit_equal(cpu(x_out), mir.x)
+    assert_bit_equal(cpu(v), mir.v)
+    assert_bit_equal(cpu(x), X, "out-of-place step must not touch x_in")
+    snap = torch.empty_like(x)
+    E.kernel_snapshot(x, snap)
+    assert_bit_equal(cpu(snap), X)
+    # mean / merge
+    mir2 = OracleEngine(K, P, 0.1, 0.9, 0.0, mode="mirror")
+    mir2.x[:] = S
+    mir2.comm_begin()
+    mir2.x[:] = X
+    mir2.comm_end()
+    sd, mean = torch.from_numpy(S).cuda(), torch.empty(P, dtype=torch.float32, device="cuda")
+    E.kernel_mean(sd, mean)
+    assert_bit_equal(cpu(mean), mir2.mean)
+    xd = torch.from_numpy(X).cuda()
+    E.kernel_merge(xd, sd, mean)
+    assert_bit_equal(cpu(xd), mir2.x)
+
+
+def test_buffers_next_to_engine_inputs_are_untouched(E):
+    """Guard bands around a caller-owned gradient buffer stay intact (no out-of-range access)."""
+    K, P = 3, 4097
+    pad = 1024
+    big = torch.full((K * P + 2 * pad,), float("nan"), device="cuda")
+    g = big[pad:pad + K * P].view(K, P)
+    g.copy_(torch.from_numpy(I.gradients(K, P, 0)).cuda())
+    eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
+    eng.set_params(I.initial_point(P))
+    eng.comm_begin(torch.cuda.Stream())
+    eng.local_step(g)
+    eng.comm_end()
+    eng.sync()
+    assert torch.isnan(big[:pad]).all() and torch.isnan(big[pad + K * P:]).all()
+    assert torch.isfinite(eng.get_params()).all()
