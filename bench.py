@@ -32,10 +32,13 @@ UNIT = "updates/s"
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20, help="timed rounds")
+    ap.add_argument("--steps", type=int, default=1000, help="timed rounds")
     ap.add_argument("--warmup", type=int, default=3, help="untimed rounds (>= 3)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18", choices=["tiny", "resnet18", "vgg16"])
+    ap.add_argument("--K", type=int, default=None, help="override the workload's worker count (profiling, sweeps)")
+    ap.add_argument("--P", type=int, default=None, help="override the workload's model size")
+    ap.add_argument("--k", type=int, default=None, help="override the workload's local steps per round")
     ap.add_argument("--snapshot", default="flip", choices=["flip", "copy"])
     ap.add_argument("--ring", type=int, default=4, help="distinct gradient buffers cycled through")
     ap.add_argument("--no-e2e", action="store_true")
@@ -264,7 +267,7 @@ def run_ours(args, wl):
     eng.set_option(E.OPT_PROFILE, 1)
     eng.profile_reset()
     torch.cuda.synchronize()
-    n_ser = min(args.steps, 10)
+    n_ser = min(args.steps, 50)
     ev0.record(compute)
     for _ in range(n_ser):
         one_round(compute)
@@ -275,14 +278,8 @@ def run_ours(args, wl):
     eng.set_option(E.OPT_PROFILE, 0)
 
     dom = "local_step"
-    traffic = None
-    try:
-        tj = json.load(open(os.path.join(ROOT, "profiles", "ncu_traffic.json")))
-        ent = tj.get(dom, {})
-        if ent.get("dram_bytes_per_element") is not None:
-            traffic = ent["dram_bytes_per_element"] * K * P
-    except (OSError, ValueError):
-        pass
+    traffic = W.NCU_DRAM_BYTES_PER_WORKER_PARAM.get(dom)
+    traffic = traffic * K * P if traffic is not None else None
     dom_tab = in_loop.get(dom, {})
     roofline = {"bound": "hbm", "kernel": dom, "achieved": dom_tab.get("gbs"), "peak": hbm_peak,
                 "unit": "GB/s", "frac": dom_tab.get("frac_of_peak"), "traffic": traffic,
@@ -308,7 +305,7 @@ def run_ours(args, wl):
             eng.comm_end()
             eng.get_mean(mean_out)                      # device -> host read of the round's result
 
-        n_e2e = max(1, min(args.steps, 10))
+        n_e2e = max(1, min(args.steps, 20))
         for _ in range(2):
             one_round_host()
         barrier()
@@ -367,6 +364,9 @@ def main():
     args = parse()
     from paper_1906_12043_b200.workloads import WORKLOADS
     wl = WORKLOADS[args.workload]
+    if args.K or args.P or args.k:
+        from dataclasses import replace
+        wl = replace(wl, name=wl.name + "-custom", K=args.K or wl.K, P=args.P or wl.P, k=args.k or wl.k)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

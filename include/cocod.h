@@ -143,7 +143,7 @@ const char *cocod_strerror(int code);
 
 /* ---------------------------------------------------------------------------------------------
  * Profiling (COCOD_OPT_PROFILE = 1): the engine brackets each of its kernels with CUDA events.
- * cocod_profile_count syncs the device and returns how many records exist (at most 4096 since
+ * cocod_profile_count syncs the device and returns how many records exist (at most 16384 since
  * the last reset); cocod_profile_get returns record i: the kernel kind and its start/end in
  * milliseconds relative to the first record's start.  Used to report per-kernel bandwidth and
  * how much of the mean kernel's lifetime overlaps local steps. */

@@ -23,7 +23,7 @@
 namespace {
 
 constexpr int kMaxWorkers = 1024;
-constexpr int kMaxProfile = 4096;
+constexpr int kMaxProfile = 16384;
 constexpr int64_t kHostChunk = int64_t(1) << 24;   // elements per staged host->device chunk (64 MiB)
 constexpr int kHostSlots = 2;
 
