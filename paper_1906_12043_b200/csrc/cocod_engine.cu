@@ -76,6 +76,7 @@ inline bool fail(cocod_engine *h, cudaError_t e)
 #define CK(h, call) do { if (fail((h), (call))) return COCOD_ERR_CUDA; } while (0)
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
 inline unsigned grid_for(int64_t items, int per_block)
 {
@@ -88,11 +89,11 @@ cudaError_t launch_local_step(const float *x_in, float *x_out, float *v, const f
 {
     using namespace cocod;
     if (n <= 0) return cudaSuccess;
-    constexpr int UNROLL = 4;
+    constexpr int THREADS = 1024, UNROLL = 1;
     int64_t done = 0;
     if (aligned16(x_in) && aligned16(x_out) && aligned16(v) && aligned16(g) && n >= 4) {
         const int64_t nvec = n / 4;
-        local_step_vec4<UNROLL><<<grid_for(nvec, kThreads * UNROLL), kThreads, 0, s>>>(
+        local_step_vec4<THREADS, UNROLL><<<grid_for(nvec, THREADS * UNROLL), THREADS, 0, s>>>(
             reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
             reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd);
         done = nvec * 4;
@@ -149,7 +150,11 @@ cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, 
                          int *n_launch)
 {
     using namespace cocod;
-    if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean)) {
+    if ((P % 8) == 0 && aligned32(x) && aligned32(snap) && aligned32(mean) && K <= 8 * 65535) {
+        constexpr int RC = 8;
+        const dim3 grid(grid_for(P / 8, kThreads), (unsigned)((K + RC - 1) / RC));
+        merge_vec8<RC><<<grid, kThreads, 0, s>>>(x, snap, mean, K, P);
+    } else if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean)) {
         const int64_t pvec = P / 4;
         merge_vec4<4><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
             reinterpret_cast<float4 *>(x), reinterpret_cast<const float4 *>(snap),
