@@ -44,6 +44,10 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-cols", type=int, default=1 << 20)
+    ap.add_argument("--sweep-K", default="2,8,16,32,64")
+    ap.add_argument("--sweep-logP", default="20,24,26,28")
+    ap.add_argument("--sweep", action="store_true",
+                    help="scaling sweep P in {2^20,2^24,2^26,2^28} x K in {2,8,16,32,64} x k in {1,8}: one JSON line per cell")
     return ap.parse_args()
 
 
@@ -360,8 +364,76 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Timing-only sweep over (P, K, k).  Values do not affect timing, so each cell reuses one
+    generated gradient buffer.  Cells whose four K x P buffers exceed 160 GB are skipped."""
+    import torch
+    from paper_1906_12043_b200 import build, engine as E, inputs as I, workloads as W
+    build.build()
+    torch.cuda.set_device(0)
+    side = torch.cuda.Stream(priority=-1)
+    compute = torch.cuda.current_stream()
+    for logP in [int(v) for v in args.sweep_logP.split(",")]:
+        for K in [int(v) for v in args.sweep_K.split(",")]:
+            P = 1 << logP
+            if K * P * 16 > 160e9:
+                continue
+            g = torch.empty((K, P), dtype=torch.float32, device="cuda")
+            I.device_gradients_into(g, 0)
+            x0 = torch.empty(P, dtype=torch.float32, device="cuda")
+            I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, 0, 0.01)
+            for k in (1, 8):
+                eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
+                eng.set_params(x0)
+                wl = W.Workload("sweep", K, P, k, 0, 0.1, 0.9, 5e-4)
+                rounds = max(3, min(200, int(0.25 / (wl.bytes_per_round() / 6.5e12))))
+
+                def one_round(s):
+                    eng.comm_begin(s)
+                    for _ in range(k):
+                        eng.local_step(g)
+                    eng.comm_end()
+
+                res = {}
+                for mode, s in (("overlapped", side), ("serial", compute)):
+                    for _ in range(3):
+                        one_round(s)
+                    eng.set_option(E.OPT_PROFILE, 1)
+                    eng.profile_reset()
+                    torch.cuda.synchronize()
+                    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    ev0.record(compute)
+                    for _ in range(rounds):
+                        one_round(s)
+                    ev1.record(compute)
+                    torch.cuda.synchronize()
+                    by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+                    eng.set_option(E.OPT_PROFILE, 0)
+                    alg = {"local_step": W.BYTES_LOCAL_STEP * K * P, "mean": W.bytes_mean(K) * K * P,
+                           "merge": W.bytes_merge(K) * K * P}
+                    res[mode] = {"ms_per_round": ev0.elapsed_time(ev1) / rounds,
+                                 "gbs": {n: round(alg[n] / (sum(b - a for a, b in iv) / len(iv) * 1e-3) / 1e9, 1)
+                                         for n, iv in by.items()},
+                                 "overlap_fraction": overlap_fraction(by)}
+                ms = res["overlapped"]["ms_per_round"]
+                print(json.dumps({
+                    "sweep": True, "K": K, "P": P, "k": k, "rounds": rounds,
+                    "updates_per_s": K * P * k / (ms * 1e-3),
+                    "hbm_gbs_whole_round": wl.bytes_per_round() / (ms * 1e-3) / 1e9,
+                    "ms_per_round": ms, "ms_per_round_serial": res["serial"]["ms_per_round"],
+                    "kernel_gbs_isolated": res["serial"]["gbs"], "kernel_gbs_overlapped": res["overlapped"]["gbs"],
+                    "overlap_fraction": res["overlapped"]["overlap_fraction"],
+                    "l2_resident": bool(K * P * 16 < 126e6)}), flush=True)
+                eng.destroy()
+            del g, x0
+            torch.cuda.empty_cache()
+
+
 def main():
     args = parse()
+    if args.sweep:
+        run_sweep(args)
+        return
     from paper_1906_12043_b200.workloads import WORKLOADS
     wl = WORKLOADS[args.workload]
     if args.K or args.P or args.k:

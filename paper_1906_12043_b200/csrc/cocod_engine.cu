@@ -135,7 +135,11 @@ cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, flo
 {
     using namespace cocod;
     const float inv_k = 1.0f / (float)K;
-    if ((P % 4) == 0 && aligned16(snap) && aligned16(mean)) {
+    if (K <= 4 && (P % 8) == 0 && aligned32(snap) && aligned32(mean)) {
+        const unsigned grid = grid_for(P / 8, kThreads);
+        if (K <= 2) mean_vec8<2><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
+        else mean_vec8<4><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
+    } else if ((P % 4) == 0 && aligned16(snap) && aligned16(mean)) {
         const int64_t pvec = P / 4;
         mean_vec4<8><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
             reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k);
@@ -151,9 +155,12 @@ cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, 
 {
     using namespace cocod;
     if ((P % 8) == 0 && aligned32(x) && aligned32(snap) && aligned32(mean) && K <= 8 * 65535) {
-        constexpr int RC = 8;
-        const dim3 grid(grid_for(P / 8, kThreads), (unsigned)((K + RC - 1) / RC));
-        merge_vec8<RC><<<grid, kThreads, 0, s>>>(x, snap, mean, K, P);
+        // rows per thread: as many as K allows up to 8 (registers scale with it)
+        const unsigned gx = grid_for(P / 8, kThreads);
+        if (K >= 8) merge_vec8<8><<<dim3(gx, (unsigned)((K + 7) / 8)), kThreads, 0, s>>>(x, snap, mean, K, P);
+        else if (K >= 4) merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x, snap, mean, K, P);
+        else if (K >= 2) merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x, snap, mean, K, P);
+        else merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x, snap, mean, K, P);
     } else if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean)) {
         const int64_t pvec = P / 4;
         merge_vec4<4><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(

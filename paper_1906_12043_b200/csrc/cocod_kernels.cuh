@@ -193,6 +193,44 @@ mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__r
     mean[c] = s;
 }
 
+// Few workers (K <= 4): a float4 per row would leave too few bytes in flight per thread, so
+// one thread owns 8 columns (256-bit loads).  Same row order.  P mod 8 == 0, 32-byte aligned.
+template <int RC>
+__global__ void __launch_bounds__(kThreads)
+mean_vec8(const float *__restrict__ snap, int K, int64_t P, const float *__restrict__ w,
+          float *__restrict__ mean, float inv_k)
+{
+    const int64_t c = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 8;
+    if (c >= P) return;
+    f32x8 s;
+    for (int i0 = 0; i0 < K; i0 += RC) {
+        f32x8 r[RC];
+#pragma unroll
+        for (int j = 0; j < RC; ++j)
+            if (i0 + j < K) r[j] = ld256_stream(snap + (int64_t)(i0 + j) * P + c);
+#pragma unroll
+        for (int j = 0; j < RC; ++j) {
+            const int i = i0 + j;
+            if (i < K) {
+                if (w != nullptr) {
+                    const float wi = __ldg(w + i);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        s.a[q] = (i == 0) ? __fmul_rn(wi, r[j].a[q]) : __fmaf_rn(wi, r[j].a[q], s.a[q]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) s.a[q] = (i == 0) ? r[j].a[q] : __fadd_rn(s.a[q], r[j].a[q]);
+                }
+            }
+        }
+    }
+    if (w == nullptr) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) s.a[q] = __fmul_rn(s.a[q], inv_k);
+    }
+    st256(mean + c, s);
+}
+
 // Any P / alignment: one thread per column, same row order.
 __global__ void __launch_bounds__(kThreads)
 mean_scalar(const float *__restrict__ snap, int K, int64_t P, const float *__restrict__ w,
