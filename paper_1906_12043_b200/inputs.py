@@ -229,3 +229,65 @@ def device_gradients_into(g, step: int, sigma: float = 0.01, seed: int = GRAD_SE
     K = g.shape[0]
     for w in range(K):
         device_gaussian_into(g[w], seed, STREAM_GRAD, w, step, p0, sigma)
+
+
+# ----------------------------------------------------------------------------- synthetic MLP workload
+# End-to-end configuration: every worker trains a 3-layer ReLU MLP (784 -> 1024 -> 1024 -> 10) on
+# minibatches of 128 Gaussian inputs whose labels come from a fixed random "teacher" MLP of the
+# same shape.  Flat parameter order: W1, b1, W2, b2, W3, b3, each W row-major [out][in].
+MLP_DIMS = (784, 1024, 1024, 10)
+MLP_BATCH = 128
+MLP_STUDENT_SEED, MLP_TEACHER_SEED, MLP_DATA_SEED = 0, 1, 2
+
+
+def mlp_segments(dims=MLP_DIMS):
+    """[(name, offset, shape)] of the flat parameter vector, and its length P."""
+    d_in, d_h1, d_h2, d_out = dims
+    segs, off = [], 0
+    for name, shape in (("W1", (d_h1, d_in)), ("b1", (d_h1,)), ("W2", (d_h2, d_h1)), ("b2", (d_h2,)),
+                        ("W3", (d_out, d_h2)), ("b3", (d_out,))):
+        n = int(np.prod(shape))
+        segs.append((name, off, shape))
+        off += n
+    return segs, off
+
+
+def mlp_init_params(seed: int, dims=MLP_DIMS) -> np.ndarray:
+    """Flat fp32 parameters: W ~ N(0, 1/fan_in), b = 0."""
+    segs, P = mlp_segments(dims)
+    out = np.zeros(P, np.float32)
+    for t, (name, off, shape) in enumerate(segs):
+        if name.startswith("W"):
+            n = int(np.prod(shape))
+            out[off:off + n] = gaussian(seed, STREAM_WEIGHT, t, 0, 0, n, 1.0 / np.sqrt(shape[1]))
+    return out
+
+
+def round_to_bf16(a: np.ndarray) -> np.ndarray:
+    """float32 array -> the nearest bfloat16 values (ties to even), returned as float32."""
+    u = np.ascontiguousarray(a, np.float32).view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32)
+
+
+def bf16_bits(a: np.ndarray) -> np.ndarray:
+    """float32 values that are exactly representable in bfloat16 -> their 16-bit patterns."""
+    return (np.ascontiguousarray(a, np.float32).view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+def mlp_batch(worker: int, step: int, batch: int = MLP_BATCH, d_in: int = MLP_DIMS[0],
+              seed: int = MLP_DATA_SEED) -> np.ndarray:
+    """Minibatch of (worker, step): batch x d_in values ~ N(0, 1), rounded once to bfloat16."""
+    x = gaussian(seed, STREAM_DATA, worker, step, 0, batch * d_in, 1.0)
+    return round_to_bf16(x).reshape(batch, d_in)
+
+
+def mlp_teacher_labels(X: np.ndarray, teacher: np.ndarray, dims=MLP_DIMS) -> np.ndarray:
+    """Labels of a minibatch: argmax of the teacher MLP's logits, computed once on the host in
+    fp64 and handed to both sides (never recomputed on the GPU, so near-ties cannot flip)."""
+    segs, _ = mlp_segments(dims)
+    p = {name: teacher[off:off + int(np.prod(shape))].astype(np.float64).reshape(shape)
+         for name, off, shape in segs}
+    h = np.maximum(X.astype(np.float64) @ p["W1"].T + p["b1"], 0.0)
+    h = np.maximum(h @ p["W2"].T + p["b2"], 0.0)
+    return np.argmax(h @ p["W3"].T + p["b3"], axis=1).astype(np.int32)
