@@ -54,7 +54,12 @@ enum {
      * values are identical. */
     COCOD_OPT_SNAPSHOT = 1,
     /* Record CUDA events around every kernel (cocod_profile_*). 0 = off (default). */
-    COCOD_OPT_PROFILE = 2
+    COCOD_OPT_PROFILE = 2,
+    /* Keep a bfloat16 copy of x (K x P, same layout) current: the local-step and merge kernels
+     * write bf16(x) next to x (22 B and 14 B + 4/K per worker-parameter instead of 20 and
+     * 12 + 4/K).  For workloads that compute gradients from bf16 weights with an fp32 master
+     * copy.  1 allocates it, 0 frees it.  Not while a communication is in flight. */
+    COCOD_OPT_BF16_SHADOW = 3
 };
 enum { COCOD_SNAPSHOT_COPY = 0, COCOD_SNAPSHOT_FLIP = 1 };
 
@@ -116,6 +121,11 @@ int cocod_set_momentum(cocod_handle *h, const float *v, int on_host);
 int cocod_get_params(cocod_handle *h, float *out, int on_host);
 int cocod_get_momentum(cocod_handle *h, float *out, int on_host);
 int cocod_get_mean(cocod_handle *h, float *out, int on_host);
+
+/* Device pointer of the bf16 shadow (K x P bfloat16), valid until the option is switched off or
+ * the handle is destroyed.  STATE if the option is off.  Reads must be ordered after the
+ * compute stream's work. */
+int cocod_get_bf16_shadow(cocod_handle *h, void **out);
 
 /* The paper changes gamma during a run (warm-up, decay at epoch 81; Section 5.1). */
 int cocod_set_lr(cocod_handle *h, float lr);

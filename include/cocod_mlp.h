@@ -1,0 +1,80 @@
+/*
+ * cocod_mlp.h -- per-worker mini-batch stochastic gradients for the end-to-end configuration
+ * (part of libcocod.so).
+ *
+ * Algorithm 1 of arxiv 1906.12043, Step II: "compute a mini-batch stochastic gradient
+ * G_tau^i = (1/M_i) sum_j grad f_i(x_tau^i, xi_tau^{i,j})".  Here f is the softmax cross-entropy
+ * of a 3-layer ReLU MLP (d_in -> d_hidden -> d_hidden -> d_out) and all K workers' gradients are
+ * computed in one batched pass: the contractions run on the sm_100a tensor cores (tcgen05.mma,
+ * bf16 operands, fp32 accumulation in TMEM, TMA-staged operands), everything else in small fused
+ * CUDA-core kernels.
+ *
+ * Precision (what the workload fixes: bf16 weights with an fp32 master copy):
+ *   parameters read by forward/backward : the bf16 shadow of the fp32 master copy (all six tensors)
+ *   hidden activations h1, h2           : rounded to bf16 after ReLU
+ *   dz3 = (softmax - onehot) / batch    : rounded to bf16; dz2, dz1 = bf16(dh * (h > 0))
+ *   every sum / product                 : fp32 accumulation; logits, softmax and loss in fp32
+ *   gradients                           : fp32, written in the flat parameter order
+ *
+ * Flat parameter order per worker: W1 [d_hidden][d_in], b1, W2 [d_hidden][d_hidden], b2,
+ * W3 [d_out][d_hidden], b3, then zero padding up to a multiple of 64 elements (the padded count
+ * is what cocod_mlp_param_count returns and what the engine must be created with: padding
+ * parameters and their gradients are always 0, so they never change any result).
+ *
+ * Same conventions as cocod.h: int return codes (COCOD_*), device pointers on the device current
+ * at create, one host thread per handle, asynchronous on the given stream.
+ */
+#ifndef COCOD_MLP_H
+#define COCOD_MLP_H
+
+#include <stdint.h>
+
+#include "cocod.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cocod_mlp cocod_mlp_handle;
+
+/* Allocate the scratch buffers (activations, their transposes, a transposed copy of W2) for K
+ * workers.  Restrictions: batch == 128, d_in % 8 == 0, d_hidden % 128 == 0, 1 <= d_out <= 16.
+ * Errors: INVALID, OOM, CUDA (also when the driver lacks the tensor-map encoder). */
+int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_hidden, int d_out);
+int cocod_mlp_destroy(cocod_mlp_handle *h);
+
+/* Padded parameters per worker (multiple of 64) and the unpadded count. */
+int64_t cocod_mlp_param_count(const cocod_mlp_handle *h);
+int64_t cocod_mlp_param_count_unpadded(const cocod_mlp_handle *h);
+
+/* One mini-batch gradient for every worker.
+ *   params_bf16 : device, K x P bfloat16 (P = padded count): the engine's bf16 shadow
+ *                 (cocod_get_bf16_shadow)
+ *   x           : device, K x batch x d_in bfloat16, the workers' mini-batches
+ *   labels      : device, K x batch int32 in [0, d_out)
+ *   grads       : device, K x P fp32, written completely (padding = 0); feed it to cocod_local_step
+ *   loss        : device, K fp32: mean cross-entropy of each worker's mini-batch
+ * Asynchronous on `stream`.  A kernel-side wait that runs out of time is reported by the next
+ * cocod_mlp_check as COCOD_ERR_TIMEOUT. */
+int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, const int32_t *labels,
+                   float *grads, float *loss, cocod_stream_t stream);
+
+/* Synchronise `stream` and report whether any kernel of this handle gave up a wait. */
+int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream);
+
+/* Number of kernels launched by this handle so far. */
+int64_t cocod_mlp_launch_count(const cocod_mlp_handle *h);
+
+/* The tensor-core building block on its own (tests, measurement):
+ *   C_w[M x N] = A_w[M x K] * B_w[N x K]^T for w in [0, batch_count)
+ * A, B: device bfloat16, reduction index contiguous, row strides lda / ldb elements (multiples of
+ * 8), worker strides in elements (multiples of 8); C: device fp32, row stride ldc.  Bases must be
+ * 16-byte aligned. */
+int cocod_gemm_tn_bf16(const void *A, const void *B, float *C, int M, int N, int K, int batch_count,
+                       int64_t lda, int64_t ldb, int64_t ldc, int64_t stride_a, int64_t stride_b,
+                       int64_t stride_c, cocod_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COCOD_MLP_H */

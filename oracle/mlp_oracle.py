@@ -44,16 +44,21 @@ def split(flat: np.ndarray, dims):
     return out
 
 
-def loss_and_grad(flat: np.ndarray, X: np.ndarray, labels: np.ndarray, dims, emulate_bf16: bool = True):
+def loss_and_grad(flat: np.ndarray, X: np.ndarray, labels: np.ndarray, dims, emulate_bf16: bool = True,
+                  return_preactivations: bool = False):
     """Mean softmax cross-entropy of the minibatch and its gradient w.r.t. the flat parameters
-    (same flat order).  Returns (loss fp64, grad fp32 array)."""
+    (same flat order).  Returns (loss fp64, grad fp32 array), plus the hidden pre-activations
+    (z1, z2) on request: ReLU is a decision "z > 0", and a comparison against another precision is
+    only meaningful for units whose |z| is not within rounding distance of 0."""
     q = bf16 if emulate_bf16 else (lambda a: np.asarray(a, np.float64))
     p = {k: q(v) for k, v in split(flat, dims).items()}
     X = np.asarray(X, np.float64)
     M = X.shape[0]
     # forward
-    h1 = q(np.maximum(X @ p["W1"].T + p["b1"], 0.0))
-    h2 = q(np.maximum(h1 @ p["W2"].T + p["b2"], 0.0))
+    z1 = X @ p["W1"].T + p["b1"]
+    h1 = q(np.maximum(z1, 0.0))
+    z2 = h1 @ p["W2"].T + p["b2"]
+    h2 = q(np.maximum(z2, 0.0))
     z3 = h2 @ p["W3"].T + p["b3"]
     zmax = z3.max(axis=1, keepdims=True)
     e = np.exp(z3 - zmax)
@@ -69,4 +74,6 @@ def loss_and_grad(flat: np.ndarray, X: np.ndarray, labels: np.ndarray, dims, emu
     dz1 = q((dz2 @ p["W2"]) * (h1 > 0))
     g["W1"], g["b1"] = dz1.T @ X, dz1.sum(0)
     flat_g = np.concatenate([g[k].ravel() for k in ("W1", "b1", "W2", "b2", "W3", "b3")])
+    if return_preactivations:
+        return loss, flat_g.astype(np.float32), (z1, z2)
     return loss, flat_g.astype(np.float32)

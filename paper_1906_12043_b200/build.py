@@ -16,7 +16,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
 TARGETS = {
-    "libcocod.so": ["cocod_engine.cu"],
+    "libcocod.so": ["cocod_engine.cu", "cocod_mlp.cu"],
     "libcocod_inputs.so": ["inputs_gen.cu"],
 }
 
@@ -25,7 +25,7 @@ def _stale(out: str, srcs: list[str]) -> bool:
     if not os.path.exists(out):
         return True
     deps = list(srcs) + [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))]
-    deps.append(os.path.join(ROOT, "include", "cocod.h"))
+    deps += [os.path.join(ROOT, "include", f) for f in os.listdir(os.path.join(ROOT, "include"))]
     t = os.path.getmtime(out)
     return any(os.path.getmtime(d) > t for d in deps)
 

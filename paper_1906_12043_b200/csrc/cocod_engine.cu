@@ -45,6 +45,7 @@ struct cocod_engine {
     float *buf[2] = {nullptr, nullptr};
     int cur = 0;
     float *v = nullptr, *mean = nullptr, *w = nullptr;
+    __nv_bfloat16 *shadow = nullptr;    // optional bf16 copy of x, kept current by every kernel that writes x
     bool weighted = false;
     const float *snap = nullptr;       // where this round's stored copies live
     bool pending_flip = false;          // FLIP mode: x still lives in the stored-copy buffer
@@ -85,24 +86,31 @@ inline unsigned grid_for(int64_t items, int per_block)
 
 // ---------------------------------------------------------------- launchers (shared with the stateless entry points)
 cudaError_t launch_local_step(const float *x_in, float *x_out, float *v, const float *g, int64_t n,
-                              float lr, float mu, float wd, cudaStream_t s, int *n_launch)
+                              float lr, float mu, float wd, __nv_bfloat16 *shadow, cudaStream_t s, int *n_launch)
 {
     using namespace cocod;
     if (n <= 0) return cudaSuccess;
     constexpr int THREADS = 1024, UNROLL = 1;
     int64_t done = 0;
-    if (aligned16(x_in) && aligned16(x_out) && aligned16(v) && aligned16(g) && n >= 4) {
+    if (aligned16(x_in) && aligned16(x_out) && aligned16(v) && aligned16(g) && n >= 4 &&
+        (shadow == nullptr || (reinterpret_cast<uintptr_t>(shadow) & 7u) == 0)) {
         const int64_t nvec = n / 4;
-        local_step_vec4<THREADS, UNROLL><<<grid_for(nvec, THREADS * UNROLL), THREADS, 0, s>>>(
-            reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
-            reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd);
+        const unsigned grid = grid_for(nvec, THREADS * UNROLL);
+        if (shadow != nullptr)
+            local_step_vec4<THREADS, UNROLL, true><<<grid, THREADS, 0, s>>>(
+                reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
+                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, shadow);
+        else
+            local_step_vec4<THREADS, UNROLL, false><<<grid, THREADS, 0, s>>>(
+                reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
+                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, nullptr);
         done = nvec * 4;
         if (n_launch) ++*n_launch;
     }
     if (done < n) {
         const int64_t rest = n - done;
         const unsigned grid = (unsigned)std::min<int64_t>((rest + kThreads - 1) / kThreads, 148 * 8);
-        local_step_scalar<<<grid, kThreads, 0, s>>>(x_in, x_out, v, g, done, rest, lr, mu, wd);
+        local_step_scalar<<<grid, kThreads, 0, s>>>(x_in, x_out, v, g, done, rest, lr, mu, wd, shadow);
         if (n_launch) ++*n_launch;
     }
     return cudaGetLastError();
@@ -150,24 +158,26 @@ cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, flo
     return cudaGetLastError();
 }
 
-cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, int64_t P, cudaStream_t s,
-                         int *n_launch)
+cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, int64_t P,
+                         __nv_bfloat16 *shadow, cudaStream_t s, int *n_launch)
 {
     using namespace cocod;
-    if ((P % 8) == 0 && aligned32(x) && aligned32(snap) && aligned32(mean) && K <= 8 * 65535) {
+    if ((P % 8) == 0 && aligned32(x) && aligned32(snap) && aligned32(mean) && K <= 8 * 65535 &&
+        (shadow == nullptr || aligned16(shadow))) {
         // rows per thread: as many as K allows up to 8 (registers scale with it)
         const unsigned gx = grid_for(P / 8, kThreads);
-        if (K >= 8) merge_vec8<8><<<dim3(gx, (unsigned)((K + 7) / 8)), kThreads, 0, s>>>(x, snap, mean, K, P);
-        else if (K >= 4) merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x, snap, mean, K, P);
-        else if (K >= 2) merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x, snap, mean, K, P);
-        else merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x, snap, mean, K, P);
-    } else if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean)) {
+        if (K >= 8) merge_vec8<8><<<dim3(gx, (unsigned)((K + 7) / 8)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
+        else if (K >= 4) merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
+        else if (K >= 2) merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
+        else merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
+    } else if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean) &&
+               (shadow == nullptr || (reinterpret_cast<uintptr_t>(shadow) & 7u) == 0)) {
         const int64_t pvec = P / 4;
         merge_vec4<4><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
             reinterpret_cast<float4 *>(x), reinterpret_cast<const float4 *>(snap),
-            reinterpret_cast<const float4 *>(mean), K, pvec);
+            reinterpret_cast<const float4 *>(mean), K, pvec, shadow);
     } else {
-        merge_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(x, snap, mean, K, P);
+        merge_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
     }
     if (n_launch) ++*n_launch;
     return cudaGetLastError();
@@ -219,6 +229,7 @@ void free_all(cocod_engine *h)
     if (h->v) cudaFree(h->v);
     if (h->mean) cudaFree(h->mean);
     if (h->w) cudaFree(h->w);
+    if (h->shadow) cudaFree(h->shadow);
     for (int i = 0; i < kHostSlots; ++i) {
         if (h->stage[i]) cudaFree(h->stage[i]);
         if (h->ev_copied[i]) cudaEventDestroy(h->ev_copied[i]);
@@ -254,6 +265,17 @@ int copy_out(cocod_engine *h, float *dst, const float *src, size_t bytes, int on
     return COCOD_OK;
 }
 
+// Recompute the bf16 shadow from x (after x was set from outside).
+int refresh_shadow(cocod_engine *h)
+{
+    if (!h->shadow) return COCOD_OK;
+    const unsigned grid = (unsigned)std::min<int64_t>((h->n + cocod::kThreads - 1) / cocod::kThreads, 148 * 16);
+    cocod::shadow_refresh<<<grid, cocod::kThreads, 0, h->compute>>>(h->buf[h->cur], h->shadow, h->n);
+    CK(h, cudaGetLastError());
+    ++h->launches;
+    return COCOD_OK;
+}
+
 // One local step over elements [off, off + len) with gradients at g (already offset).
 int step_range(cocod_engine *h, const float *g, int64_t off, int64_t len)
 {
@@ -262,7 +284,8 @@ int step_range(cocod_engine *h, const float *g, int64_t off, int64_t len)
     int nl = 0;
     {
         Bracket br(h, h->compute, COCOD_KERNEL_LOCAL_STEP);
-        CK(h, launch_local_step(x_in, x_out, h->v + off, g, len, h->lr, h->mu, h->wd, h->compute, &nl));
+        CK(h, launch_local_step(x_in, x_out, h->v + off, g, len, h->lr, h->mu, h->wd,
+                                h->shadow ? h->shadow + off : nullptr, h->compute, &nl));
     }
     h->launches += nl;
     return COCOD_OK;
@@ -409,7 +432,7 @@ int cocod_comm_end(cocod_handle *h)
     {
         Bracket br(h, h->compute, COCOD_KERNEL_MERGE);
         // with no local step since comm_begin (FLIP) x still aliases the stored copies
-        CK(h, launch_merge(h->buf[h->cur], h->snap, h->mean, h->K, h->P, h->compute, &nl));
+        CK(h, launch_merge(h->buf[h->cur], h->snap, h->mean, h->K, h->P, h->shadow, h->compute, &nl));
     }
     h->launches += nl;
     h->pending_flip = false;
@@ -446,7 +469,7 @@ int cocod_set_params(cocod_handle *h, const float *x0, int on_host)
         src, h->buf[h->cur], h->K, h->P);
     CK(h, cudaGetLastError());
     ++h->launches;
-    return COCOD_OK;
+    return refresh_shadow(h);
 }
 
 int cocod_set_params_all(cocod_handle *h, const float *x, int on_host)
@@ -454,7 +477,8 @@ int cocod_set_params_all(cocod_handle *h, const float *x, int on_host)
     if (int rc = check_live(h)) return rc;
     if (!x) return COCOD_ERR_INVALID;
     if (h->state != IDLE) return COCOD_ERR_STATE;
-    return copy_in(h, h->buf[h->cur], x, (size_t)h->n * sizeof(float), on_host);
+    if (int rc = copy_in(h, h->buf[h->cur], x, (size_t)h->n * sizeof(float), on_host)) return rc;
+    return refresh_shadow(h);
 }
 
 int cocod_set_momentum(cocod_handle *h, const float *v, int on_host)
@@ -526,6 +550,19 @@ int cocod_set_option(cocod_handle *h, int option, int value)
     case COCOD_OPT_PROFILE:
         h->profile = value != 0;
         return COCOD_OK;
+    case COCOD_OPT_BF16_SHADOW:
+        if (h->state != IDLE) return COCOD_ERR_STATE;
+        if (value && !h->shadow) {
+            cudaError_t e = cudaMalloc((void **)&h->shadow, (size_t)h->n * sizeof(__nv_bfloat16));
+            if (e != cudaSuccess) { cudaGetLastError(); h->shadow = nullptr; return COCOD_ERR_OOM; }
+            return refresh_shadow(h);
+        }
+        if (!value && h->shadow) {
+            CK(h, cudaStreamSynchronize(h->compute));
+            cudaFree(h->shadow);
+            h->shadow = nullptr;
+        }
+        return COCOD_OK;
     default:
         return COCOD_ERR_INVALID;
     }
@@ -555,6 +592,15 @@ int cocod_comm_wait(cocod_handle *h, int timeout_ms)
         if (ms >= timeout_ms) return COCOD_ERR_TIMEOUT;
         std::this_thread::sleep_for(std::chrono::microseconds(50));
     }
+}
+
+int cocod_get_bf16_shadow(cocod_handle *h, void **out)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!out) return COCOD_ERR_INVALID;
+    if (!h->shadow) return COCOD_ERR_STATE;
+    *out = h->shadow;
+    return COCOD_OK;
 }
 
 int64_t cocod_step_count(const cocod_handle *h) { return h ? h->steps : -1; }
@@ -607,7 +653,7 @@ int cocod_kernel_local_step(const float *x_in, float *x_out, float *v, const flo
                             float lr, float mu, float wd, cocod_stream_t stream)
 {
     if (!x_in || !x_out || !v || !g || n < 0) return COCOD_ERR_INVALID;
-    return launch_local_step(x_in, x_out, v, g, n, lr, mu, wd, (cudaStream_t)stream, nullptr) == cudaSuccess
+    return launch_local_step(x_in, x_out, v, g, n, lr, mu, wd, nullptr, (cudaStream_t)stream, nullptr) == cudaSuccess
                ? COCOD_OK : COCOD_ERR_CUDA;
 }
 
@@ -626,7 +672,8 @@ int cocod_kernel_mean(const float *snap, int K, int64_t P, const float *w, float
 int cocod_kernel_merge(float *x, const float *snap, const float *mean, int K, int64_t P, cocod_stream_t stream)
 {
     if (!x || !snap || !mean || K < 1 || P < 1) return COCOD_ERR_INVALID;
-    return launch_merge(x, snap, mean, K, P, (cudaStream_t)stream, nullptr) == cudaSuccess ? COCOD_OK : COCOD_ERR_CUDA;
+    return launch_merge(x, snap, mean, K, P, nullptr, (cudaStream_t)stream, nullptr) == cudaSuccess ? COCOD_OK
+                                                                                                     : COCOD_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -1,0 +1,307 @@
+// Batched bf16 GEMM for sm_100a on the 5th-generation tensor cores:
+//
+//     D_w[M x N] = A_w[M x K] * B_w[N x K]^T        for every worker w (blockIdx.z)
+//
+// A and B are both "K-major" (the reduction index is the contiguous one).  One CTA computes one
+// 128 x 128 tile of one worker:
+//   * operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
+//     4-stage shared-memory ring guarded by mbarriers;
+//   * one elected thread issues tcgen05.mma (kind::f16, bf16 inputs, fp32 accumulation) on
+//     shared-memory descriptors; the 128 x 128 fp32 accumulator lives in TMEM (128 columns);
+//   * all four warps read the accumulator back with tcgen05.ld (32 lanes x 32 columns at a time)
+//     and run a fused epilogue (bias + ReLU, ReLU-mask, or plain fp32 store).
+// Out-of-range rows / reduction columns are zero-filled by TMA, so M, N, K need not be
+// multiples of the tile; stores are predicated.
+//
+// Every wait is bounded in time: if a barrier does not flip within about two seconds the kernel
+// records a code in *error_flag, drains its own copies, frees its TMEM and returns.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cocod {
+namespace gemm {
+
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int TMEM_COLS = 128;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+enum Epilogue {
+    EPI_F32 = 0,        // c[m][n] = acc                                   (fp32, row stride ldc)
+    EPI_BIAS_RELU = 1,  // o[m][n] = oT[n][m] = bf16(max(acc + bias[n], 0))
+    EPI_MASK = 2        // o[m][n] = oT[n][m] = bf16(acc * (mask[m][n] > 0))   (o optional)
+};
+
+struct Params {
+    int M, N, K;                       // per-worker problem
+    float *c;                          // EPI_F32
+    long long c_worker_stride;         // elements
+    int ldc;
+    __nv_bfloat16 *o, *oT;             // bf16 outputs [M][N] (row stride N) and [N][M] (row stride M)
+    long long o_worker_stride;
+    const __nv_bfloat16 *bias;         // [N]
+    long long bias_worker_stride;
+    const __nv_bfloat16 *mask;         // [M][N], row stride N
+    long long mask_worker_stride;
+    int *error_flag;
+};
+
+// ------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long now_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait for a barrier phase, giving up after WAIT_LIMIT_NS or when another role has aborted.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort)
+{
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = now_ns();
+    for (unsigned it = 0;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 255u) == 255u) {
+            if (*abort) return false;
+            if (now_ns() - t0 > WAIT_LIMIT_NS) return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes "
+                 "[%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Arrive on an mbarrier once all tcgen05.mma issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes (64 bf16) with the
+// 128-byte swizzle TMA applied: 8-row groups are 1024 bytes apart (stride byte offset); the
+// leading byte offset is not used by swizzled K-major layouts.  Descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                           // leading byte offset (unused) = 16 B
+    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset = 1024 B
+    d |= (uint64_t)1 << 46;                           // descriptor version
+    d |= (uint64_t)2 << 61;                           // layout: 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+// ------------------------------------------------------------------------------------------ kernel
+template <int EPI>
+__global__ void __launch_bounds__(128)
+gemm_tn_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES), accum = smem_u32(bars + 2 * STAGES);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 1);
+    volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, wk = blockIdx.z;
+    const int nkb = (p.K + BK - 1) / BK;
+    const uint32_t smem_base = smem_u32(smem);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accum, 1);
+        abort[0] = 0;
+        abort[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    if (warp == 0) {                  // warp-collective TMEM allocation
+        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    int failed = 0;
+    if (warp == 0 && lane == 0) {
+        // ---- producer: TMA loads of the A and B tiles of every 64-wide reduction block
+        int armed = 0;
+        for (int kb = 0; kb < nkb; ++kb) {
+            const int s = kb % STAGES;
+            if (kb >= STAGES && !mbar_wait(empty0 + 8 * s, ((kb / STAGES) - 1) & 1, abort)) { failed = 1; break; }
+            mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+            const uint32_t dst = smem_base + s * STAGE_BYTES;
+            tma_load_3d(dst, &map_a, full0 + 8 * s, kb * BK, m0, wk);
+            tma_load_3d(dst + A_BYTES, &map_b, full0 + 8 * s, kb * BK, n0, wk);
+            armed = kb + 1;
+        }
+        if (failed) {                 // let copies that were already issued land before leaving
+            *abort = 1;
+            for (int kb = (armed > STAGES ? armed - STAGES : 0); kb < armed; ++kb)
+                mbar_wait(full0 + 8 * (kb % STAGES), (kb / STAGES) & 1, never);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer
+        for (int kb = 0; kb < nkb; ++kb) {
+            const int s = kb % STAGES;
+            if (!mbar_wait(full0 + 8 * s, (kb / STAGES) & 1, abort)) { failed = 2; break; }
+            tc_fence_after();
+            const uint32_t a_addr = smem_base + s * STAGE_BYTES, b_addr = a_addr + A_BYTES;
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+                const uint64_t ad = smem_desc_sw128(a_addr + k * UMMA_K * 2);
+                const uint64_t bd = smem_desc_sw128(b_addr + k * UMMA_K * 2);
+                umma_bf16(tmem_base, ad, bd, kInstrDesc, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(empty0 + 8 * s);      // frees the stage once these MMAs have read it
+        }
+        if (!failed) umma_commit(accum);      // accumulator complete
+        else *abort = 1;
+    }
+    __syncwarp();
+
+    // ---- epilogue: every thread owns one accumulator row (TMEM lane) of the tile
+    bool ok = mbar_wait(accum, 0, abort);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+        tc_fence_after();
+        const int m = m0 + warp * 32 + lane;
+        const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
+        for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(trow + c0, r);
+            tmem_ld_wait();
+            const int nb = n0 + c0;
+            if (nb >= p.N) break;
+            if (EPI == EPI_F32) {
+                if (m < p.M) {
+                    float *dst = p.c + (long long)wk * p.c_worker_stride + (long long)m * p.ldc + nb;
+                    if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4 *>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                               __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < p.N) dst[j] = __uint_as_float(r[j]);
+                    }
+                }
+            } else {
+                __align__(16) __nv_bfloat16 outv[32];
+                const __nv_bfloat16 *bias = (EPI == EPI_BIAS_RELU) ? p.bias + (long long)wk * p.bias_worker_stride : nullptr;
+                const __nv_bfloat16 *mrow = (EPI == EPI_MASK && m < p.M)
+                                                ? p.mask + (long long)wk * p.mask_worker_stride + (long long)m * p.N : nullptr;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float a = __uint_as_float(r[j]);
+                    const int n = nb + j;
+                    if (EPI == EPI_BIAS_RELU) {
+                        a = (n < p.N) ? fmaxf(a + __bfloat162float(bias[n]), 0.0f) : 0.0f;
+                    } else {
+                        const bool on = (mrow != nullptr) && (n < p.N) && (__bfloat162float(mrow[n]) > 0.0f);
+                        a = on ? a : 0.0f;
+                    }
+                    outv[j] = __float2bfloat16_rn(a);
+                }
+                if (m < p.M) {
+                    if (p.o != nullptr) {
+                        __nv_bfloat16 *dst = p.o + (long long)wk * p.o_worker_stride + (long long)m * p.N + nb;
+                        if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+                            const uint4 *src = reinterpret_cast<const uint4 *>(outv);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) reinterpret_cast<uint4 *>(dst)[j] = src[j];
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nb + j < p.N) dst[j] = outv[j];
+                        }
+                    }
+                    if (p.oT != nullptr) {
+                        __nv_bfloat16 *dstT = p.oT + (long long)wk * p.o_worker_stride + (long long)nb * p.M + m;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (nb + j < p.N) dstT[(long long)j * p.M] = outv[j];
+                    }
+                }
+            }
+        }
+    } else if (threadIdx.x == 0 && p.error_flag != nullptr) {
+        atomicExch(p.error_flag, 1);
+    }
+    if (failed && p.error_flag != nullptr) atomicExch(p.error_flag, 1 + failed);
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+}  // namespace gemm
+}  // namespace cocod

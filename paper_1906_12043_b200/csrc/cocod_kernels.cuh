@@ -12,6 +12,7 @@
 //                weighted s = w_0 * snap_0 ; s = fma(w_i, snap_i, s)
 //   merge      : x = mean + (x - snap)
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -53,6 +54,17 @@ __device__ __forceinline__ void st256(float *p, const f32x8 &r)
                     "f"(r.a[6]), "f"(r.a[7]) : "memory");
 }
 
+// bfloat16 shadow of the parameters (round to nearest even), packed stores.
+__device__ __forceinline__ uint32_t pack_bf16x2(float a, float b)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);      // .x = a (low half), .y = b
+    return *reinterpret_cast<const uint32_t *>(&h);
+}
+__device__ __forceinline__ void st_shadow4(__nv_bfloat16 *p, const float4 &x)
+{
+    *reinterpret_cast<uint2 *>(p) = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+}
+
 __device__ __forceinline__ void sgd_update(float4 &x, float4 &v, const float4 &g, float lr, float mu, float wd)
 {
     float d;
@@ -68,10 +80,11 @@ __device__ __forceinline__ void sgd_update(float4 &x, float4 &v, const float4 &g
 // Measured on B200 (K*P = 187 M, back-to-back launches): 1024 threads x 1 float4 (a CTA sweeps
 // 16 KB of each stream in one go) sustains 7.02 TB/s, 256 x 4 sustains 6.84 TB/s; streaming
 // (evict-first) hints on g made no difference, so plain loads are used.
-template <int THREADS, int UNROLL>
+// SHADOW: also write bf16(x) to `shadow` (22 B instead of 20 B per worker-parameter).
+template <int THREADS, int UNROLL, bool SHADOW>
 __global__ void __launch_bounds__(THREADS)
 local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__restrict__ g,
-                int64_t nvec, float lr, float mu, float wd)
+                int64_t nvec, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
 {
     const int64_t base = (int64_t)blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
     float4 xr[UNROLL], vr[UNROLL], gr[UNROLL];
@@ -89,6 +102,7 @@ local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__re
             sgd_update(xr[u], vr[u], gr[u], lr, mu, wd);
             st_plain(v + i, vr[u]);
             st_plain(x_out + i, xr[u]);
+            if (SHADOW) st_shadow4(shadow + 4 * i, xr[u]);
         }
     } else {
 #pragma unroll
@@ -99,6 +113,7 @@ local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__re
                 sgd_update(xx, vv, gg, lr, mu, wd);
                 st_plain(v + i, vv);
                 st_plain(x_out + i, xx);
+                if (SHADOW) st_shadow4(shadow + 4 * i, xx);
             }
         }
     }
@@ -107,7 +122,7 @@ local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__re
 // Scalar path: misaligned pointers and the n mod 4 tail.  Elements [first, first + count).
 __global__ void __launch_bounds__(kThreads)
 local_step_scalar(const float *x_in, float *x_out, float *v, const float *__restrict__ g,
-                  int64_t first, int64_t count, float lr, float mu, float wd)
+                  int64_t first, int64_t count, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += stride) {
@@ -115,7 +130,9 @@ local_step_scalar(const float *x_in, float *x_out, float *v, const float *__rest
         const float d = __fmaf_rn(wd, x_in[e], g[e]);
         const float vn = __fmaf_rn(mu, v[e], d);
         v[e] = vn;
-        x_out[e] = __fmaf_rn(-lr, vn, x_in[e]);
+        const float xn = __fmaf_rn(-lr, vn, x_in[e]);
+        x_out[e] = xn;
+        if (shadow != nullptr) shadow[e] = __float2bfloat16_rn(xn);
     }
 }
 
@@ -256,7 +273,8 @@ mean_scalar(const float *__restrict__ snap, int K, int64_t P, const float *__res
 // merge with no local step in between): every element is read before it is written.
 template <int RC>
 __global__ void __launch_bounds__(kThreads)
-merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K, int64_t pvec)
+merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K, int64_t pvec,
+           __nv_bfloat16 *__restrict__ shadow)
 {
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (c >= pvec) return;
@@ -280,6 +298,7 @@ merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K
                 o.z = __fadd_rn(m.z, __fsub_rn(xr[j].z, sr[j].z));
                 o.w = __fadd_rn(m.w, __fsub_rn(xr[j].w, sr[j].w));
                 st_plain(x + e, o);
+                if (shadow != nullptr) st_shadow4(shadow + 4 * e, o);
             }
     }
 }
@@ -290,7 +309,8 @@ merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K
 // sustains 6.48 TB/s.  x may alias snap.
 template <int RC>
 __global__ void __launch_bounds__(kThreads)
-merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P)
+merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P,
+           __nv_bfloat16 *__restrict__ shadow)
 {
     const int64_t c = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 8;
     if (c >= P) return;
@@ -312,18 +332,25 @@ merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, i
 #pragma unroll
             for (int q = 0; q < 8; ++q) o.a[q] = __fadd_rn(m.a[q], __fsub_rn(xr[j].a[q], sr[j].a[q]));
             st256(x + e, o);
+            if (shadow != nullptr)
+                *reinterpret_cast<uint4 *>(shadow + e) =
+                    make_uint4(pack_bf16x2(o.a[0], o.a[1]), pack_bf16x2(o.a[2], o.a[3]),
+                               pack_bf16x2(o.a[4], o.a[5]), pack_bf16x2(o.a[6], o.a[7]));
         }
 }
 
 __global__ void __launch_bounds__(kThreads)
-merge_scalar(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P)
+merge_scalar(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P,
+             __nv_bfloat16 *__restrict__ shadow)
 {
     const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (p >= P) return;
     const float m = mean[p];
     for (int i = 0; i < K; ++i) {
         const int64_t e = (int64_t)i * P + p;
-        x[e] = __fadd_rn(m, __fsub_rn(x[e], snap[e]));
+        const float o = __fadd_rn(m, __fsub_rn(x[e], snap[e]));
+        x[e] = o;
+        if (shadow != nullptr) shadow[e] = __float2bfloat16_rn(o);
     }
 }
 
@@ -335,6 +362,15 @@ broadcast_rows(const float *__restrict__ x0, float *__restrict__ x, int K, int64
     if (p >= P) return;
     const float a = x0[p];
     for (int i = 0; i < K; ++i) x[(int64_t)i * P + p] = a;
+}
+
+// shadow[e] = bf16(x[e]) for a whole buffer (after the parameters were set from outside).
+__global__ void __launch_bounds__(kThreads)
+shadow_refresh(const float *__restrict__ x, __nv_bfloat16 *__restrict__ shadow, int64_t n)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += stride)
+        shadow[e] = __float2bfloat16_rn(x[e]);
 }
 
 }  // namespace cocod

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcocod.so")
 
 OK, ERR_INVALID, ERR_OOM, ERR_STATE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
-OPT_SNAPSHOT, OPT_PROFILE = 1, 2
+OPT_SNAPSHOT, OPT_PROFILE, OPT_BF16_SHADOW = 1, 2, 3
 SNAPSHOT_COPY, SNAPSHOT_FLIP = 0, 1
 KERNEL_LOCAL_STEP, KERNEL_SNAPSHOT, KERNEL_MEAN, KERNEL_MERGE = 0, 1, 2, 3
 KERNEL_NAMES = {0: "local_step", 1: "snapshot", 2: "mean", 3: "merge"}
@@ -35,6 +35,7 @@ SIGNATURES = {
     "cocod_get_params": (_i, [_vp, _vp, _i]),
     "cocod_get_momentum": (_i, [_vp, _vp, _i]),
     "cocod_get_mean": (_i, [_vp, _vp, _i]),
+    "cocod_get_bf16_shadow": (_i, [_vp, ctypes.POINTER(_vp)]),
     "cocod_set_lr": (_i, [_vp, _f]),
     "cocod_set_batch_sizes": (_i, [_vp, ctypes.POINTER(ctypes.c_double)]),
     "cocod_set_option": (_i, [_vp, _i, _i]),
@@ -92,6 +93,21 @@ def _stream(s):
     if s is None:
         return None
     return s.cuda_stream if hasattr(s, "cuda_stream") else int(s)
+
+
+def _device_view(ptr: int, shape, dtype):
+    """Wrap device memory owned by the library as a torch tensor (no copy, no ownership)."""
+    import torch
+    itemsize = torch.empty((), dtype=dtype).element_size()
+    n = 1
+    for d in shape:
+        n *= int(d)
+
+    class _Mem:
+        __cuda_array_interface__ = {"shape": (n * itemsize,), "typestr": "|u1", "data": (int(ptr), False),
+                                    "version": 2}
+
+    return torch.as_tensor(_Mem(), device="cuda").view(dtype).view(*shape)
 
 
 class Engine:
@@ -198,6 +214,13 @@ class Engine:
         self._ck(self._lib.cocod_get_mean(self._h, _ptr(out), self._check_tensor(out, self.P, "out")),
                  "cocod_get_mean")
         return out
+
+    def bf16_shadow(self):
+        """The engine's bf16 copy of x as a K x P torch.bfloat16 CUDA tensor (a view, no copy)."""
+        import torch
+        ptr = _vp()
+        self._ck(self._lib.cocod_get_bf16_shadow(self._h, ctypes.byref(ptr)), "cocod_get_bf16_shadow")
+        return _device_view(ptr.value, (self.K, self.P), torch.bfloat16)
 
     def set_lr(self, lr: float):
         self._ck(self._lib.cocod_set_lr(self._h, lr), "cocod_set_lr")

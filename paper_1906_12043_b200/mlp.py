@@ -1,0 +1,104 @@
+"""Thin ctypes binding over the MLP-gradient entry points of libcocod.so (include/cocod_mlp.h).
+
+Marshalling only: the gradients are computed by the library's CUDA kernels (tcgen05 GEMMs and
+small fused kernels).  No CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+
+from . import engine as _E
+
+_vp, _i, _i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+
+SIGNATURES = {
+    "cocod_mlp_create": (_i, [ctypes.POINTER(_vp), _i, _i, _i, _i, _i]),
+    "cocod_mlp_destroy": (_i, [_vp]),
+    "cocod_mlp_param_count": (_i64, [_vp]),
+    "cocod_mlp_param_count_unpadded": (_i64, [_vp]),
+    "cocod_mlp_grad": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "cocod_mlp_check": (_i, [_vp, _vp]),
+    "cocod_mlp_launch_count": (_i64, [_vp]),
+    "cocod_gemm_tn_bf16": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i64, _i64, _i64, _i64, _i64, _i64, _vp]),
+}
+
+_declared = False
+
+
+def load():
+    global _declared
+    lib = _E.load()
+    if not _declared:
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _declared = True
+    return lib
+
+
+def _cur_stream(stream):
+    import torch
+    return _E._stream(stream) if stream is not None else torch.cuda.current_stream().cuda_stream
+
+
+class MLPGrad:
+    """Batched mini-batch gradients of the 3-layer ReLU MLP for K workers."""
+
+    def __init__(self, K: int, batch: int = 128, d_in: int = 784, d_hidden: int = 1024, d_out: int = 10):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("the MLP gradient path needs a CUDA device (there is no CPU fallback)")
+        self._lib = load()
+        self._h = _vp()
+        rc = self._lib.cocod_mlp_create(ctypes.byref(self._h), K, batch, d_in, d_hidden, d_out)
+        if rc != _E.OK:
+            self._h = None
+            raise _E.CocodError(rc, "cocod_mlp_create")
+        self.K, self.batch, self.dims = K, batch, (d_in, d_hidden, d_hidden, d_out)
+        self.P = int(self._lib.cocod_mlp_param_count(self._h))
+        self.P_raw = int(self._lib.cocod_mlp_param_count_unpadded(self._h))
+
+    def grad(self, params_bf16, x, labels, grads, loss, stream=None):
+        """params_bf16: K x P bf16; x: K x batch x d_in bf16; labels: K x batch int32;
+        grads: K x P fp32 (out); loss: K fp32 (out).  All CUDA tensors, contiguous."""
+        import torch
+        K, P, B, d_in = self.K, self.P, self.batch, self.dims[0]
+        for t, dt, n, nm in ((params_bf16, torch.bfloat16, K * P, "params_bf16"), (x, torch.bfloat16, K * B * d_in, "x"),
+                             (labels, torch.int32, K * B, "labels"), (grads, torch.float32, K * P, "grads"),
+                             (loss, torch.float32, K, "loss")):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == dt and t.numel() == n):
+                raise ValueError(f"{nm}: need a contiguous CUDA {dt} tensor of {n} elements")
+        rc = self._lib.cocod_mlp_grad(self._h, params_bf16.data_ptr(), x.data_ptr(), labels.data_ptr(),
+                                      grads.data_ptr(), loss.data_ptr(), _cur_stream(stream))
+        if rc != _E.OK:
+            raise _E.CocodError(rc, "cocod_mlp_grad")
+
+    def check(self, stream=None):
+        rc = self._lib.cocod_mlp_check(self._h, _cur_stream(stream))
+        if rc != _E.OK:
+            raise _E.CocodError(rc, "cocod_mlp_check")
+
+    @property
+    def launch_count(self) -> int:
+        return int(self._lib.cocod_mlp_launch_count(self._h))
+
+    def destroy(self):
+        if getattr(self, "_h", None):
+            h, self._h = self._h, None
+            self._lib.cocod_mlp_destroy(h)
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def gemm_tn_bf16(A, B, C, stream=None):
+    """C[w] = A[w] @ B[w].T for CUDA tensors A (W x M x K bf16), B (W x N x K bf16), C (W x M x N fp32)."""
+    W, M, K = A.shape
+    N = B.shape[1]
+    rc = load().cocod_gemm_tn_bf16(A.data_ptr(), B.data_ptr(), C.data_ptr(), M, N, K, W, A.stride(1), B.stride(1),
+                                   C.stride(1), A.stride(0), B.stride(0), C.stride(0), _cur_stream(stream))
+    if rc != _E.OK:
+        raise _E.CocodError(rc, "cocod_gemm_tn_bf16")

@@ -15,9 +15,13 @@ def libs():
 
 
 def declared_functions():
-    src = open(os.path.join(ROOT, "include", "cocod.h")).read()
-    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
-    return sorted(set(re.findall(r"\b(cocod_[a-z_0-9]+)\s*\(", src)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in sorted(os.listdir(inc)):
+        src = open(os.path.join(inc, f)).read()
+        src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+        names |= set(re.findall(r"\b(cocod_[a-z_0-9]+)\s*\(", src))
+    return sorted(names)
 
 
 def test_header_declares_the_five_calls_of_the_algorithm():
@@ -33,9 +37,10 @@ def test_library_exports_every_declared_symbol(libs):
 
 
 def test_binding_covers_every_declared_symbol(libs):
-    from paper_1906_12043_b200 import engine
-    assert sorted(engine.SIGNATURES) == declared_functions()
+    from paper_1906_12043_b200 import engine, mlp
+    assert sorted(list(engine.SIGNATURES) + list(mlp.SIGNATURES)) == declared_functions()
     engine.load()
+    mlp.load()
 
 
 def test_error_paths_that_touch_no_device(libs):
@@ -56,6 +61,16 @@ def test_error_paths_that_touch_no_device(libs):
     assert lib.cocod_create(ctypes.byref(out), 1024, 2 ** 61, 0.1, 0.9, 0.0) == engine.ERR_INVALID
     assert lib.cocod_create(None, 4, 10, 0.1, 0.9, 0.0) == engine.ERR_INVALID
     assert lib.cocod_kernel_mean(None, 4, 10, None, None, None) == engine.ERR_INVALID
+    from paper_1906_12043_b200 import mlp
+    mlp.load()
+    assert lib.cocod_mlp_create(None, 2, 128, 784, 1024, 10) == engine.ERR_INVALID
+    assert lib.cocod_mlp_create(ctypes.byref(out), 2, 64, 784, 1024, 10) == engine.ERR_INVALID
+    assert lib.cocod_mlp_create(ctypes.byref(out), 2, 128, 783, 1024, 10) == engine.ERR_INVALID
+    assert lib.cocod_mlp_create(ctypes.byref(out), 2, 128, 784, 1000, 10) == engine.ERR_INVALID
+    assert lib.cocod_mlp_create(ctypes.byref(out), 2, 128, 784, 1024, 17) == engine.ERR_INVALID
+    assert lib.cocod_mlp_grad(None, None, None, None, None, None, None) == engine.ERR_INVALID
+    assert lib.cocod_mlp_destroy(None) == engine.OK
+    assert lib.cocod_gemm_tn_bf16(None, None, None, 1, 1, 1, 1, 8, 8, 8, 8, 8, 8, None) == engine.ERR_INVALID
 
 
 def test_engine_refuses_to_run_without_a_gpu(libs):
