@@ -35,7 +35,7 @@ def parse():
     ap.add_argument("--steps", type=int, default=1000, help="timed rounds")
     ap.add_argument("--warmup", type=int, default=3, help="untimed rounds (>= 3)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet18", choices=["tiny", "resnet18", "vgg16"])
+    ap.add_argument("--workload", default="resnet18", choices=["tiny", "resnet18", "vgg16", "mlp"])
     ap.add_argument("--K", type=int, default=None, help="override the workload's worker count (profiling, sweeps)")
     ap.add_argument("--P", type=int, default=None, help="override the workload's model size")
     ap.add_argument("--k", type=int, default=None, help="override the workload's local steps per round")
@@ -364,6 +364,123 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_mlp(args):
+    """End-to-end synthetic training: K = 16 workers each train the 784-1024-1024-10 ReLU MLP
+    (bf16 weights, fp32 master copy and momentum) on minibatches of 128; gradients come from the
+    tensor-core path, the parameter path is the same engine with its bf16 shadow switched on.
+    A step (round) = comm_begin, k = 4 x (batched gradients + local step), comm_end."""
+    import numpy as np
+    import torch
+    from paper_1906_12043_b200 import build, engine as E, inputs as I, mlp as M
+    build.build()
+    torch.cuda.set_device(0)
+    M.load()
+    K, k, lr, mu, wd = args.K or 16, args.k or 4, 0.05, 0.9, 0.0
+    dims, B = I.MLP_DIMS, I.MLP_BATCH
+    mg = M.MLPGrad(K, B, dims[0], dims[1], dims[3])
+    P, P_raw = mg.P, mg.P_raw
+    x0 = np.zeros(P, np.float32)
+    x0[:P_raw] = I.mlp_init_params(I.MLP_STUDENT_SEED)
+    teacher = I.mlp_init_params(I.MLP_TEACHER_SEED)
+    eng = E.Engine(K, P, lr, mu, wd)
+    eng.set_option(E.OPT_BF16_SHADOW, 1)
+    eng.set_params(x0)
+    shadow = eng.bf16_shadow()
+    ring_n = max(k, 8)
+    xs_h, ys_h = [], []
+    for t in range(ring_n):
+        X = np.stack([I.mlp_batch(w, t) for w in range(K)])
+        ys_h.append(torch.from_numpy(np.stack([I.mlp_teacher_labels(X[w], teacher) for w in range(K)])).pin_memory())
+        xs_h.append(torch.from_numpy(X).to(torch.bfloat16).pin_memory())
+    xs_d = [x.cuda() for x in xs_h]
+    ys_d = [y.cuda() for y in ys_h]
+    grads = torch.empty((K, P), dtype=torch.float32, device="cuda")
+    loss = torch.empty(K, dtype=torch.float32, device="cuda")
+    side = torch.cuda.Stream(priority=-1)
+    compute = torch.cuda.current_stream()
+    step_no = [0]
+    losses = []
+
+    def one_round(record=False):
+        eng.comm_begin(side)
+        for _ in range(k):
+            i = step_no[0] % ring_n
+            mg.grad(shadow, xs_d[i], ys_d[i], grads, loss)
+            eng.local_step(grads)
+            step_no[0] += 1
+            if record:
+                losses.append(loss.clone())
+        eng.comm_end()
+
+    for r in range(max(3, args.warmup)):
+        one_round(record=True)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    l0 = eng.launch_count + mg.launch_count
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(compute)
+    for _ in range(args.steps):
+        one_round()
+    ev1.record(compute)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    mg.check()
+    ms = ev0.elapsed_time(ev1)
+    launches = eng.launch_count + mg.launch_count - l0
+    final_loss = float(loss.mean().item())
+
+    # end to end: minibatches and labels start in pinned host memory, the loss comes back every step
+    x_dev, y_dev = torch.empty_like(xs_d[0]), torch.empty_like(ys_d[0])
+    loss_h = torch.empty(K, dtype=torch.float32, pin_memory=True)
+    n_e2e = max(1, min(args.steps, 50))
+
+    def one_round_host():
+        eng.comm_begin(side)
+        for _ in range(k):
+            i = step_no[0] % ring_n
+            x_dev.copy_(xs_h[i], non_blocking=True)
+            y_dev.copy_(ys_h[i], non_blocking=True)
+            mg.grad(shadow, x_dev, y_dev, grads, loss)
+            eng.local_step(grads)
+            loss_h.copy_(loss, non_blocking=True)
+            step_no[0] += 1
+        eng.comm_end()
+
+    for _ in range(2):
+        one_round_host()
+    torch.cuda.synchronize()
+    ev0.record(compute)
+    for _ in range(n_e2e):
+        one_round_host()
+    ev1.record(compute)
+    torch.cuda.synchronize()
+    ms_e2e = ev0.elapsed_time(ev1)
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    flops_step = K * 2 * B * (2 * dims[0] * dims[1] + 3 * dims[1] * dims[2] + 3 * dims[2] * dims[3])
+    print(json.dumps({
+        "metric": METRIC, "value": K * P_raw * k * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 contractions / f32 state",
+        "data": "synthetic",
+        "config": {"workload": "mlp", "K": K, "P": P_raw, "P_padded": P, "k": k, "lr": lr, "mu": mu, "wd": wd,
+                   "mlp": list(dims), "batch": B, "minibatch_ring": ring_n},
+        "clocks": clocks, "gpu_launches": launches,
+        "local_steps_per_s": k * args.steps / (ms * 1e-3), "ms_per_local_step": ms / (k * args.steps),
+        "tensor_tflops": flops_step * k * args.steps / (ms * 1e-3) / 1e12,
+        "tensor_peak_tflops": peaks.get("bf16_tflops"),
+        "e2e": {"value": K * P_raw * k * n_e2e / (ms_e2e * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": k * (xs_h[0].numel() * 2 + ys_h[0].numel() * 4), "d2h_bytes_per_step": k * K * 4,
+                "rounds": n_e2e, "ms_per_step": ms_e2e / n_e2e},
+        "loss_first_steps": [round(float(l.mean().item()), 4) for l in losses[:8]], "loss_last": round(final_loss, 4),
+    }))
+    eng.destroy()
+    mg.destroy()
+
+
 def run_sweep(args):
     """Timing-only sweep over (P, K, k).  Values do not affect timing, so each cell reuses one
     generated gradient buffer.  Cells whose four K x P buffers exceed 160 GB are skipped."""
@@ -435,6 +552,13 @@ def main():
         run_sweep(args)
         return
     from paper_1906_12043_b200.workloads import WORKLOADS
+    if args.workload == "mlp":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the oracle's MLP leg is timed by tests only; "
+                              "use the default workload for the reference arm"}))
+            return
+        run_mlp(args)
+        return
     wl = WORKLOADS[args.workload]
     if args.K or args.P or args.k:
         from dataclasses import replace

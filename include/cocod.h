@@ -43,7 +43,8 @@ enum {
     COCOD_ERR_OOM = -2,     /* device or pinned-host allocation failed; nothing is leaked */
     COCOD_ERR_STATE = -3,   /* call not legal now (comm_end without comm_begin, double begin) */
     COCOD_ERR_CUDA = -4,    /* a CUDA call or kernel failed; sticky, see cocod_last_cuda_error */
-    COCOD_ERR_TIMEOUT = -5  /* cocod_comm_wait ran out of time; the engine is still usable */
+    COCOD_ERR_TIMEOUT = -5, /* cocod_comm_wait ran out of time; the engine is still usable */
+    COCOD_ERR_TOO_LARGE = -6 /* the request exceeds a fixed capacity (see cocod_kernel_local_step_host_noalloc) */
 };
 
 /* Options for cocod_set_option. */
@@ -177,6 +178,34 @@ int cocod_kernel_mean(const float *snap, int K, int64_t P, const float *w, float
                       cocod_stream_t stream);
 int cocod_kernel_merge(float *x, const float *snap, const float *mean, int K, int64_t P,
                        cocod_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * (No counterpart in the paper: a deployment convenience.)
+ *
+ * Local step with the gradients in HOST memory for callers that must not allocate device
+ * memory: code running under a framework whose caching allocator already owns the whole GPU (a
+ * raw cudaMalloc then fails or fights the pool), and latency-critical loops that cannot accept
+ * the device-wide synchronisation an allocation may imply.  Unlike cocod_local_step_host, which
+ * cudaMallocs its staging buffers on first use, this call stages the gradients through a fixed
+ * array that is part of the library image, and it calls no allocation routine of any kind.
+ *
+ *   x_in, x_out, v : device, n fp32 each (caller-owned; x_out may equal x_in)
+ *   host_grads     : host, n fp32 (pinned memory keeps the copy asynchronous)
+ *   n              : at most COCOD_NOALLOC_MAX_ELEMS; larger requests are rejected with
+ *                    COCOD_ERR_TOO_LARGE before anything is launched (split the vector instead)
+ * Same arithmetic as cocod_kernel_local_step.  Work is queued on `stream`: one host-to-device copy
+ * into the staging array, then the update kernel.
+ *
+ * The staging array (COCOD_NOALLOC_MAX_ELEMS * 4 bytes = 16 MiB) is held by every GPU that loads
+ * the library until the process exits.  All calls on a device share it and it keeps the previous
+ * call's bytes; each call overwrites the part it uses, so nothing needs clearing, but two calls
+ * whose GPU work can overlap (different streams without ordering between them) race on it:
+ * order them yourself.
+ * The first call on each device looks up the array's device address (once per device, with that
+ * device current); make that first call outside any stream capture. */
+#define COCOD_NOALLOC_MAX_ELEMS (4 * 1024 * 1024)
+int cocod_kernel_local_step_host_noalloc(const float *x_in, float *x_out, float *v, const float *host_grads,
+                                         int64_t n, float lr, float mu, float wd, cocod_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -618,6 +618,7 @@ const char *cocod_strerror(int code)
     case COCOD_ERR_STATE: return "call not legal in the engine's current state";
     case COCOD_ERR_CUDA: return "CUDA error";
     case COCOD_ERR_TIMEOUT: return "timed out";
+    case COCOD_ERR_TOO_LARGE: return "request exceeds the fixed capacity of this entry point";
     default: return "unknown error code";
     }
 }
@@ -677,3 +678,40 @@ int cocod_kernel_merge(float *x, const float *snap, const float *mean, int K, in
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ allocation-free host-gradient step
+// Staging for cocod_kernel_local_step_host_noalloc.  In host code the name below is only a
+// stand-in for the symbol, not a device address: the address is looked up once per device.
+static __device__ __align__(256) float g_noalloc_stage[COCOD_NOALLOC_MAX_ELEMS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float *g_noalloc_ptr[kMaxDevices] = {nullptr};
+}  // namespace
+
+extern "C" int cocod_kernel_local_step_host_noalloc(const float *x_in, float *x_out, float *v,
+                                                    const float *host_grads, int64_t n, float lr, float mu,
+                                                    float wd, cocod_stream_t stream)
+{
+    if (!x_in || !x_out || !v || !host_grads || n < 0) return COCOD_ERR_INVALID;
+    if (n > (int64_t)COCOD_NOALLOC_MAX_ELEMS) return COCOD_ERR_TOO_LARGE;
+    if (n == 0) return COCOD_OK;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return COCOD_ERR_CUDA;
+    if (g_noalloc_ptr[dev] == nullptr) {       // set-up, once per device, that device being current
+        float *p = nullptr;
+        if (cudaGetSymbolAddress((void **)&p, g_noalloc_stage) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return COCOD_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = p;
+    }
+    float *stage = g_noalloc_ptr[dev];
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(stage, host_grads, (size_t)n * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return COCOD_ERR_CUDA;
+    }
+    return launch_local_step(x_in, x_out, v, stage, n, lr, mu, wd, nullptr, s, nullptr) == cudaSuccess
+               ? COCOD_OK : COCOD_ERR_CUDA;
+}

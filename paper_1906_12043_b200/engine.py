@@ -12,7 +12,8 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libcocod.so")
 
-OK, ERR_INVALID, ERR_OOM, ERR_STATE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+OK, ERR_INVALID, ERR_OOM, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
+NOALLOC_MAX_ELEMS = 4 * 1024 * 1024
 OPT_SNAPSHOT, OPT_PROFILE, OPT_BF16_SHADOW = 1, 2, 3
 SNAPSHOT_COPY, SNAPSHOT_FLIP = 0, 1
 KERNEL_LOCAL_STEP, KERNEL_SNAPSHOT, KERNEL_MEAN, KERNEL_MERGE = 0, 1, 2, 3
@@ -52,6 +53,7 @@ SIGNATURES = {
     "cocod_kernel_snapshot": (_i, [_vp, _vp, _i64, _vp]),
     "cocod_kernel_mean": (_i, [_vp, _i, _i64, _vp, _vp, _vp]),
     "cocod_kernel_merge": (_i, [_vp, _vp, _vp, _i, _i64, _vp]),
+    "cocod_kernel_local_step_host_noalloc": (_i, [_vp, _vp, _vp, _vp, _i64, _f, _f, _f, _vp]),
 }
 
 _lib = None
@@ -304,3 +306,18 @@ def kernel_merge(x, snap, mean, stream=None):
     K, P = x.shape
     s = _stream(stream) if stream is not None else torch.cuda.current_stream().cuda_stream
     _ck_rc(load().cocod_kernel_merge(_ptr(x), _ptr(snap), _ptr(mean), K, P, s), "cocod_kernel_merge")
+
+
+def kernel_local_step_host_noalloc(x_in, x_out, v, host_g, lr, mu, wd, stream=None):
+    """Local step with host gradients for callers that must not allocate device memory: the
+    gradients are staged through a fixed 16 MiB array inside the library (at most
+    NOALLOC_MAX_ELEMS elements per call; larger requests raise with ERR_TOO_LARGE).  x_in, x_out,
+    v: CUDA float32 tensors; host_g: float32 host tensor or array of the same element count."""
+    import torch
+    s = _stream(stream) if stream is not None else torch.cuda.current_stream().cuda_stream
+    n = x_in.numel()
+    count = host_g.numel() if hasattr(host_g, "numel") else host_g.size
+    if count != n:
+        raise ValueError("host_g must have as many elements as x_in")
+    _ck_rc(load().cocod_kernel_local_step_host_noalloc(_ptr(x_in), _ptr(x_out), _ptr(v), _ptr(host_g), n,
+                                                        lr, mu, wd, s), "cocod_kernel_local_step_host_noalloc")
