@@ -37,8 +37,7 @@ extern "C" {
 
 typedef struct cocod_mlp cocod_mlp_handle;
 
-/* Allocate the scratch buffers (activations, their transposes, a transposed copy of W2) for K
- * workers.  Restrictions: batch == 128, d_in % 8 == 0, d_hidden % 128 == 0, 1 <= d_out <= 16.
+/* Allocate the scratch buffers (hidden activations and their gradients) for K workers.  Restrictions: batch == 128, d_in % 8 == 0, d_hidden % 128 == 0, 1 <= d_out <= 16.
  * Errors: INVALID, OOM, CUDA (also when the driver lacks the tensor-map encoder). */
 int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_hidden, int d_out);
 int cocod_mlp_destroy(cocod_mlp_handle *h);
@@ -66,13 +65,15 @@ int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream);
 int64_t cocod_mlp_launch_count(const cocod_mlp_handle *h);
 
 /* The tensor-core building block on its own (tests, measurement):
- *   C_w[M x N] = A_w[M x K] * B_w[N x K]^T for w in [0, batch_count)
- * A, B: device bfloat16, reduction index contiguous, row strides lda / ldb elements (multiples of
- * 8), worker strides in elements (multiples of 8); C: device fp32, row stride ldc.  Bases must be
- * 16-byte aligned. */
-int cocod_gemm_tn_bf16(const void *A, const void *B, float *C, int M, int N, int K, int batch_count,
-                       int64_t lda, int64_t ldb, int64_t ldc, int64_t stride_a, int64_t stride_b,
-                       int64_t stride_c, cocod_stream_t stream);
+ *   C_w[m][n] = sum_k A_w(m, k) * B_w(n, k)   for w in [0, batch_count)
+ * A, B: device bfloat16.  With a_rows_contiguous = 0, A is stored [M][K] (reduction index
+ * contiguous, row stride lda); with 1 it is stored [K][M] (row index contiguous, row stride lda).
+ * Likewise B: [N][K] or [K][N] with ldb.  No operand is copied or transposed.  lda, ldb and the
+ * worker strides are in elements and must be multiples of 8; bases 16-byte aligned.
+ * C: device fp32 [M][N], row stride ldc.  Blocks until the result is complete. */
+int cocod_gemm_bf16(const void *A, const void *B, float *C, int M, int N, int K, int batch_count,
+                    int a_rows_contiguous, int b_rows_contiguous, int64_t lda, int64_t ldb, int64_t ldc,
+                    int64_t stride_a, int64_t stride_b, int64_t stride_c, cocod_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -1,15 +1,18 @@
 // Batched bf16 GEMM for sm_100a on the 5th-generation tensor cores:
 //
-//     D_w[M x N] = A_w[M x K] * B_w[N x K]^T        for every worker w (blockIdx.z)
+//     D_w[m][n] = sum_k A_w(m, k) * B_w(n, k)        for every worker w (blockIdx.z)
 //
-// A and B are both "K-major" (the reduction index is the contiguous one).  One CTA computes one
-// 128 x 128 tile of one worker:
+// Each operand may be stored "K-major" (the reduction index k is the contiguous one: A is [M][K],
+// B is [N][K]) or "MN-major" (m resp. n is contiguous: A is [K][M], B is [K][N]); the tensor cores
+// read both forms from shared memory, so no operand is ever transposed in memory.  One CTA
+// computes one 128 x 128 tile of one worker:
 //   * operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
-//     4-stage shared-memory ring guarded by mbarriers;
+//     shared-memory ring of up to 4 stages guarded by mbarriers;
 //   * one elected thread issues tcgen05.mma (kind::f16, bf16 inputs, fp32 accumulation) on
 //     shared-memory descriptors; the 128 x 128 fp32 accumulator lives in TMEM (128 columns);
 //   * all four warps read the accumulator back with tcgen05.ld (32 lanes x 32 columns at a time)
-//     and run a fused epilogue (bias + ReLU, ReLU-mask, or plain fp32 store).
+//     and run a fused epilogue: bias + ReLU or ReLU-mask with packed bf16 stores, or an fp32 store
+//     that goes through swizzled shared memory and TMA bulk stores (full 128-byte lines).
 // Out-of-range rows / reduction columns are zero-filled by TMA, so M, N, K need not be
 // multiples of the tile; stores are predicated.
 //
@@ -27,13 +30,14 @@ namespace gemm {
 constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 128;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+constexpr int MAX_STAGES = STAGES;
+__host__ __device__ constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */; }
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Epilogue {
-    EPI_F32 = 0,        // c[m][n] = acc                                   (fp32, row stride ldc)
-    EPI_BIAS_RELU = 1,  // o[m][n] = oT[n][m] = bf16(max(acc + bias[n], 0))
-    EPI_MASK = 2        // o[m][n] = oT[n][m] = bf16(acc * (mask[m][n] > 0))   (o optional)
+    EPI_F32 = 0,        // c[m][n] = acc                         (fp32, row stride ldc; TMA store if map_c_ok)
+    EPI_BIAS_RELU = 1,  // o[m][n] = bf16(max(acc + bias[n], 0))
+    EPI_MASK = 2        // o[m][n] = bf16(acc * (mask[m][n] > 0))
 };
 
 struct Params {
@@ -41,12 +45,14 @@ struct Params {
     float *c;                          // EPI_F32
     long long c_worker_stride;         // elements
     int ldc;
-    __nv_bfloat16 *o, *oT;             // bf16 outputs [M][N] (row stride N) and [N][M] (row stride M)
+    int map_c_ok;                      // EPI_F32: map_c describes c, use TMA stores
+    __nv_bfloat16 *o;                  // bf16 output [M][N], row stride N
     long long o_worker_stride;
     const __nv_bfloat16 *bias;         // [N]
     long long bias_worker_stride;
     const __nv_bfloat16 *mask;         // [M][N], row stride N
     long long mask_worker_stride;
+    int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
     int *error_flag;
 };
 
@@ -95,6 +101,17 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map
                  "[%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void tma_store_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
@@ -134,32 +151,45 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor of a K-major tile stored as rows of 128 bytes (64 bf16) with the
-// 128-byte swizzle TMA applied: 8-row groups are 1024 bytes apart (stride byte offset); the
-// leading byte offset is not used by swizzled K-major layouts.  Descriptor version 1 (sm_100).
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+// Shared-memory matrix descriptors (version 1 = sm_100, 128-byte swizzle), for tiles laid out by TMA:
+//  * K-major tile: rows (m or n) of 128 bytes = 64 bf16 along k; 8-row groups are 1024 bytes apart
+//    (stride byte offset); the leading byte offset is unused.  One MMA (k = 16) advances 32 bytes.
+//  * MN-major tile: rows are k, each 128 bytes = 64 bf16 along m (or n); 8-row groups (8 values of
+//    k) are 1024 bytes apart (stride byte offset), and the second block of 64 m/n values lives one
+//    whole 64-row block later (leading byte offset = 64 * 128 bytes).  One MMA (k = 16) advances two
+//    8-row groups = 2048 bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major)
 {
     uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);          // start address, 16-byte units
-    d |= (uint64_t)1 << 16;                           // leading byte offset (unused) = 16 B
-    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset = 1024 B
-    d |= (uint64_t)1 << 46;                           // descriptor version
-    d |= (uint64_t)2 << 61;                           // layout: 128-byte swizzle
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);                              // start address, 16-byte units
+    d |= (uint64_t)(mn_major ? (BK * 128) >> 4 : 1) << 16;               // leading byte offset
+    d |= (uint64_t)(1024 >> 4) << 32;                                     // stride byte offset = 1024 B
+    d |= (uint64_t)1 << 46;                                               // descriptor version
+    d |= (uint64_t)2 << 61;                                               // layout: 128-byte swizzle
     return d;
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 128.
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+// Instruction descriptor: D fp32, A and B bf16, M = 128, N = 128, operand majors as given.
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
 
 // ------------------------------------------------------------------------------------------ kernel
-template <int EPI>
+// Tensor maps: a K-major operand is {k (contiguous), rows, workers} with box {64, 128, 1}; an
+// MN-major operand is {m or n (contiguous), k, workers} with box {64, 64, 1} (two boxes per tile).
+// map_c (EPI_F32 only): {n (contiguous), m, workers} fp32 with box {32, 128, 1}, 128-byte swizzle.
+template <int EPI, bool A_MN, bool B_MN>
 __global__ void __launch_bounds__(128)
-gemm_tn_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const Params p)
+gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+          const __grid_constant__ CUtensorMap map_c, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES), accum = smem_u32(bars + 2 * STAGES);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 1);
+    const int stages = p.stages;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + stages * STAGE_BYTES);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_STAGES), accum = smem_u32(bars + 2 * MAX_STAGES);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 1);
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
 
@@ -169,7 +199,7 @@ gemm_tn_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ 
     const uint32_t smem_base = smem_u32(smem);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
         }
@@ -177,7 +207,7 @@ gemm_tn_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ 
         abort[0] = 0;
         abort[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_async_smem();
     }
     __syncwarp();
     if (warp == 0) {                  // warp-collective TMEM allocation
@@ -194,65 +224,91 @@ gemm_tn_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ 
         // ---- producer: TMA loads of the A and B tiles of every 64-wide reduction block
         int armed = 0;
         for (int kb = 0; kb < nkb; ++kb) {
-            const int s = kb % STAGES;
-            if (kb >= STAGES && !mbar_wait(empty0 + 8 * s, ((kb / STAGES) - 1) & 1, abort)) { failed = 1; break; }
-            mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
-            const uint32_t dst = smem_base + s * STAGE_BYTES;
-            tma_load_3d(dst, &map_a, full0 + 8 * s, kb * BK, m0, wk);
-            tma_load_3d(dst + A_BYTES, &map_b, full0 + 8 * s, kb * BK, n0, wk);
+            const int s = kb % stages;
+            if (kb >= stages && !mbar_wait(empty0 + 8 * s, ((kb / stages) - 1) & 1, abort)) { failed = 1; break; }
+            const uint32_t bar = full0 + 8 * s;
+            mbar_expect_tx(bar, STAGE_BYTES);
+            const uint32_t dst_a = smem_base + s * STAGE_BYTES, dst_b = dst_a + A_BYTES;
+            if (A_MN) {
+                tma_load_3d(dst_a, &map_a, bar, m0, kb * BK, wk);
+                tma_load_3d(dst_a + BK * 128, &map_a, bar, m0 + 64, kb * BK, wk);
+            } else {
+                tma_load_3d(dst_a, &map_a, bar, kb * BK, m0, wk);
+            }
+            if (B_MN) {
+                tma_load_3d(dst_b, &map_b, bar, n0, kb * BK, wk);
+                tma_load_3d(dst_b + BK * 128, &map_b, bar, n0 + 64, kb * BK, wk);
+            } else {
+                tma_load_3d(dst_b, &map_b, bar, kb * BK, n0, wk);
+            }
             armed = kb + 1;
         }
         if (failed) {                 // let copies that were already issued land before leaving
-            *abort = 1;
-            for (int kb = (armed > STAGES ? armed - STAGES : 0); kb < armed; ++kb)
-                mbar_wait(full0 + 8 * (kb % STAGES), (kb / STAGES) & 1, never);
+            abort[0] = 1;
+            for (int kb = (armed > stages ? armed - stages : 0); kb < armed; ++kb)
+                mbar_wait(full0 + 8 * (kb % stages), (kb / stages) & 1, never);
         }
     } else if (warp == 1 && lane == 0) {
         // ---- MMA issuer
+        constexpr uint32_t idesc = instr_desc(A_MN, B_MN);
+        constexpr uint32_t a_step = A_MN ? 2048u : (uint32_t)(UMMA_K * 2), b_step = B_MN ? 2048u : (uint32_t)(UMMA_K * 2);
         for (int kb = 0; kb < nkb; ++kb) {
-            const int s = kb % STAGES;
-            if (!mbar_wait(full0 + 8 * s, (kb / STAGES) & 1, abort)) { failed = 2; break; }
+            const int s = kb % stages;
+            if (!mbar_wait(full0 + 8 * s, (kb / stages) & 1, abort)) { failed = 2; break; }
             tc_fence_after();
             const uint32_t a_addr = smem_base + s * STAGE_BYTES, b_addr = a_addr + A_BYTES;
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k) {
-                const uint64_t ad = smem_desc_sw128(a_addr + k * UMMA_K * 2);
-                const uint64_t bd = smem_desc_sw128(b_addr + k * UMMA_K * 2);
-                umma_bf16(tmem_base, ad, bd, kInstrDesc, (kb > 0 || k > 0) ? 1u : 0u);
+                const uint64_t ad = smem_desc(a_addr + k * a_step, A_MN);
+                const uint64_t bd = smem_desc(b_addr + k * b_step, B_MN);
+                umma_bf16(tmem_base, ad, bd, idesc, (kb > 0 || k > 0) ? 1u : 0u);
             }
             umma_commit(empty0 + 8 * s);      // frees the stage once these MMAs have read it
         }
         if (!failed) umma_commit(accum);      // accumulator complete
-        else *abort = 1;
+        else abort[0] = 1;
     }
     __syncwarp();
 
     // ---- epilogue: every thread owns one accumulator row (TMEM lane) of the tile
     bool ok = mbar_wait(accum, 0, abort);
     ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    if (__syncthreads_and(ok ? 1 : 0)) {
         tc_fence_after();
-        const int m = m0 + warp * 32 + lane;
+        const int row = warp * 32 + lane;
+        const int m = m0 + row;
         const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
         for (int c0 = 0; c0 < BN; c0 += 32) {
+            const int nb = n0 + c0;
+            if (nb >= p.N) break;                      // uniform over the CTA
             uint32_t r[32];
             tmem_ld32(trow + c0, r);
             tmem_ld_wait();
-            const int nb = n0 + c0;
-            if (nb >= p.N) break;
             if (EPI == EPI_F32) {
-                if (m < p.M) {
-                    float *dst = p.c + (long long)wk * p.c_worker_stride + (long long)m * p.ldc + nb;
-                    if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4 *>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                                               __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (nb + j < p.N) dst[j] = __uint_as_float(r[j]);
+                if (p.map_c_ok) {
+                    // stage the 128 x 32 fp32 chunk in shared memory (all MMAs are done, so the ring is
+                    // free) with the 128-byte swizzle: 16-byte piece j of row r sits at piece j ^ (r & 7)
+                    const int buf = (c0 >> 5) & 1;
+                    if (c0 >= 64) {                    // this buffer was handed to a bulk store two chunks ago
+                        if (threadIdx.x == 0) tma_store_wait_read<1>();
+                        __syncthreads();
                     }
+                    uint8_t *tile = smem + buf * (BM * 128);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4 *>(tile + row * 128 + ((j ^ (row & 7)) << 4)) =
+                            make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                    fence_async_smem();
+                    __syncthreads();
+                    if (threadIdx.x == 0) {
+                        tma_store_3d(&map_c, smem_u32(tile), nb, m0, wk);
+                        tma_store_commit();
+                    }
+                } else if (m < p.M) {
+                    float *dst = p.c + (long long)wk * p.c_worker_stride + (long long)m * p.ldc + nb;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (nb + j < p.N) dst[j] = __uint_as_float(r[j]);
                 }
             } else {
                 __align__(16) __nv_bfloat16 outv[32];
@@ -272,27 +328,20 @@ gemm_tn_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ 
                     outv[j] = __float2bfloat16_rn(a);
                 }
                 if (m < p.M) {
-                    if (p.o != nullptr) {
-                        __nv_bfloat16 *dst = p.o + (long long)wk * p.o_worker_stride + (long long)m * p.N + nb;
-                        if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
-                            const uint4 *src = reinterpret_cast<const uint4 *>(outv);
+                    __nv_bfloat16 *dst = p.o + (long long)wk * p.o_worker_stride + (long long)m * p.N + nb;
+                    if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
+                        const uint4 *src = reinterpret_cast<const uint4 *>(outv);
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) reinterpret_cast<uint4 *>(dst)[j] = src[j];
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (nb + j < p.N) dst[j] = outv[j];
-                        }
-                    }
-                    if (p.oT != nullptr) {
-                        __nv_bfloat16 *dstT = p.oT + (long long)wk * p.o_worker_stride + (long long)nb * p.M + m;
+                        for (int j = 0; j < 4; ++j) reinterpret_cast<uint4 *>(dst)[j] = src[j];
+                    } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (nb + j < p.N) dstT[(long long)j * p.M] = outv[j];
+                            if (nb + j < p.N) dst[j] = outv[j];
                     }
                 }
             }
         }
+        if (EPI == EPI_F32 && p.map_c_ok && threadIdx.x == 0) tma_store_wait_read<0>();   // smem must outlive the reads
     } else if (threadIdx.x == 0 && p.error_flag != nullptr) {
         atomicExch(p.error_flag, 1);
     }

@@ -1,22 +1,22 @@
 // Per-worker mini-batch gradients of the 3-layer ReLU MLP (Algorithm 1, Step II: "compute a
 // mini-batch stochastic gradient"), batched over the K workers.  Declared in include/cocod_mlp.h.
 //
-// Data flow of one call (every matrix below exists once per worker; "T" = stored transposed so
-// that each tensor-core contraction sees both operands with the reduction index contiguous):
+// Data flow of one call (every matrix exists once per worker; no matrix is ever transposed in
+// memory: the tensor cores read an operand either with the reduction index contiguous or with the
+// row index contiguous):
 //
-//   xT  = transpose(x)                                    w2T = transpose(W2)
-//   h1, h1T  = bf16(relu(x  W1^T + b1))        GEMM 128 x d_h x d_in    epilogue bias+ReLU
-//   h2       = bf16(relu(h1 W2^T + b2))        GEMM 128 x d_h x d_h     epilogue bias+ReLU
-//   logits = h2 W3^T + b3 ; loss ; dz3 = bf16((softmax - onehot)/batch)        CUDA cores
-//   dW3 = dz3^T h2 ; db3 = colsum dz3                                           CUDA cores
-//   dz2, dz2T = bf16((dz3 W3) * (h2 > 0)) ; db2 = colsum dz2                    CUDA cores
-//   dz1T     = bf16((dz2 W2) * (h1 > 0))       GEMM 128 x d_h x d_h (B = w2T)  epilogue mask
-//   db1 = rowsum dz1T                                                           CUDA cores
-//   dW2 = dz2T h1T^T                           GEMM d_h x d_h x 128            epilogue fp32
-//   dW1 = dz1T xT^T                            GEMM d_h x d_in x 128           epilogue fp32
+//   h1 = bf16(relu(x  W1^T + b1))     GEMM 128 x d_h x d_in   A = x, B = W1            epilogue bias+ReLU
+//   h2 = bf16(relu(h1 W2^T + b2))     GEMM 128 x d_h x d_h    A = h1, B = W2           epilogue bias+ReLU
+//   logits = h2 W3^T + b3 ; loss ; dz3 = bf16((softmax - onehot)/batch)                CUDA cores
+//   dz2 = bf16((dz3 W3) * (h2 > 0)) ; dW3 = dz3^T h2 ; db3, db2 = column sums           CUDA cores
+//   dz1 = bf16((dz2 W2) * (h1 > 0))   GEMM 128 x d_h x d_h    A = dz2, B = W2 read [k][n]  epilogue mask
+//   db1 = column sums of dz1                                                           CUDA cores
+//   dW2 = dz2^T h1                    GEMM d_h x d_h x 128    A = dz2 read [k][m], B = h1 read [k][n]   fp32 out
+//   dW1 = dz1^T x                     GEMM d_h x d_in x 128   A = dz1 read [k][m], B = x  read [k][n]   fp32 out
 #include "cocod_mlp.h"
 #include "cocod_gemm_sm100.cuh"
 
+#include <algorithm>
 #include <cstdio>
 #include <new>
 
@@ -46,135 +46,187 @@ EncodeTiledFn get_encoder()
     return fn;
 }
 
-// 3-D map over a batched K-major bf16 matrix: dims {cols (contiguous), rows, workers}; one box is
-// a 64-column x 128-row tile of one worker, stored with the 128-byte swizzle.
+// 3-D maps over a batched row-major matrix: dims {cols (contiguous), rows, workers}.  `box_rows` is
+// 128 for a K-major operand tile, 64 for an MN-major one; a box is 64 bf16 columns wide (128 bytes,
+// the swizzle span).
 bool make_map(CUtensorMap *m, const void *base, uint64_t cols, uint64_t rows, uint64_t workers, uint64_t ld,
-              uint64_t worker_stride)
+              uint64_t worker_stride, uint32_t box_rows)
 {
     EncodeTiledFn enc = get_encoder();
     if (!enc) return false;
     const cuuint64_t dims[3] = {cols, rows, workers};
     const cuuint64_t strides[2] = {ld * sizeof(bf16), worker_stride * sizeof(bf16)};
-    const cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BM, 1};
+    const cuuint32_t box[3] = {64, box_rows, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+inline bool map_k(CUtensorMap *m, const void *base, uint64_t k, uint64_t rows, uint64_t workers, uint64_t ld, uint64_t ws)
+{
+    return make_map(m, base, k, rows, workers, ld, ws, 128);
+}
+inline bool map_mn(CUtensorMap *m, const void *base, uint64_t mn, uint64_t k, uint64_t workers, uint64_t ld, uint64_t ws)
+{
+    return make_map(m, base, mn, k, workers, ld, ws, 64);
+}
+// fp32 output map for the TMA-store epilogue: box = 32 columns (128 bytes) x 128 rows.
+bool map_out(CUtensorMap *m, float *base, uint64_t cols, uint64_t rows, uint64_t workers, uint64_t ld,
+             uint64_t worker_stride)
+{
+    EncodeTiledFn enc = get_encoder();
+    if (!enc) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) || (ld % 4) || (worker_stride % 4)) return false;
+    const cuuint64_t dims[3] = {cols, rows, workers};
+    const cuuint64_t strides[2] = {ld * sizeof(float), worker_stride * sizeof(float)};
+    const cuuint32_t box[3] = {32, 128, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 
-template <int EPI>
-cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const Params &p, int workers, cudaStream_t s)
+template <int EPI, bool A_MN, bool B_MN>
+cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &c, const Params &p, int workers,
+                        cudaStream_t s)
 {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tn_bf16<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(gemm_bf16<EPI, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             smem_bytes(MAX_STAGES));
         if (e != cudaSuccess) return e;
         configured = true;
     }
     const dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, workers);
-    gemm_tn_bf16<EPI><<<grid, 128, SMEM_BYTES, s>>>(a, b, p);
+    gemm_bf16<EPI, A_MN, B_MN><<<grid, 128, smem_bytes(p.stages), s>>>(a, b, c, p);
     return cudaGetLastError();
 }
 
-// ------------------------------------------------------------------------------------------ small kernels
-// out[w][c][r] = in[w][r][c]; 32 x 32 tiles through shared memory.
-__global__ void __launch_bounds__(256)
-transpose_bf16(const bf16 *__restrict__ in, bf16 *__restrict__ out, int R, int C, long long in_ld,
-               long long in_worker_stride, long long out_worker_stride)
-{
-    __shared__ bf16 tile[32][33];
-    const bf16 *src = in + (long long)blockIdx.z * in_worker_stride;
-    bf16 *dst = out + (long long)blockIdx.z * out_worker_stride;
-    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    for (int i = ty; i < 32; i += 8) {
-        const int r = r0 + i, c = c0 + tx;
-        if (r < R && c < C) tile[i][tx] = src[(long long)r * in_ld + c];
-    }
-    __syncthreads();
-    for (int i = ty; i < 32; i += 8) {
-        const int c = c0 + i, r = r0 + tx;
-        if (r < R && c < C) dst[(long long)c * R + r] = tile[tx][i];
-    }
-}
+inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK - 1) / BK)); }
 
-// One warp per (worker, sample): logits = h2 W3^T + b3 (fp32), row loss, dz3 = bf16((softmax - onehot)/batch)
-// kept as fp32 values in dz3[w][b][16].
+// ------------------------------------------------------------------------------------------ small kernels
+// Output layer forward and loss.  One CTA = 16 samples of one worker; W3 and b3 sit in shared memory;
+// each warp handles two samples: logits = h2 W3^T + b3 (fp32), row loss = -log softmax[label],
+// dz3 = bf16((softmax - onehot) / batch) kept as fp32 values in dz3[w][b][16].  grid (B / 16, K).
 __global__ void __launch_bounds__(256)
 head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long long P, long long oW3, long long ob3,
             const int *__restrict__ labels, float *__restrict__ dz3, float *__restrict__ rowloss, int B, int d_h,
             int d_out)
 {
-    const int gw = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    const int w = gw / B, b = gw % B;
-    const bf16 *hrow = h2 + ((long long)w * B + b) * d_h;
+    extern __shared__ __align__(16) uint8_t head_smem[];
+    bf16 *sW3 = reinterpret_cast<bf16 *>(head_smem);                 // [d_out][d_h]
+    const int w = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bf16 *W3 = params + (long long)w * P + oW3;
-    float acc[16];
+    for (int i = threadIdx.x * 8; i < d_out * d_h; i += 256 * 8)
+        *reinterpret_cast<uint4 *>(sW3 + i) = *reinterpret_cast<const uint4 *>(W3 + i);
+    __syncthreads();
+    const bf16 *b3 = params + (long long)w * P + ob3;
+    for (int sidx = 0; sidx < 2; ++sidx) {
+        const int b = blockIdx.x * 16 + warp * 2 + sidx;
+        const bf16 *hrow = h2 + ((long long)w * B + b) * d_h;
+        float acc[16];
 #pragma unroll
-    for (int c = 0; c < 16; ++c) acc[c] = 0.0f;
-    for (int j = lane; j < d_h; j += 32) {
-        const float h = __bfloat162float(hrow[j]);
+        for (int c = 0; c < 16; ++c) acc[c] = 0.0f;
+        for (int j = lane * 8; j < d_h; j += 256) {
+            const uint4 hv = *reinterpret_cast<const uint4 *>(hrow + j);
+            const bf16 *hp = reinterpret_cast<const bf16 *>(&hv);
+            float hf[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) hf[q] = __bfloat162float(hp[q]);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) {
+                if (c < d_out) {
+                    const uint4 wv = *reinterpret_cast<const uint4 *>(sW3 + c * d_h + j);
+                    const bf16 *wp = reinterpret_cast<const bf16 *>(&wv);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) acc[c] = fmaf(hf[q], __bfloat162float(wp[q]), acc[c]);
+                }
+            }
+        }
 #pragma unroll
         for (int c = 0; c < 16; ++c)
-            if (c < d_out) acc[c] = fmaf(h, __bfloat162float(W3[(long long)c * d_h + j]), acc[c]);
-    }
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
+            for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+        // lane c finishes class c
+        float z = -INFINITY;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
-    if (lane == 0) {
-        const bf16 *b3 = params + (long long)w * P + ob3;
-        float z[16], zmax = -INFINITY;
-        for (int c = 0; c < d_out; ++c) {
-            z[c] = acc[c] + __bfloat162float(b3[c]);
-            zmax = fmaxf(zmax, z[c]);
-        }
-        float s = 0.0f;
-        for (int c = 0; c < d_out; ++c) {
-            z[c] = expf(z[c] - zmax);
-            s += z[c];
-        }
+        for (int c = 0; c < 16; ++c)
+            if (lane == c && c < d_out) z = acc[c] + __bfloat162float(b3[c]);
+        float zmax = z;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+        const float e = (lane < d_out) ? expf(z - zmax) : 0.0f;
+        float ssum = e;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
         const int y = labels[(long long)w * B + b];
-        const float inv = 1.0f / s, invB = 1.0f / (float)B;
-        float lz = 0.0f;
-        for (int c = 0; c < 16; ++c) {
-            float d = 0.0f;
-            if (c < d_out) {
-                const float pc = z[c] * inv;
-                if (c == y) lz = pc;
-                d = __bfloat162float(__float2bfloat16_rn((pc - (c == y ? 1.0f : 0.0f)) * invB));
-            }
-            dz3[((long long)w * B + b) * 16 + c] = d;
+        const float pc = e / ssum;
+        if (lane < 16) {
+            const float d = (lane < d_out) ? (pc - (lane == y ? 1.0f : 0.0f)) / (float)B : 0.0f;
+            dz3[((long long)w * B + b) * 16 + lane] = __bfloat162float(__float2bfloat16_rn(d));
         }
-        rowloss[(long long)w * B + b] = -logf(lz);
+        const float py = __shfl_sync(0xffffffffu, pc, y);
+        if (lane == 0) rowloss[(long long)w * B + b] = -logf(py);
     }
 }
 
-// dW3[c][j] = sum_b dz3[b][c] h2[b][j]; db3[c] = sum_b dz3[b][c]; loss[w] = mean_b rowloss; the
-// gradient's zero padding.  grid (d_h / 256, K).
+// Everything downstream of dz3 that runs on CUDA cores, for 32 hidden units j and all 128 samples:
+//   dz2[b][j] = bf16((sum_c dz3[b][c] W3[c][j]) * (h2[b][j] > 0)),  db2[j] = sum_b dz2[b][j],
+//   dW3[c][j] = sum_b dz3[b][c] h2[b][j];
+// the CTA with blockIdx.x == 0 also writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the
+// zero padding of the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32, K).
 __global__ void __launch_bounds__(256)
-head_dw3(const bf16 *__restrict__ h2, const float *__restrict__ dz3, const float *__restrict__ rowloss,
-         float *__restrict__ grads, float *__restrict__ loss, long long P, long long P_raw, long long oW3,
-         long long ob3, int B, int d_h, int d_out)
+head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, const float *__restrict__ dz3,
+              const float *__restrict__ rowloss, bf16 *__restrict__ dz2, float *__restrict__ grads,
+              float *__restrict__ loss, long long P, long long P_raw, long long oW3, long long ob2, long long ob3,
+              int B, int d_h, int d_out)
 {
     __shared__ float sdz[128 * 16];
-    const int w = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
+    __shared__ float red[8][16][33];
+    __shared__ float colsum[8][33];
+    const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
     for (int i = threadIdx.x; i < B * 16; i += 256) sdz[i] = dz3[(long long)w * B * 16 + i];
+    const int j = j0 + lane;
+    float w3[16], acc3[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+        w3[c] = (c < d_out) ? __bfloat162float(params[(long long)w * P + oW3 + (long long)c * d_h + j]) : 0.0f;
+        acc3[c] = 0.0f;
+    }
     __syncthreads();
-    float acc[16];
+    float csum = 0.0f;
+    for (int b = wp; b < B; b += 8) {
+        const long long e = ((long long)w * B + b) * d_h + j;
+        const float h = __bfloat162float(h2[e]);
+        float a = 0.0f;
 #pragma unroll
-    for (int c = 0; c < 16; ++c) acc[c] = 0.0f;
-    if (j < d_h) {
-        const bf16 *col = h2 + (long long)w * B * d_h + j;
-        for (int b = 0; b < B; ++b) {
-            const float h = __bfloat162float(col[(long long)b * d_h]);
-#pragma unroll
-            for (int c = 0; c < 16; ++c) acc[c] = fmaf(sdz[b * 16 + c], h, acc[c]);
+        for (int c = 0; c < 16; ++c) {
+            const float d = sdz[b * 16 + c];
+            a = fmaf(d, w3[c], a);
+            acc3[c] = fmaf(d, h, acc3[c]);
         }
-        float *g = grads + (long long)w * P + oW3;
+        const bf16 v = __float2bfloat16_rn(h > 0.0f ? a : 0.0f);
+        dz2[e] = v;
+        csum += __bfloat162float(v);
+    }
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-            if (c < d_out) g[(long long)c * d_h + j] = acc[c];
+    for (int c = 0; c < 16; ++c) red[wp][c][lane] = acc3[c];
+    colsum[wp][lane] = csum;
+    __syncthreads();
+    for (int i = threadIdx.x; i < 16 * 32; i += 256) {
+        const int c = i >> 5, l = i & 31;
+        if (c < d_out) {
+            float s = 0.0f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) s += red[q][c][l];
+            grads[(long long)w * P + oW3 + (long long)c * d_h + j0 + l] = s;
+        }
+    }
+    if (threadIdx.x < 32) {
+        float s = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) s += colsum[q][threadIdx.x];
+        grads[(long long)w * P + ob2 + j0 + threadIdx.x] = s;
     }
     if (blockIdx.x == 0) {
         if (threadIdx.x < d_out) {
@@ -191,58 +243,16 @@ head_dw3(const bf16 *__restrict__ h2, const float *__restrict__ dz3, const float
     }
 }
 
-// dz2[b][j] = bf16((sum_c dz3[b][c] W3[c][j]) * (h2[b][j] > 0)); also dz2T[j][b] and db2[j] = sum_b dz2[b][j].
-// One CTA = 32 columns j x all 128 samples.  grid (d_h / 32, K).
+// db1[j] = sum_b dz1[b][j]: one thread per hidden unit, samples in order.  grid (d_h / 256, K).
 __global__ void __launch_bounds__(256)
-head_dz2(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, const float *__restrict__ dz3,
-         bf16 *__restrict__ dz2, bf16 *__restrict__ dz2T, float *__restrict__ grads, long long P, long long oW3,
-         long long ob2, int B, int d_h, int d_out)
+colsum_bf16(const bf16 *__restrict__ dz, float *__restrict__ grads, long long P, long long ob, int B, int d_h)
 {
-    __shared__ float sdz[128 * 16];
-    __shared__ bf16 tile[32][128 + 8];
-    const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
-    for (int i = threadIdx.x; i < B * 16; i += 256) sdz[i] = dz3[(long long)w * B * 16 + i];
-    const int j = j0 + lane;
-    float w3[16];
-#pragma unroll
-    for (int c = 0; c < 16; ++c)
-        w3[c] = (c < d_out) ? __bfloat162float(params[(long long)w * P + oW3 + (long long)c * d_h + j]) : 0.0f;
-    __syncthreads();
-    for (int b = wp; b < B; b += 8) {
-        float a = 0.0f;
-#pragma unroll
-        for (int c = 0; c < 16; ++c) a = fmaf(sdz[b * 16 + c], w3[c], a);
-        const long long e = ((long long)w * B + b) * d_h + j;
-        const bf16 v = __float2bfloat16_rn(__bfloat162float(h2[e]) > 0.0f ? a : 0.0f);
-        dz2[e] = v;
-        tile[lane][b] = v;
-    }
-    __syncthreads();
-    // transposed rows: 32 rows x 128 samples, 16 bytes per thread
-    for (int i = threadIdx.x; i < 32 * (B / 8); i += 256) {
-        const int r = i / (B / 8), q = i % (B / 8);
-        *reinterpret_cast<uint4 *>(dz2T + ((long long)w * d_h + j0 + r) * B + q * 8) =
-            *reinterpret_cast<const uint4 *>(&tile[r][q * 8]);
-    }
-    if (threadIdx.x < 32) {
-        float s = 0.0f;
-        for (int b = 0; b < B; ++b) s += __bfloat162float(tile[threadIdx.x][b]);
-        grads[(long long)w * P + ob2 + j0 + threadIdx.x] = s;
-    }
-}
-
-// db1[j] = sum_b dz1T[j][b]: one warp per row, fixed summation order.
-__global__ void __launch_bounds__(256)
-rowsum_bf16(const bf16 *__restrict__ dzT, float *__restrict__ grads, long long P, long long ob, int B, int d_h)
-{
-    const int w = blockIdx.y, j = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int w = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
     if (j >= d_h) return;
-    const bf16 *row = dzT + ((long long)w * d_h + j) * B;
+    const bf16 *col = dz + (long long)w * B * d_h + j;
     float s = 0.0f;
-    for (int b = lane; b < B; b += 32) s += __bfloat162float(row[b]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    if (lane == 0) grads[(long long)w * P + ob + j] = s;
+    for (int b = 0; b < B; ++b) s += __bfloat162float(col[(long long)b * d_h]);
+    grads[(long long)w * P + ob + j] = s;
 }
 
 }  // namespace
@@ -250,11 +260,11 @@ rowsum_bf16(const bf16 *__restrict__ dzT, float *__restrict__ grads, long long P
 struct cocod_mlp {
     int K, B, d_in, d_h, d_out;
     long long P, P_raw, oW1, ob1, oW2, ob2, oW3, ob3;
-    bf16 *xT = nullptr, *h1 = nullptr, *h1T = nullptr, *h2 = nullptr, *dz2 = nullptr, *dz2T = nullptr,
-         *dz1T = nullptr, *w2T = nullptr;
+    bf16 *h1 = nullptr, *h2 = nullptr, *dz2 = nullptr, *dz1 = nullptr;
     float *dz3 = nullptr, *rowloss = nullptr;
     int *error_flag = nullptr;
-    CUtensorMap m_h1, m_dz2, m_w2T, m_dz2T, m_h1T, m_dz1T, m_xT;      // maps over scratch (fixed addresses)
+    // maps over scratch (fixed addresses): reduction-contiguous (k) and row-contiguous (mn) views
+    CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
     long long launches = 0;
 };
 
@@ -262,7 +272,7 @@ namespace {
 
 void mlp_free(cocod_mlp *h)
 {
-    void *ptrs[] = {h->xT, h->h1, h->h1T, h->h2, h->dz2, h->dz2T, h->dz1T, h->w2T, h->dz3, h->rowloss, h->error_flag};
+    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag};
     for (void *p : ptrs) if (p) cudaFree(p);
     delete h;
 }
@@ -291,31 +301,27 @@ int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_h
     const size_t act = (size_t)K * batch * d_hidden * sizeof(bf16);
     cudaError_t e = cudaSuccess;
     auto alloc = [&](void **p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
-    alloc((void **)&h->xT, (size_t)K * batch * d_in * sizeof(bf16));
     alloc((void **)&h->h1, act);
-    alloc((void **)&h->h1T, act);
     alloc((void **)&h->h2, act);
     alloc((void **)&h->dz2, act);
-    alloc((void **)&h->dz2T, act);
-    alloc((void **)&h->dz1T, act);
-    alloc((void **)&h->w2T, (size_t)K * d_hidden * d_hidden * sizeof(bf16));
+    alloc((void **)&h->dz1, act);
     alloc((void **)&h->dz3, (size_t)K * batch * 16 * sizeof(float));
     alloc((void **)&h->rowloss, (size_t)K * batch * sizeof(float));
     alloc((void **)&h->error_flag, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->error_flag, 0, sizeof(int));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(head_logits, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * d_hidden * (int)sizeof(bf16));
     if (e != cudaSuccess) {
         cudaGetLastError();
         mlp_free(h);
         return e == cudaErrorMemoryAllocation ? COCOD_ERR_OOM : COCOD_ERR_CUDA;
     }
-    const uint64_t uK = K, uB = batch, uh = d_hidden, ui = d_in;
-    bool ok = make_map(&h->m_h1, h->h1, uh, uB, uK, uh, uB * uh)           // [B][d_h]
-              && make_map(&h->m_dz2, h->dz2, uh, uB, uK, uh, uB * uh)      // [B][d_h]
-              && make_map(&h->m_w2T, h->w2T, uh, uh, uK, uh, uh * uh)      // [d_h in][d_h out]
-              && make_map(&h->m_dz2T, h->dz2T, uB, uh, uK, uB, uh * uB)    // [d_h][B]
-              && make_map(&h->m_h1T, h->h1T, uB, uh, uK, uB, uh * uB)      // [d_h][B]
-              && make_map(&h->m_dz1T, h->dz1T, uB, uh, uK, uB, uh * uB)    // [d_h][B]
-              && make_map(&h->m_xT, h->xT, uB, ui, uK, uB, ui * uB);       // [d_in][B]
+    const uint64_t uK = K, uB = batch, uh = d_hidden;
+    // activations are [B][d_h] per worker: as a reduction-contiguous operand the reduction runs over
+    // d_h; as a row-contiguous operand the reduction runs over the batch.
+    bool ok = map_k(&h->k_h1, h->h1, uh, uB, uK, uh, uB * uh) && map_k(&h->k_dz2, h->dz2, uh, uB, uK, uh, uB * uh) &&
+              map_mn(&h->mn_dz2, h->dz2, uh, uB, uK, uh, uB * uh) && map_mn(&h->mn_h1, h->h1, uh, uB, uK, uh, uB * uh) &&
+              map_mn(&h->mn_dz1, h->dz1, uh, uB, uK, uh, uB * uh);
     if (!ok) {
         mlp_free(h);
         return COCOD_ERR_CUDA;
@@ -340,69 +346,60 @@ int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, 
                    float *loss, cocod_stream_t stream)
 {
     if (!h || !params_bf16 || !x || !labels || !grads || !loss) return COCOD_ERR_INVALID;
-    if ((reinterpret_cast<uintptr_t>(params_bf16) & 15u) || (reinterpret_cast<uintptr_t>(x) & 15u))
+    if ((reinterpret_cast<uintptr_t>(params_bf16) & 15u) || (reinterpret_cast<uintptr_t>(x) & 15u) ||
+        (reinterpret_cast<uintptr_t>(grads) & 15u))
         return COCOD_ERR_INVALID;
     cudaStream_t s = (cudaStream_t)stream;
     const bf16 *prm = static_cast<const bf16 *>(params_bf16);
     const bf16 *xin = static_cast<const bf16 *>(x);
     const int K = h->K, B = h->B, d_in = h->d_in, d_h = h->d_h, d_out = h->d_out;
     const long long P = h->P;
-    // maps over caller memory: x [B][d_in], W1 [d_h][d_in], W2 [d_h][d_h]
-    CUtensorMap m_x, m_w1, m_w2;
-    if (!make_map(&m_x, xin, d_in, B, K, d_in, (uint64_t)B * d_in) ||
-        !make_map(&m_w1, prm + h->oW1, d_in, d_h, K, d_in, P) ||
-        !make_map(&m_w2, prm + h->oW2, d_h, d_h, K, d_h, P))
+    const uint64_t uK = K, uB = B, uh = d_h, ui = d_in, uP = P;
+    // maps over caller memory
+    CUtensorMap k_x, mn_x, k_w1, k_w2, mn_w2, c_w1, c_w2, none{};
+    if (!map_k(&k_x, xin, ui, uB, uK, ui, uB * ui) || !map_mn(&mn_x, xin, ui, uB, uK, ui, uB * ui) ||
+        !map_k(&k_w1, prm + h->oW1, ui, uh, uK, ui, uP) || !map_k(&k_w2, prm + h->oW2, uh, uh, uK, uh, uP) ||
+        !map_mn(&mn_w2, prm + h->oW2, uh, uh, uK, uh, uP) ||
+        !map_out(&c_w1, grads + h->oW1, ui, uh, uK, ui, uP) || !map_out(&c_w2, grads + h->oW2, uh, uh, uK, uh, uP))
         return COCOD_ERR_CUDA;
 #define LAUNCH_OK() do { if (cudaGetLastError() != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
-    // transposed copies: xT [d_in][B], w2T [d_h in][d_h out]
-    transpose_bf16<<<dim3((d_in + 31) / 32, (B + 31) / 32, K), 256, 0, s>>>(xin, h->xT, B, d_in, d_in,
-                                                                            (long long)B * d_in, (long long)B * d_in);
-    LAUNCH_OK();
-    transpose_bf16<<<dim3(d_h / 32, d_h / 32, K), 256, 0, s>>>(prm + h->oW2, h->w2T, d_h, d_h, d_h, P,
-                                                               (long long)d_h * d_h);
-    LAUNCH_OK();
+#define GEMM_OK(call) do { if ((call) != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
     Params p{};
     p.error_flag = h->error_flag;
     // h1 = relu(x W1^T + b1)
-    p.M = B; p.N = d_h; p.K = d_in;
-    p.o = h->h1; p.oT = h->h1T; p.o_worker_stride = (long long)B * d_h;
+    p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
+    p.o = h->h1; p.o_worker_stride = (long long)B * d_h;
     p.bias = prm + h->ob1; p.bias_worker_stride = P;
-    if (launch_gemm<EPI_BIAS_RELU>(m_x, m_w1, p, K, s) != cudaSuccess) return COCOD_ERR_CUDA;
-    ++h->launches;
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, none, p, K, s)));
     // h2 = relu(h1 W2^T + b2)
-    p.K = d_h; p.o = h->h2; p.oT = nullptr; p.bias = prm + h->ob2;
-    if (launch_gemm<EPI_BIAS_RELU>(h->m_h1, m_w2, p, K, s) != cudaSuccess) return COCOD_ERR_CUDA;
-    ++h->launches;
-    // output layer, loss, dz3, dW3, db3, dz2, db2
-    head_logits<<<K * B / 8, 256, 0, s>>>(h->h2, prm, P, h->oW3, h->ob3, labels, h->dz3, h->rowloss, B, d_h, d_out);
+    p.K = d_h; p.stages = stages_for(d_h); p.o = h->h2; p.bias = prm + h->ob2;
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, none, p, K, s)));
+    // output layer, loss, dz3; then dz2, dW3, db3, db2
+    head_logits<<<dim3(B / 16, K), 256, (size_t)d_out * d_h * sizeof(bf16), s>>>(h->h2, prm, P, h->oW3, h->ob3, labels,
+                                                                                h->dz3, h->rowloss, B, d_h, d_out);
     LAUNCH_OK();
-    head_dw3<<<dim3((d_h + 255) / 256, K), 256, 0, s>>>(h->h2, h->dz3, h->rowloss, grads, loss, P, h->P_raw, h->oW3,
-                                                        h->ob3, B, d_h, d_out);
+    head_backward<<<dim3(d_h / 32, K), 256, 0, s>>>(h->h2, prm, h->dz3, h->rowloss, h->dz2, grads, loss, P, h->P_raw,
+                                                    h->oW3, h->ob2, h->ob3, B, d_h, d_out);
     LAUNCH_OK();
-    head_dz2<<<dim3(d_h / 32, K), 256, 0, s>>>(h->h2, prm, h->dz3, h->dz2, h->dz2T, grads, P, h->oW3, h->ob2, B, d_h,
-                                               d_out);
-    LAUNCH_OK();
-    // dz1T = ((dz2 W2) * (h1 > 0))^T
+    // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
     Params q{};
     q.error_flag = h->error_flag;
-    q.M = B; q.N = d_h; q.K = d_h;
-    q.o = nullptr; q.oT = h->dz1T; q.o_worker_stride = (long long)B * d_h;
+    q.M = B; q.N = d_h; q.K = d_h; q.stages = stages_for(d_h);
+    q.o = h->dz1; q.o_worker_stride = (long long)B * d_h;
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
-    if (launch_gemm<EPI_MASK>(h->m_dz2, h->m_w2T, q, K, s) != cudaSuccess) return COCOD_ERR_CUDA;
-    ++h->launches;
-    rowsum_bf16<<<dim3((d_h + 7) / 8, K), 256, 0, s>>>(h->dz1T, grads, P, h->ob1, B, d_h);
+    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, none, q, K, s)));
+    colsum_bf16<<<dim3((d_h + 255) / 256, K), 256, 0, s>>>(h->dz1, grads, P, h->ob1, B, d_h);
     LAUNCH_OK();
-    // dW2 = dz2T h1T^T, dW1 = dz1T xT^T
+    // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
     Params r{};
     r.error_flag = h->error_flag;
-    r.M = d_h; r.N = d_h; r.K = B;
-    r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h;
-    if (launch_gemm<EPI_F32>(h->m_dz2T, h->m_h1T, r, K, s) != cudaSuccess) return COCOD_ERR_CUDA;
-    ++h->launches;
+    r.M = d_h; r.N = d_h; r.K = B; r.stages = stages_for(B);
+    r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
+    GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s)));
     r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
-    if (launch_gemm<EPI_F32>(h->m_dz1T, h->m_xT, r, K, s) != cudaSuccess) return COCOD_ERR_CUDA;
-    ++h->launches;
+    GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s)));
 #undef LAUNCH_OK
+#undef GEMM_OK
     return COCOD_OK;
 }
 
@@ -416,18 +413,22 @@ int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream)
     return flag ? COCOD_ERR_TIMEOUT : COCOD_OK;
 }
 
-int cocod_gemm_tn_bf16(const void *A, const void *B, float *C, int M, int N, int Kd, int batch_count, int64_t lda,
-                       int64_t ldb, int64_t ldc, int64_t stride_a, int64_t stride_b, int64_t stride_c,
-                       cocod_stream_t stream)
+int cocod_gemm_bf16(const void *A, const void *B, float *C, int M, int N, int Kd, int batch_count, int a_rows_contiguous,
+                    int b_rows_contiguous, int64_t lda, int64_t ldb, int64_t ldc, int64_t stride_a, int64_t stride_b,
+                    int64_t stride_c, cocod_stream_t stream)
 {
     if (!A || !B || !C || M < 1 || N < 1 || Kd < 1 || batch_count < 1 || batch_count > 65535) return COCOD_ERR_INVALID;
-    if ((lda % 8) || (ldb % 8) || (stride_a % 8) || (stride_b % 8) || lda < Kd || ldb < Kd || ldc < N)
+    const int64_t a_cols = a_rows_contiguous ? M : Kd, a_rows = a_rows_contiguous ? Kd : M;
+    const int64_t b_cols = b_rows_contiguous ? N : Kd, b_rows = b_rows_contiguous ? Kd : N;
+    if ((lda % 8) || (ldb % 8) || (stride_a % 8) || (stride_b % 8) || lda < a_cols || ldb < b_cols || ldc < N)
         return COCOD_ERR_INVALID;
     if ((reinterpret_cast<uintptr_t>(A) & 15u) || (reinterpret_cast<uintptr_t>(B) & 15u)) return COCOD_ERR_INVALID;
-    CUtensorMap ma, mb;
-    const uint64_t sa = batch_count > 1 ? (uint64_t)stride_a : (uint64_t)M * lda;
-    const uint64_t sb = batch_count > 1 ? (uint64_t)stride_b : (uint64_t)N * ldb;
-    if (!make_map(&ma, A, Kd, M, batch_count, lda, sa) || !make_map(&mb, B, Kd, N, batch_count, ldb, sb))
+    CUtensorMap ma, mb, mc{};
+    const uint64_t sa = batch_count > 1 ? (uint64_t)stride_a : (uint64_t)a_rows * lda;
+    const uint64_t sb = batch_count > 1 ? (uint64_t)stride_b : (uint64_t)b_rows * ldb;
+    const uint64_t sc = batch_count > 1 ? (uint64_t)stride_c : (uint64_t)M * ldc;
+    if (!make_map(&ma, A, a_cols, a_rows, batch_count, lda, sa, a_rows_contiguous ? 64 : 128) ||
+        !make_map(&mb, B, b_cols, b_rows, batch_count, ldb, sb, b_rows_contiguous ? 64 : 128))
         return COCOD_ERR_CUDA;
     static int *flag = nullptr;
     if (!flag) {
@@ -435,13 +436,20 @@ int cocod_gemm_tn_bf16(const void *A, const void *B, float *C, int M, int N, int
         cudaMemset(flag, 0, sizeof(int));
     }
     Params p{};
-    p.M = M; p.N = N; p.K = Kd;
-    p.c = C; p.c_worker_stride = stride_c; p.ldc = (int)ldc;
+    p.M = M; p.N = N; p.K = Kd; p.stages = stages_for(Kd);
+    p.c = C; p.c_worker_stride = (long long)sc; p.ldc = (int)ldc;
+    p.map_c_ok = map_out(&mc, C, N, M, batch_count, ldc, sc) ? 1 : 0;      // else: plain predicated stores
     p.error_flag = flag;
-    if (launch_gemm<EPI_F32>(ma, mb, p, batch_count, (cudaStream_t)stream) != cudaSuccess) return COCOD_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e;
+    if (a_rows_contiguous && b_rows_contiguous) e = launch_gemm<EPI_F32, true, true>(ma, mb, mc, p, batch_count, s);
+    else if (a_rows_contiguous) e = launch_gemm<EPI_F32, true, false>(ma, mb, mc, p, batch_count, s);
+    else if (b_rows_contiguous) e = launch_gemm<EPI_F32, false, true>(ma, mb, mc, p, batch_count, s);
+    else e = launch_gemm<EPI_F32, false, false>(ma, mb, mc, p, batch_count, s);
+    if (e != cudaSuccess) return COCOD_ERR_CUDA;
     int f = 0;
-    if (cudaMemcpyAsync(&f, flag, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess ||
-        cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess)
+    if (cudaMemcpyAsync(&f, flag, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
         return COCOD_ERR_CUDA;
     if (f) {
         cudaMemset(flag, 0, sizeof(int));

@@ -19,7 +19,7 @@ SIGNATURES = {
     "cocod_mlp_grad": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "cocod_mlp_check": (_i, [_vp, _vp]),
     "cocod_mlp_launch_count": (_i64, [_vp]),
-    "cocod_gemm_tn_bf16": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i64, _i64, _i64, _i64, _i64, _i64, _vp]),
+    "cocod_gemm_bf16": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i64, _i64, _i64, _vp]),
 }
 
 _declared = False
@@ -94,11 +94,14 @@ class MLPGrad:
             pass
 
 
-def gemm_tn_bf16(A, B, C, stream=None):
-    """C[w] = A[w] @ B[w].T for CUDA tensors A (W x M x K bf16), B (W x N x K bf16), C (W x M x N fp32)."""
-    W, M, K = A.shape
-    N = B.shape[1]
-    rc = load().cocod_gemm_tn_bf16(A.data_ptr(), B.data_ptr(), C.data_ptr(), M, N, K, W, A.stride(1), B.stride(1),
-                                   C.stride(1), A.stride(0), B.stride(0), C.stride(0), _cur_stream(stream))
+def gemm_bf16(A, B, C, a_rows_contiguous=False, b_rows_contiguous=False, stream=None):
+    """C[w][m][n] = sum_k A_w(m, k) B_w(n, k) for CUDA tensors: A is W x M x K (or W x K x M when
+    a_rows_contiguous), B is W x N x K (or W x K x N when b_rows_contiguous), both bf16; C is
+    W x M x N fp32."""
+    W, M, N = C.shape
+    K = A.shape[1] if a_rows_contiguous else A.shape[2]
+    rc = load().cocod_gemm_bf16(A.data_ptr(), B.data_ptr(), C.data_ptr(), M, N, K, W, int(a_rows_contiguous),
+                                int(b_rows_contiguous), A.stride(1), B.stride(1), C.stride(1), A.stride(0),
+                                B.stride(0), C.stride(0), _cur_stream(stream))
     if rc != _E.OK:
-        raise _E.CocodError(rc, "cocod_gemm_tn_bf16")
+        raise _E.CocodError(rc, "cocod_gemm_bf16")

@@ -70,7 +70,7 @@ def test_error_paths_that_touch_no_device(libs):
     assert lib.cocod_mlp_create(ctypes.byref(out), 2, 128, 784, 1024, 17) == engine.ERR_INVALID
     assert lib.cocod_mlp_grad(None, None, None, None, None, None, None) == engine.ERR_INVALID
     assert lib.cocod_mlp_destroy(None) == engine.OK
-    assert lib.cocod_gemm_tn_bf16(None, None, None, 1, 1, 1, 1, 8, 8, 8, 8, 8, 8, None) == engine.ERR_INVALID
+    assert lib.cocod_gemm_bf16(None, None, None, 1, 1, 1, 1, 0, 0, 8, 8, 8, 8, 8, 8, None) == engine.ERR_INVALID
 
 
 def test_engine_refuses_to_run_without_a_gpu(libs):

@@ -46,14 +46,19 @@ def bf16_tensor(a):
     return torch.from_numpy(a).cuda().to(torch.bfloat16)
 
 
+@pytest.mark.parametrize("a_t,b_t", [(False, False), (False, True), (True, True), (True, False)])
 @pytest.mark.parametrize("W,Mm,N,K", [(1, 128, 128, 64), (1, 128, 128, 256), (3, 128, 256, 784), (2, 256, 384, 128),
-                                      (16, 128, 1024, 1024), (2, 1024, 784, 128), (1, 100, 200, 72), (2, 130, 8, 1000)])
-def test_tensor_core_gemm_matches_the_definition(M, W, Mm, N, K):
+                                      (16, 128, 1024, 1024), (2, 1024, 784, 128), (1, 104, 200, 72), (2, 136, 8, 1000)])
+def test_tensor_core_gemm_matches_the_definition(M, W, Mm, N, K, a_t, b_t):
+    """Every storage combination: operands with the reduction index contiguous ([M][K], [N][K]) or
+    with the row index contiguous ([K][M], [K][N]); tiles, ragged edges, batches."""
     rng = np.random.default_rng(W * 7 + Mm + N + K)
     A = I.round_to_bf16(rng.standard_normal((W, Mm, K)).astype(np.float32))
     B = I.round_to_bf16(rng.standard_normal((W, N, K)).astype(np.float32))
     C = torch.full((W, Mm, N), float("nan"), dtype=torch.float32, device="cuda")
-    M.gemm_tn_bf16(bf16_tensor(A), bf16_tensor(B), C)
+    Ad = bf16_tensor(np.ascontiguousarray(A.transpose(0, 2, 1)) if a_t else A)
+    Bd = bf16_tensor(np.ascontiguousarray(B.transpose(0, 2, 1)) if b_t else B)
+    M.gemm_bf16(Ad, Bd, C, a_rows_contiguous=a_t, b_rows_contiguous=b_t)
     want = np.einsum("wmk,wnk->wmn", A.astype(np.float64), B.astype(np.float64))
     got = cpu(C).astype(np.float64)
     assert np.isfinite(got).all()
