@@ -195,9 +195,18 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
     }
     __syncthreads();
     float csum = 0.0f;
-    for (int b = wp; b < B; b += 8) {
+    float hreg[16];                               // this thread's 16 samples of column j, loaded up front
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+        const int b = wp + 8 * q;
+        hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
+    }
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+        const int b = wp + 8 * q;
+        if (b >= B) break;
         const long long e = ((long long)w * B + b) * d_h + j;
-        const float h = __bfloat162float(h2[e]);
+        const float h = hreg[q];
         float a = 0.0f;
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
@@ -251,7 +260,13 @@ colsum_bf16(const bf16 *__restrict__ dz, float *__restrict__ grads, long long P,
     if (j >= d_h) return;
     const bf16 *col = dz + (long long)w * B * d_h + j;
     float s = 0.0f;
-    for (int b = 0; b < B; ++b) s += __bfloat162float(col[(long long)b * d_h]);
+    for (int b0 = 0; b0 < B; b0 += 16) {          // 16 independent loads in flight, summed in sample order
+        float t[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) t[q] = (b0 + q < B) ? __bfloat162float(col[(long long)(b0 + q) * d_h]) : 0.0f;
+#pragma unroll
+        for (int q = 0; q < 16; ++q) s += t[q];
+    }
     grads[(long long)w * P + ob + j] = s;
 }
 
