@@ -75,6 +75,13 @@ int cocod_gemm_bf16(const void *A, const void *B, float *C, int M, int N, int K,
                     int a_rows_contiguous, int b_rows_contiguous, int64_t lda, int64_t ldb, int64_t ldc,
                     int64_t stride_a, int64_t stride_b, int64_t stride_c, cocod_stream_t stream);
 
+/* Self-test of the kernels' bounded waits (failure detection without a GPU fault): launches one
+ * tile whose operand copies are deliberately never issued, so the thread that issues the tensor-core
+ * instructions waits on a barrier nothing will flip.  After wait_ms (1..2000) the kernel gives up,
+ * records the fact, releases its tensor memory and returns; the call then returns COCOD_ERR_TIMEOUT
+ * and the CUDA context stays usable.  (COCOD_OK would mean the wait did not run out.) */
+int cocod_gemm_wait_selftest(int wait_ms, cocod_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

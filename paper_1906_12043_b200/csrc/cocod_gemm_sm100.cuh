@@ -54,6 +54,8 @@ struct Params {
     long long mask_worker_stride;
     int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
     int *error_flag;
+    unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
+    int debug_no_loads;                // self-test: the producer issues nothing, so the waits run out
 };
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
@@ -83,15 +85,16 @@ __device__ __forceinline__ unsigned long long now_ns()
     return t;
 }
 // Wait for a barrier phase, giving up after WAIT_LIMIT_NS or when another role has aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort,
+                                          unsigned long long limit_ns)
 {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = now_ns();
     for (unsigned it = 0;; ++it) {
         if (mbar_try(bar, parity)) return true;
-        if ((it & 255u) == 255u) {
+        if ((it & 63u) == 63u) {
             if (*abort) return false;
-            if (now_ns() - t0 > WAIT_LIMIT_NS) return false;
+            if (now_ns() - t0 > limit_ns) return false;
         }
     }
 }
@@ -197,6 +200,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, wk = blockIdx.z;
     const int nkb = (p.K + BK - 1) / BK;
     const uint32_t smem_base = smem_u32(smem);
+    const unsigned long long limit = p.wait_ns ? p.wait_ns : WAIT_LIMIT_NS;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -223,9 +227,9 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     if (warp == 0 && lane == 0) {
         // ---- producer: TMA loads of the A and B tiles of every 64-wide reduction block
         int armed = 0;
-        for (int kb = 0; kb < nkb; ++kb) {
+        for (int kb = 0; kb < nkb && !p.debug_no_loads; ++kb) {
             const int s = kb % stages;
-            if (kb >= stages && !mbar_wait(empty0 + 8 * s, ((kb / stages) - 1) & 1, abort)) { failed = 1; break; }
+            if (kb >= stages && !mbar_wait(empty0 + 8 * s, ((kb / stages) - 1) & 1, abort, limit)) { failed = 1; break; }
             const uint32_t bar = full0 + 8 * s;
             mbar_expect_tx(bar, STAGE_BYTES);
             const uint32_t dst_a = smem_base + s * STAGE_BYTES, dst_b = dst_a + A_BYTES;
@@ -246,7 +250,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (failed) {                 // let copies that were already issued land before leaving
             abort[0] = 1;
             for (int kb = (armed > stages ? armed - stages : 0); kb < armed; ++kb)
-                mbar_wait(full0 + 8 * (kb % stages), (kb / stages) & 1, never);
+                mbar_wait(full0 + 8 * (kb % stages), (kb / stages) & 1, never, limit);
         }
     } else if (warp == 1 && lane == 0) {
         // ---- MMA issuer
@@ -254,7 +258,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         constexpr uint32_t a_step = A_MN ? 2048u : (uint32_t)(UMMA_K * 2), b_step = B_MN ? 2048u : (uint32_t)(UMMA_K * 2);
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % stages;
-            if (!mbar_wait(full0 + 8 * s, (kb / stages) & 1, abort)) { failed = 2; break; }
+            if (!mbar_wait(full0 + 8 * s, (kb / stages) & 1, abort, limit)) { failed = 2; break; }
             tc_fence_after();
             const uint32_t a_addr = smem_base + s * STAGE_BYTES, b_addr = a_addr + A_BYTES;
 #pragma unroll
@@ -271,7 +275,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     __syncwarp();
 
     // ---- epilogue: every thread owns one accumulator row (TMEM lane) of the tile
-    bool ok = mbar_wait(accum, 0, abort);
+    bool ok = mbar_wait(accum, 0, abort, limit + limit / 2);
     ok = __all_sync(0xffffffffu, ok);
     if (__syncthreads_and(ok ? 1 : 0)) {
         tc_fence_after();

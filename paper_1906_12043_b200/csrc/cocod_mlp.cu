@@ -473,4 +473,33 @@ int cocod_gemm_bf16(const void *A, const void *B, float *C, int M, int N, int Kd
     return COCOD_OK;
 }
 
+// Self-test of the bounded waits: one tile whose operand copies are never issued.
+int cocod_gemm_wait_selftest(int wait_ms, cocod_stream_t stream)
+{
+    if (wait_ms < 1 || wait_ms > 2000) return COCOD_ERR_INVALID;
+    static bf16 *buf = nullptr;
+    static int *flag = nullptr;
+    if (!buf) {
+        if (cudaMalloc((void **)&buf, 128 * 64 * sizeof(bf16)) != cudaSuccess) return COCOD_ERR_OOM;
+        if (cudaMalloc((void **)&flag, sizeof(int)) != cudaSuccess) return COCOD_ERR_OOM;
+        cudaMemset(buf, 0, 128 * 64 * sizeof(bf16));
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(flag, 0, sizeof(int), s) != cudaSuccess) return COCOD_ERR_CUDA;
+    CUtensorMap m, none{};
+    if (!map_k(&m, buf, 64, 128, 1, 64, 128 * 64)) return COCOD_ERR_CUDA;
+    Params p{};
+    p.M = 128; p.N = 128; p.K = 64; p.stages = 1;
+    p.c = nullptr; p.map_c_ok = 0;
+    p.error_flag = flag;
+    p.wait_ns = (unsigned long long)wait_ms * 1000000ull;
+    p.debug_no_loads = 1;
+    if (launch_gemm<EPI_F32, false, false>(m, m, none, p, 1, s) != cudaSuccess) return COCOD_ERR_CUDA;
+    int f = 0;
+    if (cudaMemcpyAsync(&f, flag, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    return f ? COCOD_ERR_TIMEOUT : COCOD_OK;
+}
+
 }  // extern "C"

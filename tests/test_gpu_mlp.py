@@ -283,3 +283,15 @@ def test_end_to_end_rounds_match_the_oracle_loop(M, E):
     for a, b in curve2:
         assert abs(a - b) < 2e-2 * abs(b)
     assert curve2[-1][0] < curve2[0][0]              # it learns
+
+
+def test_a_wait_that_nothing_satisfies_times_out_and_leaves_the_gpu_usable(M, E):
+    """Failure detection without a fault: the tile's operand copies are never issued, the waiting
+    threads give up after 50 ms, the kernel frees its tensor memory and reports the timeout; the
+    context then still runs correct work."""
+    assert M.gemm_wait_selftest(50) == E.ERR_TIMEOUT
+    A = I.round_to_bf16(np.random.default_rng(0).standard_normal((1, 128, 64)).astype(np.float32))
+    C = torch.zeros((1, 128, 128), dtype=torch.float32, device="cuda")
+    M.gemm_bf16(bf16_tensor(A), bf16_tensor(A), C)
+    np.testing.assert_allclose(cpu(C)[0], A[0].astype(np.float64) @ A[0].astype(np.float64).T, rtol=0, atol=1e-4)
+    assert M.gemm_wait_selftest(20) == E.ERR_TIMEOUT     # and again

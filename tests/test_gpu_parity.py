@@ -290,6 +290,21 @@ def test_state_machine_and_argument_errors(E):
     eng.destroy()                                   # idempotent
 
 
+def test_comm_wait_reports_timeout_then_completion(E):
+    """Host-side failure detection: polling the averaging with no time allowance returns TIMEOUT (or
+    OK if it already finished) and never blocks; a later wait with allowance returns OK."""
+    K, P = 16, 4_000_000
+    eng = E.Engine(K, P, 0.1, 0.9, 0.0)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        torch.cuda._sleep(200_000_000)              # keeps the side stream busy for ~0.1 s
+    eng.comm_begin(side)
+    assert eng.comm_wait(0) == E.ERR_TIMEOUT
+    assert eng.comm_wait(5000) == E.OK
+    eng.comm_end()
+    eng.sync()
+
+
 def test_host_gradient_entry_point_matches_device_entry_point(E):
     K, P = 4, 300_000
     x0 = I.initial_point(P)
