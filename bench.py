@@ -41,6 +41,8 @@ def parse():
     ap.add_argument("--k", type=int, default=None, help="override the workload's local steps per round")
     ap.add_argument("--snapshot", default="flip", choices=["flip", "copy"])
     ap.add_argument("--ring", type=int, default=4, help="distinct gradient buffers cycled through")
+    ap.add_argument("--graph", action="store_true",
+                    help="replay the timed rounds from a CUDA graph of two rounds (launch-bound workloads)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-cols", type=int, default=1 << 20)
@@ -230,22 +232,54 @@ def run_ours(args, wl):
     # ---- device-resident timed region
     for _ in range(max(3, args.warmup)):
         one_round(side)
-    eng.set_option(E.OPT_PROFILE, 1)
-    eng.profile_reset()
+    graph = None
+    if args.graph:
+        # two rounds = one full cycle of the buffer flip; the side-stream mean is captured with them
+        cap = torch.cuda.Stream()
+        eng.sync()
+        eng.set_stream(cap)
+        with torch.cuda.stream(cap):
+            one_round(side)
+            one_round(side)
+        torch.cuda.synchronize()
+        step_no[0] = 0
+        l_before = eng.launch_count
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=cap):
+            one_round(side)
+            one_round(side)
+        launches_per_replay = eng.launch_count - l_before
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+    else:
+        eng.set_option(E.OPT_PROFILE, 1)
+        eng.profile_reset()
     barrier()
     sampler = ClockSampler(local_rank) if rank == 0 else None
     launches0 = eng.launch_count
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(compute)
-    for _ in range(args.steps):
-        one_round(side)
+    if graph is not None:
+        args.steps = max(2, args.steps // 2 * 2)
+        for _ in range(args.steps // 2):
+            graph.replay()
+    else:
+        for _ in range(args.steps):
+            one_round(side)
     ev1.record(compute)
     barrier()
     clocks = sampler.stop() if sampler else None
     ms = ev0.elapsed_time(ev1)
-    launches = eng.launch_count - launches0
-    by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
-    eng.set_option(E.OPT_PROFILE, 0)
+    if graph is not None:
+        launches = launches_per_replay * (args.steps // 2)
+        by = {}
+        eng.sync()
+        eng.set_stream(compute)
+    else:
+        launches = eng.launch_count - launches0
+        by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+        eng.set_option(E.OPT_PROFILE, 0)
     if world > 1:
         t = torch.tensor([ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -284,7 +318,7 @@ def run_ours(args, wl):
     dom = "local_step"
     traffic = W.NCU_DRAM_BYTES_PER_WORKER_PARAM.get(dom)
     traffic = traffic * K * P if traffic is not None else None
-    dom_tab = in_loop.get(dom, {})
+    dom_tab = in_loop.get(dom) or isolated.get(dom, {})      # graph replays carry no per-kernel events
     roofline = {"bound": "hbm", "kernel": dom, "achieved": dom_tab.get("gbs"), "peak": hbm_peak,
                 "unit": "GB/s", "frac": dom_tab.get("frac_of_peak"), "traffic": traffic,
                 "peak_kind": peak_kind, "algorithmic_bytes_per_launch": alg_bytes[dom],
@@ -347,7 +381,7 @@ def run_ours(args, wl):
             "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "K": K, "P": P, "k": k, "lr": wl.lr, "mu": wl.mu, "wd": wl.wd,
-                       "snapshot": args.snapshot, "gradient_ring": len(ring),
+                       "snapshot": args.snapshot, "gradient_ring": len(ring), "cuda_graph": bool(args.graph),
                        "l2": "inputs larger than L2 (each K x P buffer is %.0f MB, L2 is 126 MB)" % (K * P * 4 / 1e6)
                              if K * P * 4 > 126e6 else "L2-resident workload: not an HBM number",
                        "sharding": "columns, no exchange" if world > 1 else "single GPU"},
@@ -415,18 +449,44 @@ def run_mlp(args):
     for r in range(max(3, args.warmup)):
         one_round(record=True)
     torch.cuda.synchronize()
+    graph = None
+    if args.graph:
+        cap = torch.cuda.Stream()
+        eng.set_stream(cap)
+        with torch.cuda.stream(cap):
+            one_round()
+            one_round()
+        torch.cuda.synchronize()
+        step_no[0] = 0
+        lb = eng.launch_count + mg.launch_count
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=cap):
+            one_round()
+            one_round()
+        per_replay = eng.launch_count + mg.launch_count - lb
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        args.steps = max(2, args.steps // 2 * 2)
     sampler = ClockSampler(0)
     l0 = eng.launch_count + mg.launch_count
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(compute)
-    for _ in range(args.steps):
-        one_round()
+    if graph is not None:
+        for _ in range(args.steps // 2):
+            graph.replay()
+    else:
+        for _ in range(args.steps):
+            one_round()
     ev1.record(compute)
     torch.cuda.synchronize()
     clocks = sampler.stop()
     mg.check()
     ms = ev0.elapsed_time(ev1)
-    launches = eng.launch_count + mg.launch_count - l0
+    launches = per_replay * (args.steps // 2) if graph is not None else eng.launch_count + mg.launch_count - l0
+    if graph is not None:
+        eng.sync()
+        eng.set_stream(compute)
     final_loss = float(loss.mean().item())
 
     # end to end: minibatches and labels start in pinned host memory, the loss comes back every step
@@ -467,7 +527,7 @@ def run_mlp(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 contractions / f32 state",
         "data": "synthetic",
         "config": {"workload": "mlp", "K": K, "P": P_raw, "P_padded": P, "k": k, "lr": lr, "mu": mu, "wd": wd,
-                   "mlp": list(dims), "batch": B, "minibatch_ring": ring_n},
+                   "mlp": list(dims), "batch": B, "minibatch_ring": ring_n, "cuda_graph": bool(args.graph)},
         "clocks": clocks, "gpu_launches": launches,
         "local_steps_per_s": k * args.steps / (ms * 1e-3), "ms_per_local_step": ms / (k * args.steps),
         "tensor_tflops": flops_step * k * args.steps / (ms * 1e-3) / 1e12,

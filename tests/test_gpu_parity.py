@@ -356,6 +356,53 @@ def test_save_restore_resumes_bit_exactly(E):
     assert_bit_equal(cpu(c.get_momentum()), cpu(a.get_momentum()))
 
 
+def test_rounds_replayed_from_a_cuda_graph_match_eager_rounds(E):
+    """No call of a round blocks the host, so two rounds (one full cycle of the buffer flip) can be
+    captured into a CUDA graph, side-stream averaging included, and replayed; the replays must equal
+    eagerly issued rounds bit for bit."""
+    K, P, k = 4, 100_000, 4
+    x0 = I.initial_point(P)
+    cap = torch.cuda.Stream()
+    side = torch.cuda.Stream(priority=-1)
+    static_g = [torch.empty((K, P), dtype=torch.float32, device="cuda") for _ in range(2 * k)]
+    eager, graphed = E.Engine(K, P, 0.1, 0.9, 5e-4), E.Engine(K, P, 0.1, 0.9, 5e-4)
+    for eng in (eager, graphed):
+        eng.set_params(x0)
+    graphed.sync()
+    graphed.set_stream(cap)
+
+    def two_rounds(eng):
+        for r in range(2):
+            eng.comm_begin(side)
+            for s in range(k):
+                eng.local_step(static_g[r * k + s])
+            eng.comm_end()
+
+    def load(block):
+        for i, g in enumerate(static_g):
+            g.copy_(torch.from_numpy(I.gradients(K, P, block * 2 * k + i)))
+
+    load(0)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(cap):
+        two_rounds(graphed)                          # warm-up on the capture stream
+    two_rounds(eager)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    load(1)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=cap):
+        two_rounds(graphed)
+    for block in (1, 2, 3):
+        load(block)
+        torch.cuda.synchronize()
+        graph.replay()
+        two_rounds(eager)
+        torch.cuda.synchronize()
+        assert_bit_equal(cpu(graphed.get_params()), cpu(eager.get_params()), f"x after block {block}")
+        assert_bit_equal(cpu(graphed.get_momentum()), cpu(eager.get_momentum()), f"v after block {block}")
+
+
 def test_learning_rate_schedule_and_profile_records(E):
     K, P = 2, 4096
     eng = E.Engine(K, P, 0.1, 0.9, 0.0)
