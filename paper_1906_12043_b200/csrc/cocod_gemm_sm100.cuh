@@ -7,7 +7,7 @@
 // read both forms from shared memory, so no operand is ever transposed in memory.  One CTA
 // computes one 128 x 128 tile of one worker:
 //   * operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
-//     shared-memory ring of up to 4 stages guarded by mbarriers;
+//     shared-memory ring of up to 6 stages (32 KB each) guarded by mbarriers;
 //   * one elected thread issues tcgen05.mma (kind::f16, bf16 inputs, fp32 accumulation) on
 //     shared-memory descriptors; the 128 x 128 fp32 accumulator lives in TMEM (128 columns);
 //   * all four warps read the accumulator back with tcgen05.ld (32 lanes x 32 columns at a time)
@@ -27,11 +27,14 @@
 namespace cocod {
 namespace gemm {
 
-constexpr int BM = 128, BN = 128, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int BM = 128, BN = 128, BK = 64, STAGES = 6, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 128;
 constexpr int MAX_STAGES = STAGES;
-__host__ __device__ constexpr int smem_bytes(int stages) { return stages * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */; }
+// ring (at least two stages: the fp32 epilogue stages a whole 128 x 128 tile = 64 KB there) + alignment
+// slack + a tail holding the barriers (256 B) and the bias tile (512 B)
+__host__ __device__ constexpr int ring_stages(int stages) { return stages < 2 ? 2 : stages; }
+__host__ __device__ constexpr int smem_bytes(int stages) { return ring_stages(stages) * STAGE_BYTES + 1024 + 1024; }
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Epilogue {
@@ -56,7 +59,15 @@ struct Params {
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
     int debug_no_loads;                // self-test: the producer issues nothing, so the waits run out
+#ifdef COCOD_GEMM_TRACE
+    unsigned long long *trace;         // tuning builds only: 8 timestamps per CTA
+#endif
 };
+#ifdef COCOD_GEMM_TRACE
+#define COCOD_TRACE(i) do { if (p.trace && (threadIdx.x & 31) == 0) p.trace[((blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x) * 8 + (i)] = now_ns(); } while (0)
+#else
+#define COCOD_TRACE(i) do { } while (0)
+#endif
 
 // ------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -189,12 +200,15 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    if (threadIdx.x == 0) COCOD_TRACE(0);
     const int stages = p.stages;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + stages * STAGE_BYTES);
+    uint8_t *tail = smem + ring_stages(stages) * STAGE_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_STAGES), accum = smem_u32(bars + 2 * MAX_STAGES);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 1);
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
+    float *sbias = reinterpret_cast<float *>(tail + 256);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, wk = blockIdx.z;
@@ -202,7 +216,30 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     const uint32_t smem_base = smem_u32(smem);
     const unsigned long long limit = p.wait_ns ? p.wait_ns : WAIT_LIMIT_NS;
 
+    // One k-block's operand tiles into stage s (producer thread only).
+    auto issue_loads = [&](int kb, int s) {
+        const uint32_t bar = full0 + 8 * s;
+        mbar_expect_tx(bar, STAGE_BYTES);
+        const uint32_t dst_a = smem_base + s * STAGE_BYTES, dst_b = dst_a + A_BYTES;
+        if (A_MN) {
+            tma_load_3d(dst_a, &map_a, bar, m0, kb * BK, wk);
+            tma_load_3d(dst_a + BK * 128, &map_a, bar, m0 + 64, kb * BK, wk);
+        } else {
+            tma_load_3d(dst_a, &map_a, bar, kb * BK, m0, wk);
+        }
+        if (B_MN) {
+            tma_load_3d(dst_b, &map_b, bar, n0, kb * BK, wk);
+            tma_load_3d(dst_b + BK * 128, &map_b, bar, n0 + 64, kb * BK, wk);
+        } else {
+            tma_load_3d(dst_b, &map_b, bar, kb * BK, n0, wk);
+        }
+    };
+
+    int armed = 0;
     if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
+        if (EPI == EPI_F32 && p.map_c_ok) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
         for (int s = 0; s < stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
@@ -212,6 +249,9 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         abort[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
+        // the first ring of copies starts now, under the rest of the set-up
+        if (!p.debug_no_loads)
+            for (; armed < nkb && armed < stages; ++armed) issue_loads(armed, armed);
     }
     __syncwarp();
     if (warp == 0) {                  // warp-collective TMEM allocation
@@ -222,29 +262,18 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (threadIdx.x == 0) COCOD_TRACE(1);
 
     int failed = 0;
+    const int row = warp * 32 + lane;
+    const int m = m0 + row;
+    uint4 maskv[16];                  // EPI_MASK: this thread's 128 mask values, fetched while the MMAs run
     if (warp == 0 && lane == 0) {
-        // ---- producer: TMA loads of the A and B tiles of every 64-wide reduction block
-        int armed = 0;
-        for (int kb = 0; kb < nkb && !p.debug_no_loads; ++kb) {
+        // ---- producer: the remaining k-blocks, each as soon as its stage is free again
+        for (int kb = armed; kb < nkb && !p.debug_no_loads; ++kb) {
             const int s = kb % stages;
-            if (kb >= stages && !mbar_wait(empty0 + 8 * s, ((kb / stages) - 1) & 1, abort, limit)) { failed = 1; break; }
-            const uint32_t bar = full0 + 8 * s;
-            mbar_expect_tx(bar, STAGE_BYTES);
-            const uint32_t dst_a = smem_base + s * STAGE_BYTES, dst_b = dst_a + A_BYTES;
-            if (A_MN) {
-                tma_load_3d(dst_a, &map_a, bar, m0, kb * BK, wk);
-                tma_load_3d(dst_a + BK * 128, &map_a, bar, m0 + 64, kb * BK, wk);
-            } else {
-                tma_load_3d(dst_a, &map_a, bar, kb * BK, m0, wk);
-            }
-            if (B_MN) {
-                tma_load_3d(dst_b, &map_b, bar, n0, kb * BK, wk);
-                tma_load_3d(dst_b + BK * 128, &map_b, bar, n0 + 64, kb * BK, wk);
-            } else {
-                tma_load_3d(dst_b, &map_b, bar, kb * BK, n0, wk);
-            }
+            if (!mbar_wait(empty0 + 8 * s, ((kb / stages) - 1) & 1, abort, limit)) { failed = 1; break; }
+            issue_loads(kb, s);
             armed = kb + 1;
         }
         if (failed) {                 // let copies that were already issued land before leaving
@@ -259,6 +288,8 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         for (int kb = 0; kb < nkb; ++kb) {
             const int s = kb % stages;
             if (!mbar_wait(full0 + 8 * s, (kb / stages) & 1, abort, limit)) { failed = 2; break; }
+            if (kb == 0) COCOD_TRACE(2);
+            if (kb == nkb - 1) COCOD_TRACE(3);
             tc_fence_after();
             const uint32_t a_addr = smem_base + s * STAGE_BYTES, b_addr = a_addr + A_BYTES;
 #pragma unroll
@@ -271,67 +302,88 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         }
         if (!failed) umma_commit(accum);      // accumulator complete
         else abort[0] = 1;
+    } else if (warp >= 2) {
+        // ---- idle warps fetch what the epilogue needs besides the accumulator
+        if (EPI == EPI_BIAS_RELU) {
+            const __nv_bfloat16 *bias = p.bias + (long long)wk * p.bias_worker_stride;
+            for (int i = threadIdx.x - 64; i < BN; i += 64) sbias[i] = (n0 + i < p.N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
+        }
+    }
+    if (EPI == EPI_MASK) {
+        const __nv_bfloat16 *mrow = p.mask + (long long)wk * p.mask_worker_stride + (long long)m * p.N + n0;
+        const bool vec = (m < p.M) && (n0 + BN <= p.N) && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            if (vec) {
+                maskv[q] = *reinterpret_cast<const uint4 *>(mrow + q * 8);
+            } else {
+                __align__(16) __nv_bfloat16 t[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    t[e] = (m < p.M && n0 + q * 8 + e < p.N) ? mrow[q * 8 + e] : __float2bfloat16_rn(0.0f);
+                maskv[q] = *reinterpret_cast<const uint4 *>(t);
+            }
+        }
     }
     __syncwarp();
 
     // ---- epilogue: every thread owns one accumulator row (TMEM lane) of the tile
     bool ok = mbar_wait(accum, 0, abort, limit + limit / 2);
     ok = __all_sync(0xffffffffu, ok);
-    if (__syncthreads_and(ok ? 1 : 0)) {
+    if (__syncthreads_and(ok ? 1 : 0)) {          // (also makes sbias visible)
+        if (threadIdx.x == 0) COCOD_TRACE(4);
         tc_fence_after();
-        const int row = warp * 32 + lane;
-        const int m = m0 + row;
         const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-            const int nb = n0 + c0;
-            if (nb >= p.N) break;                      // uniform over the CTA
-            uint32_t r[32];
-            tmem_ld32(trow + c0, r);
-            tmem_ld_wait();
-            if (EPI == EPI_F32) {
-                if (p.map_c_ok) {
-                    // stage the 128 x 32 fp32 chunk in shared memory (all MMAs are done, so the ring is
-                    // free) with the 128-byte swizzle: 16-byte piece j of row r sits at piece j ^ (r & 7)
-                    const int buf = (c0 >> 5) & 1;
-                    if (c0 >= 64) {                    // this buffer was handed to a bulk store two chunks ago
-                        if (threadIdx.x == 0) tma_store_wait_read<1>();
-                        __syncthreads();
-                    }
-                    uint8_t *tile = smem + buf * (BM * 128);
+        uint32_t r[4][32];                         // the whole 128-column accumulator row
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(trow + c * 32, r[c]);
+        tmem_ld_wait();
+        if (EPI == EPI_F32) {
+            if (p.map_c_ok) {
+                // stage the 128 x 128 fp32 tile in the (now idle) ring as four 128 x 32 sub-tiles with the
+                // 128-byte swizzle (16-byte piece j of row r sits at piece j ^ (r & 7)), then bulk-store them
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint8_t *tile = smem + c * (BM * 128);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         *reinterpret_cast<uint4 *>(tile + row * 128 + ((j ^ (row & 7)) << 4)) =
-                            make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
-                    fence_async_smem();
-                    __syncthreads();
-                    if (threadIdx.x == 0) {
-                        tma_store_3d(&map_c, smem_u32(tile), nb, m0, wk);
-                        tma_store_commit();
-                    }
-                } else if (m < p.M) {
-                    float *dst = p.c + (long long)wk * p.c_worker_stride + (long long)m * p.ldc + nb;
+                            make_uint4(r[c][4 * j], r[c][4 * j + 1], r[c][4 * j + 2], r[c][4 * j + 3]);
+                }
+                fence_async_smem();
+                __syncthreads();
+                if (threadIdx.x == 0) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        if (n0 + c * 32 < p.N) tma_store_3d(&map_c, smem_base + c * (BM * 128), n0 + c * 32, m0, wk);
+                    tma_store_commit();
+                    tma_store_wait_read<0>();      // shared memory must outlive the reads
+                }
+            } else if (m < p.M) {
+                float *dst = p.c + (long long)wk * p.c_worker_stride + (long long)m * p.ldc + n0;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (nb + j < p.N) dst[j] = __uint_as_float(r[j]);
-                }
-            } else {
+                        if (n0 + c * 32 + j < p.N) dst[c * 32 + j] = __uint_as_float(r[c][j]);
+            }
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const int nb = n0 + c * 32;
                 __align__(16) __nv_bfloat16 outv[32];
-                const __nv_bfloat16 *bias = (EPI == EPI_BIAS_RELU) ? p.bias + (long long)wk * p.bias_worker_stride : nullptr;
-                const __nv_bfloat16 *mrow = (EPI == EPI_MASK && m < p.M)
-                                                ? p.mask + (long long)wk * p.mask_worker_stride + (long long)m * p.N : nullptr;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    float a = __uint_as_float(r[j]);
-                    const int n = nb + j;
+                    float a = __uint_as_float(r[c][j]);
                     if (EPI == EPI_BIAS_RELU) {
-                        a = (n < p.N) ? fmaxf(a + __bfloat162float(bias[n]), 0.0f) : 0.0f;
+                        a = fmaxf(a + sbias[c * 32 + j], 0.0f);
                     } else {
-                        const bool on = (mrow != nullptr) && (n < p.N) && (__bfloat162float(mrow[n]) > 0.0f);
-                        a = on ? a : 0.0f;
+                        const __nv_bfloat16 *mk = reinterpret_cast<const __nv_bfloat16 *>(&maskv[c * 4 + (j >> 3)]);
+                        a = (__bfloat162float(mk[j & 7]) > 0.0f) ? a : 0.0f;
                     }
                     outv[j] = __float2bfloat16_rn(a);
                 }
-                if (m < p.M) {
+                if (m < p.M && nb < p.N) {
                     __nv_bfloat16 *dst = p.o + (long long)wk * p.o_worker_stride + (long long)m * p.N + nb;
                     if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
                         const uint4 *src = reinterpret_cast<const uint4 *>(outv);
@@ -345,7 +397,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 }
             }
         }
-        if (EPI == EPI_F32 && p.map_c_ok && threadIdx.x == 0) tma_store_wait_read<0>();   // smem must outlive the reads
     } else if (threadIdx.x == 0 && p.error_flag != nullptr) {
         atomicExch(p.error_flag, 1);
     }
@@ -353,6 +404,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) COCOD_TRACE(5);
     if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
 }
 

@@ -105,9 +105,10 @@ cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtens
 inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK - 1) / BK)); }
 
 // ------------------------------------------------------------------------------------------ small kernels
-// Output layer forward and loss.  One CTA = 16 samples of one worker; W3 and b3 sit in shared memory;
-// each warp handles two samples: logits = h2 W3^T + b3 (fp32), row loss = -log softmax[label],
-// dz3 = bf16((softmax - onehot) / batch) kept as fp32 values in dz3[w][b][16].  grid (B / 16, K).
+// Output layer forward and loss.  One CTA = 8 samples of one worker (one per warp); W3 sits in shared
+// memory; every lane loads its slices of the h2 row up front (all loads in flight at once):
+// logits = h2 W3^T + b3 (fp32), row loss = -log softmax[label], dz3 = bf16((softmax - onehot) / batch)
+// kept as fp32 values in dz3[w][b][16].  grid (B / 8, K).
 __global__ void __launch_bounds__(256)
 head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long long P, long long oW3, long long ob3,
             const int *__restrict__ labels, float *__restrict__ dz3, float *__restrict__ rowloss, int B, int d_h,
@@ -116,58 +117,76 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
     extern __shared__ __align__(16) uint8_t head_smem[];
     bf16 *sW3 = reinterpret_cast<bf16 *>(head_smem);                 // [d_out][d_h]
     const int w = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.x * 8 + warp;
+    const bf16 *hrow = h2 + ((long long)w * B + b) * d_h;
+    constexpr int MAXV = 4;                                          // 4 x 256 columns per pass
+    uint4 hv[MAXV];
+#pragma unroll
+    for (int q = 0; q < MAXV; ++q) {
+        const int j = lane * 8 + q * 256;
+        hv[q] = (j < d_h) ? *reinterpret_cast<const uint4 *>(hrow + j) : make_uint4(0, 0, 0, 0);
+    }
     const bf16 *W3 = params + (long long)w * P + oW3;
     for (int i = threadIdx.x * 8; i < d_out * d_h; i += 256 * 8)
         *reinterpret_cast<uint4 *>(sW3 + i) = *reinterpret_cast<const uint4 *>(W3 + i);
-    __syncthreads();
     const bf16 *b3 = params + (long long)w * P + ob3;
-    for (int sidx = 0; sidx < 2; ++sidx) {
-        const int b = blockIdx.x * 16 + warp * 2 + sidx;
-        const bf16 *hrow = h2 + ((long long)w * B + b) * d_h;
-        float acc[16];
+    const float bias = (lane < d_out) ? __bfloat162float(b3[lane]) : 0.0f;
+    const int y = labels[(long long)w * B + b];
+    __syncthreads();
+    float acc[16];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) acc[c] = 0.0f;
-        for (int j = lane * 8; j < d_h; j += 256) {
-            const uint4 hv = *reinterpret_cast<const uint4 *>(hrow + j);
-            const bf16 *hp = reinterpret_cast<const bf16 *>(&hv);
-            float hf[8];
+    for (int c = 0; c < 16; ++c) acc[c] = 0.0f;
+    for (int j0 = 0; j0 < d_h; j0 += 256 * MAXV) {
+        if (j0 > 0) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) hf[q] = __bfloat162float(hp[q]);
-#pragma unroll
-            for (int c = 0; c < 16; ++c) {
-                if (c < d_out) {
-                    const uint4 wv = *reinterpret_cast<const uint4 *>(sW3 + c * d_h + j);
-                    const bf16 *wp = reinterpret_cast<const bf16 *>(&wv);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) acc[c] = fmaf(hf[q], __bfloat162float(wp[q]), acc[c]);
-                }
+            for (int q = 0; q < MAXV; ++q) {
+                const int j = j0 + lane * 8 + q * 256;
+                hv[q] = (j < d_h) ? *reinterpret_cast<const uint4 *>(hrow + j) : make_uint4(0, 0, 0, 0);
             }
         }
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
+        for (int q = 0; q < MAXV; ++q) {
+            const int j = j0 + lane * 8 + q * 256;
+            if (j < d_h) {
+                const bf16 *hp = reinterpret_cast<const bf16 *>(&hv[q]);
+                float hf[8];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
-        // lane c finishes class c
-        float z = -INFINITY;
+                for (int e = 0; e < 8; ++e) hf[e] = __bfloat162float(hp[e]);
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-            if (lane == c && c < d_out) z = acc[c] + __bfloat162float(b3[c]);
-        float zmax = z;
+                for (int c = 0; c < 16; ++c) {
+                    if (c < d_out) {
+                        const uint4 wv = *reinterpret_cast<const uint4 *>(sW3 + c * d_h + j);
+                        const bf16 *wp = reinterpret_cast<const bf16 *>(&wv);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
-        const float e = (lane < d_out) ? expf(z - zmax) : 0.0f;
-        float ssum = e;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
-        const int y = labels[(long long)w * B + b];
-        const float pc = e / ssum;
-        if (lane < 16) {
-            const float d = (lane < d_out) ? (pc - (lane == y ? 1.0f : 0.0f)) / (float)B : 0.0f;
-            dz3[((long long)w * B + b) * 16 + lane] = __bfloat162float(__float2bfloat16_rn(d));
+                        for (int e = 0; e < 8; ++e) acc[c] = fmaf(hf[e], __bfloat162float(wp[e]), acc[c]);
+                    }
+                }
+            }
         }
-        const float py = __shfl_sync(0xffffffffu, pc, y);
-        if (lane == 0) rowloss[(long long)w * B + b] = -logf(py);
     }
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+    // lane c finishes class c
+    float z = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+        if (lane == c && c < d_out) z = acc[c] + bias;
+    float zmax = z;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+    const float e = (lane < d_out) ? expf(z - zmax) : 0.0f;
+    float ssum = e;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
+    const float pc = e / ssum;
+    if (lane < 16) {
+        const float d = (lane < d_out) ? (pc - (lane == y ? 1.0f : 0.0f)) / (float)B : 0.0f;
+        dz3[((long long)w * B + b) * 16 + lane] = __bfloat162float(__float2bfloat16_rn(d));
+    }
+    const float py = __shfl_sync(0xffffffffu, pc, y);
+    if (lane == 0) rowloss[(long long)w * B + b] = -logf(py);
 }
 
 // Everything downstream of dz3 that runs on CUDA cores, for 32 hidden units j and all 128 samples:
@@ -175,18 +194,26 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
 //   dW3[c][j] = sum_b dz3[b][c] h2[b][j];
 // the CTA with blockIdx.x == 0 also writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the
 // zero padding of the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32, K).
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, const float *__restrict__ dz3,
               const float *__restrict__ rowloss, bf16 *__restrict__ dz2, float *__restrict__ grads,
               float *__restrict__ loss, long long P, long long P_raw, long long oW3, long long ob2, long long ob3,
               int B, int d_h, int d_out)
 {
+    constexpr int NW = 4;                          // warps per CTA; warp wp owns samples wp, wp + 4, ...
     __shared__ float sdz[128 * 16];
-    __shared__ float red[8][16][33];
-    __shared__ float colsum[8][33];
+    __shared__ float red[NW][16][33];
+    __shared__ float colsum[NW][33];
     const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
-    for (int i = threadIdx.x; i < B * 16; i += 256) sdz[i] = dz3[(long long)w * B * 16 + i];
     const int j = j0 + lane;
+    // first batch of this thread's h2 values: in flight while dz3 and W3 are fetched
+    float hreg[16];
+#pragma unroll
+    for (int q = 0; q < 16; ++q) {
+        const int b = wp + NW * q;
+        hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
+    }
+    for (int i = threadIdx.x; i < B * 16; i += 32 * NW) sdz[i] = dz3[(long long)w * B * 16 + i];
     float w3[16], acc3[16];
 #pragma unroll
     for (int c = 0; c < 16; ++c) {
@@ -195,46 +222,49 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
     }
     __syncthreads();
     float csum = 0.0f;
-    float hreg[16];                               // this thread's 16 samples of column j, loaded up front
+    for (int q0 = 0; q0 * NW < B; q0 += 16) {
+        if (q0 > 0) {
 #pragma unroll
-    for (int q = 0; q < 16; ++q) {
-        const int b = wp + 8 * q;
-        hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
-    }
-#pragma unroll
-    for (int q = 0; q < 16; ++q) {
-        const int b = wp + 8 * q;
-        if (b >= B) break;
-        const long long e = ((long long)w * B + b) * d_h + j;
-        const float h = hreg[q];
-        float a = 0.0f;
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-            const float d = sdz[b * 16 + c];
-            a = fmaf(d, w3[c], a);
-            acc3[c] = fmaf(d, h, acc3[c]);
+            for (int q = 0; q < 16; ++q) {
+                const int b = wp + NW * (q0 + q);
+                hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
+            }
         }
-        const bf16 v = __float2bfloat16_rn(h > 0.0f ? a : 0.0f);
-        dz2[e] = v;
-        csum += __bfloat162float(v);
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const int b = wp + NW * (q0 + q);
+            if (b < B) {
+                const float h = hreg[q];
+                float a = 0.0f;
+#pragma unroll
+                for (int c = 0; c < 16; ++c) {
+                    const float d = sdz[b * 16 + c];
+                    a = fmaf(d, w3[c], a);
+                    acc3[c] = fmaf(d, h, acc3[c]);
+                }
+                const bf16 v = __float2bfloat16_rn(h > 0.0f ? a : 0.0f);
+                dz2[((long long)w * B + b) * d_h + j] = v;
+                csum += __bfloat162float(v);
+            }
+        }
     }
 #pragma unroll
     for (int c = 0; c < 16; ++c) red[wp][c][lane] = acc3[c];
     colsum[wp][lane] = csum;
     __syncthreads();
-    for (int i = threadIdx.x; i < 16 * 32; i += 256) {
+    for (int i = threadIdx.x; i < 16 * 32; i += 32 * NW) {
         const int c = i >> 5, l = i & 31;
         if (c < d_out) {
             float s = 0.0f;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) s += red[q][c][l];
+            for (int q = 0; q < NW; ++q) s += red[q][c][l];
             grads[(long long)w * P + oW3 + (long long)c * d_h + j0 + l] = s;
         }
     }
     if (threadIdx.x < 32) {
         float s = 0.0f;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) s += colsum[q][threadIdx.x];
+        for (int q = 0; q < NW; ++q) s += colsum[q][threadIdx.x];
         grads[(long long)w * P + ob2 + j0 + threadIdx.x] = s;
     }
     if (blockIdx.x == 0) {
@@ -248,26 +278,37 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
             for (int b = 0; b < B; ++b) s += rowloss[(long long)w * B + b];
             loss[w] = s / (float)B;
         }
-        for (long long i = P_raw + threadIdx.x; i < P; i += 256) grads[(long long)w * P + i] = 0.0f;
+        for (long long i = P_raw + threadIdx.x; i < P; i += 32 * NW) grads[(long long)w * P + i] = 0.0f;
     }
 }
 
-// db1[j] = sum_b dz1[b][j]: one thread per hidden unit, samples in order.  grid (d_h / 256, K).
+// db1[j] = sum_b dz1[b][j].  One CTA = 32 hidden units; warp wp sums samples wp, wp + 8, ... (all its
+// loads in flight at once), then the 8 partial sums are added in warp order.  grid (d_h / 32, K).
 __global__ void __launch_bounds__(256)
 colsum_bf16(const bf16 *__restrict__ dz, float *__restrict__ grads, long long P, long long ob, int B, int d_h)
 {
-    const int w = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
-    if (j >= d_h) return;
+    __shared__ float part[8][33];
+    const int w = blockIdx.y, lane = threadIdx.x & 31, wp = threadIdx.x >> 5, j = blockIdx.x * 32 + lane;
     const bf16 *col = dz + (long long)w * B * d_h + j;
     float s = 0.0f;
-    for (int b0 = 0; b0 < B; b0 += 16) {          // 16 independent loads in flight, summed in sample order
+    for (int q0 = 0; q0 * 8 < B; q0 += 16) {
         float t[16];
 #pragma unroll
-        for (int q = 0; q < 16; ++q) t[q] = (b0 + q < B) ? __bfloat162float(col[(long long)(b0 + q) * d_h]) : 0.0f;
+        for (int q = 0; q < 16; ++q) {
+            const int b = wp + 8 * (q0 + q);
+            t[q] = (b < B && j < d_h) ? __bfloat162float(col[(long long)b * d_h]) : 0.0f;
+        }
 #pragma unroll
         for (int q = 0; q < 16; ++q) s += t[q];
     }
-    grads[(long long)w * P + ob + j] = s;
+    part[wp][lane] = s;
+    __syncthreads();
+    if (threadIdx.x < 32 && j < d_h) {
+        float r = 0.0f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) r += part[q][threadIdx.x];
+        grads[(long long)w * P + ob + j] = r;
+    }
 }
 
 }  // namespace
@@ -390,10 +431,10 @@ int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, 
     p.K = d_h; p.stages = stages_for(d_h); p.o = h->h2; p.bias = prm + h->ob2;
     GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, none, p, K, s)));
     // output layer, loss, dz3; then dz2, dW3, db3, db2
-    head_logits<<<dim3(B / 16, K), 256, (size_t)d_out * d_h * sizeof(bf16), s>>>(h->h2, prm, P, h->oW3, h->ob3, labels,
+    head_logits<<<dim3(B / 8, K), 256, (size_t)d_out * d_h * sizeof(bf16), s>>>(h->h2, prm, P, h->oW3, h->ob3, labels,
                                                                                 h->dz3, h->rowloss, B, d_h, d_out);
     LAUNCH_OK();
-    head_backward<<<dim3(d_h / 32, K), 256, 0, s>>>(h->h2, prm, h->dz3, h->rowloss, h->dz2, grads, loss, P, h->P_raw,
+    head_backward<<<dim3(d_h / 32, K), 128, 0, s>>>(h->h2, prm, h->dz3, h->rowloss, h->dz2, grads, loss, P, h->P_raw,
                                                     h->oW3, h->ob2, h->ob3, B, d_h, d_out);
     LAUNCH_OK();
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
@@ -403,7 +444,7 @@ int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, 
     q.o = h->dz1; q.o_worker_stride = (long long)B * d_h;
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
     GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, none, q, K, s)));
-    colsum_bf16<<<dim3((d_h + 255) / 256, K), 256, 0, s>>>(h->dz1, grads, P, h->ob1, B, d_h);
+    colsum_bf16<<<dim3((d_h + 31) / 32, K), 256, 0, s>>>(h->dz1, grads, P, h->ob1, B, d_h);
     LAUNCH_OK();
     // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
     Params r{};
