@@ -58,12 +58,12 @@ struct cocod_engine {
     float *stage[kHostSlots] = {nullptr, nullptr};
     cudaEvent_t ev_copied[kHostSlots] = {nullptr, nullptr}, ev_consumed[kHostSlots] = {nullptr, nullptr};
     bool slot_used[kHostSlots] = {false, false};
+    bool host_ready = false;            // copy stream, staging buffers and their events all exist
     // bookkeeping
     int64_t steps = 0, launches = 0;
     int cuda_error = 0;
     bool profile = false;
     std::vector<ProfileRec> prof;
-    std::vector<cudaEvent_t> ev_pool;
 };
 
 namespace {
@@ -342,8 +342,9 @@ int cocod_destroy(cocod_handle *h)
 {
     if (!h) return COCOD_OK;
     cudaStreamSynchronize(h->compute);
-    if (h->side) cudaStreamSynchronize(h->side);
+    cudaEventSynchronize(h->ev_mean);      // last work on the borrowed side stream (no-op if never recorded)
     if (h->copy) cudaStreamSynchronize(h->copy);
+    cudaGetLastError();
     const int rc = h->cuda_error ? COCOD_ERR_CUDA : COCOD_OK;
     free_all(h);
     return rc;
@@ -362,15 +363,21 @@ int cocod_local_step_host(cocod_handle *h, const float *host_grads)
 {
     if (int rc = check_live(h)) return rc;
     if (!host_grads) return COCOD_ERR_INVALID;
-    if (!h->copy) {
-        CK(h, cudaStreamCreateWithFlags(&h->copy, cudaStreamNonBlocking));
+    if (!h->host_ready) {           // first use: all or nothing, so a failed attempt can be retried
         const int64_t cap = std::min<int64_t>(kHostChunk, h->n);
-        for (int i = 0; i < kHostSlots; ++i) {
-            cudaError_t e = cudaMalloc((void **)&h->stage[i], (size_t)cap * sizeof(float));
-            if (e != cudaSuccess) { cudaGetLastError(); return COCOD_ERR_OOM; }
-            CK(h, cudaEventCreateWithFlags(&h->ev_copied[i], cudaEventDisableTiming));
-            CK(h, cudaEventCreateWithFlags(&h->ev_consumed[i], cudaEventDisableTiming));
+        cudaError_t e = h->copy ? cudaSuccess : cudaStreamCreateWithFlags(&h->copy, cudaStreamNonBlocking);
+        for (int i = 0; i < kHostSlots && e == cudaSuccess; ++i) {
+            if (!h->stage[i]) e = cudaMalloc((void **)&h->stage[i], (size_t)cap * sizeof(float));
+            if (e == cudaSuccess && !h->ev_copied[i]) e = cudaEventCreateWithFlags(&h->ev_copied[i], cudaEventDisableTiming);
+            if (e == cudaSuccess && !h->ev_consumed[i]) e = cudaEventCreateWithFlags(&h->ev_consumed[i], cudaEventDisableTiming);
         }
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            for (int i = 0; i < kHostSlots; ++i)
+                if (h->stage[i]) { cudaFree(h->stage[i]); h->stage[i] = nullptr; }
+            return e == cudaErrorMemoryAllocation ? COCOD_ERR_OOM : COCOD_ERR_CUDA;
+        }
+        h->host_ready = true;
     }
     int slot = 0;
     for (int64_t off = 0; off < h->n; off += kHostChunk, slot = (slot + 1) % kHostSlots) {
@@ -572,7 +579,7 @@ int cocod_sync(cocod_handle *h)
 {
     if (!h) return COCOD_ERR_INVALID;
     fail(h, cudaStreamSynchronize(h->compute));
-    if (h->side && h->side != h->compute) fail(h, cudaStreamSynchronize(h->side));
+    fail(h, cudaEventSynchronize(h->ev_mean));      // side-stream work (no-op if never recorded)
     if (h->copy) fail(h, cudaStreamSynchronize(h->copy));
     return h->cuda_error ? COCOD_ERR_CUDA : COCOD_OK;
 }
