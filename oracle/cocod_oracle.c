@@ -142,9 +142,22 @@ void oracle_mean_f64(int K, int64_t P, const double *snap, const double *M, doub
     }
 }
 
-/* fp32 order: uniform  -> s = snap_0; s = s + snap_i (i = 1..K-1); mean = s * (1.0f / K)
- *             weighted -> s = w_0 * snap_0; s = fma(w_i, snap_i, s); mean = s
- * with w_i = (float)(M_i / sum_j M_j) rounded once from fp64. */
+/* fp32 order of the mirror mode.  Algorithm 1 fixes no summation order for the mean, so the mirror
+ * takes the order of the device kernels: workers are taken in blocks of 8 consecutive rows; a block
+ * is summed as a balanced pairwise tree ((t0+t1)+(t2+t3))+((t4+t5)+(t6+t7)) in which absent rows are
+ * skipped (not added as zeros); block sums are accumulated in block order.  Equal batch sizes:
+ * t_i = snap_i and mean = s * (1.0f / K).  Otherwise t_i = w_i * snap_i with
+ * w_i = (float)(M_i / sum_j M_j) rounded once from fp64, and mean = s. */
+static float tree8_f32(const float *t, int cnt)
+{
+    float a[4], b[2];
+    for (int j = 0; j < 4; ++j) a[j] = (2 * j + 1 < cnt) ? t[2 * j] + t[2 * j + 1] : t[2 * j];
+    const int c1 = (cnt + 1) / 2;
+    for (int j = 0; j < 2; ++j) b[j] = (2 * j + 1 < c1) ? a[2 * j] + a[2 * j + 1] : a[2 * j];
+    const int c2 = (c1 + 1) / 2;
+    return (c2 > 1) ? b[0] + b[1] : b[0];
+}
+
 void oracle_mean_mirror(int K, int64_t P, const float *snap, const double *M, float *mean)
 {
     float w[1024];
@@ -156,16 +169,18 @@ void oracle_mean_mirror(int K, int64_t P, const float *snap, const double *M, fl
     const float invK = 1.0f / (float)K;
 #pragma omp parallel for num_threads(g_threads) schedule(static)
     for (int64_t p = 0; p < P; ++p) {
-        float s;
-        if (M) {
-            s = w[0] * snap[p];
-            for (int i = 1; i < K; ++i) s = fmaf(w[i], snap[(int64_t)i * P + p], s);
-        } else {
-            s = snap[p];
-            for (int i = 1; i < K; ++i) s = s + snap[(int64_t)i * P + p];
-            s = s * invK;
+        float s = 0.0f;
+        for (int i0 = 0; i0 < K; i0 += 8) {
+            float t[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            const int cnt = (K - i0 < 8) ? (K - i0) : 8;
+            for (int j = 0; j < cnt; ++j) {
+                const float v = snap[(int64_t)(i0 + j) * P + p];
+                t[j] = M ? w[i0 + j] * v : v;
+            }
+            const float blk = tree8_f32(t, cnt);
+            s = (i0 == 0) ? blk : s + blk;
         }
-        mean[p] = s;
+        mean[p] = M ? s : s * invK;
     }
 }
 

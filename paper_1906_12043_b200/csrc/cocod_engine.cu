@@ -149,7 +149,7 @@ cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, flo
         else mean_vec8<4><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
     } else if ((P % 4) == 0 && aligned16(snap) && aligned16(mean)) {
         const int64_t pvec = P / 4;
-        mean_vec4<8><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
+        mean_vec4<<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
             reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k);
     } else {
         mean_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);

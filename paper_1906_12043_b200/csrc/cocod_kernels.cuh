@@ -8,8 +8,11 @@
 // Arithmetic order is fixed (and mirrored by the test oracle's fp32 mode, so results can be
 // compared bit for bit):
 //   local step : d = fma(wd, x, g) ; v = fma(mu, v, d) ; x = fma(-lr, v, x)
-//   mean       : uniform  s = snap_0 ; s = s + snap_i (i = 1..K-1) ; mean = s * (1/K)
-//                weighted s = w_0 * snap_0 ; s = fma(w_i, snap_i, s)
+//   mean       : rows are taken in blocks of 8 consecutive workers; a block is summed as a balanced
+//                pairwise tree ((t0+t1)+(t2+t3))+((t4+t5)+(t6+t7)) (absent rows are skipped, not
+//                added as zeros), block sums are accumulated in block order; t_i = snap_i and
+//                mean = s * (1/K) for equal weights, t_i = w_i * snap_i and mean = s otherwise.
+//                (Rounding error grows with log2(8) + K/8 additions instead of K.)
 //   merge      : x = mean + (x - snap)
 #pragma once
 #include <cuda_bf16.h>
@@ -164,9 +167,72 @@ snapshot_scalar(const float *__restrict__ x, float *__restrict__ snap, int64_t f
 }
 
 // ------------------------------------------------------------------------------------------ average model (Step I)
-// One thread owns one float4 of columns and walks the K rows in order, RC row loads in flight
-// at a time (RC * 16 B per thread).  Needs P mod 4 == 0 and 16-byte aligned bases.
-template <int RC>
+// Balanced pairwise sum of the first cnt (1..8) entries of t[], skipping absent entries.
+__device__ __forceinline__ float tree8(const float (&t)[8], int cnt)
+{
+    float a[4], b[2];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) a[j] = (2 * j + 1 < cnt) ? __fadd_rn(t[2 * j], t[2 * j + 1]) : t[2 * j];
+    const int c1 = (cnt + 1) >> 1;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) b[j] = (2 * j + 1 < c1) ? __fadd_rn(a[2 * j], a[2 * j + 1]) : a[2 * j];
+    const int c2 = (c1 + 1) >> 1;
+    return (c2 > 1) ? __fadd_rn(b[0], b[1]) : b[0];
+}
+__device__ __forceinline__ float tree8_full(const float (&t)[8])
+{
+    return __fadd_rn(__fadd_rn(__fadd_rn(t[0], t[1]), __fadd_rn(t[2], t[3])),
+                     __fadd_rn(__fadd_rn(t[4], t[5]), __fadd_rn(t[6], t[7])));
+}
+
+// Sum over the K rows of the NV columns held by one thread.  Rows are taken in blocks of 8 (all loads
+// of a block in flight together); full blocks run without predicates, the last partial block with.
+// CAP < 8 is for few workers (K <= CAP): a single partial block with only CAP loads per thread.
+// load(i, v) fills v[0..NV) with the thread's values of row i.
+template <int NV, int CAP, typename Load>
+__device__ __forceinline__ void mean_rows(float (&s)[NV], int K, const float *__restrict__ w, float inv_k, Load load)
+{
+    int i0 = 0;
+    if (CAP == 8) {
+        for (; i0 + 8 <= K; i0 += 8) {
+            float r[8][NV];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) load(i0 + j, r[j]);
+#pragma unroll
+            for (int q = 0; q < NV; ++q) {
+                float t[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) t[j] = (w != nullptr) ? __fmul_rn(__ldg(w + i0 + j), r[j][q]) : r[j][q];
+                const float blk = tree8_full(t);
+                s[q] = (i0 == 0) ? blk : __fadd_rn(s[q], blk);
+            }
+        }
+    }
+    if (i0 < K) {
+        const int cnt = K - i0;                    // 1 .. CAP (CAP == 8: at most 7)
+        float r[CAP][NV];
+#pragma unroll
+        for (int j = 0; j < CAP; ++j)
+            if (j < cnt) load(i0 + j, r[j]);
+#pragma unroll
+        for (int q = 0; q < NV; ++q) {
+            float t[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                t[j] = 0.0f;
+                if (j < CAP && j < cnt) t[j] = (w != nullptr) ? __fmul_rn(__ldg(w + i0 + j), r[j < CAP ? j : 0][q]) : r[j < CAP ? j : 0][q];
+            }
+            const float blk = tree8(t, cnt);
+            s[q] = (i0 == 0) ? blk : __fadd_rn(s[q], blk);
+        }
+    }
+    if (w == nullptr) {
+#pragma unroll
+        for (int q = 0; q < NV; ++q) s[q] = __fmul_rn(s[q], inv_k);
+    }
+}
+
+// One thread owns one float4 of columns.  Needs P mod 4 == 0 and 16-byte aligned bases.
 __global__ void __launch_bounds__(kThreads)
 mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__restrict__ w,
           float4 *__restrict__ mean, float inv_k)
@@ -174,97 +240,45 @@ mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__r
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (c >= pvec) return;
     const float4 *col = snap + c;
-    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i0 = 0; i0 < K; i0 += RC) {
-        float4 r[RC];
-#pragma unroll
-        for (int j = 0; j < RC; ++j)
-            if (i0 + j < K) r[j] = ld_stream(col + (int64_t)(i0 + j) * pvec);
-#pragma unroll
-        for (int j = 0; j < RC; ++j) {
-            const int i = i0 + j;
-            if (i < K) {
-                if (w != nullptr) {
-                    const float wi = __ldg(w + i);
-                    if (i == 0) {
-                        s.x = __fmul_rn(wi, r[j].x); s.y = __fmul_rn(wi, r[j].y);
-                        s.z = __fmul_rn(wi, r[j].z); s.w = __fmul_rn(wi, r[j].w);
-                    } else {
-                        s.x = __fmaf_rn(wi, r[j].x, s.x); s.y = __fmaf_rn(wi, r[j].y, s.y);
-                        s.z = __fmaf_rn(wi, r[j].z, s.z); s.w = __fmaf_rn(wi, r[j].w, s.w);
-                    }
-                } else {
-                    if (i == 0) s = r[j];
-                    else {
-                        s.x = __fadd_rn(s.x, r[j].x); s.y = __fadd_rn(s.y, r[j].y);
-                        s.z = __fadd_rn(s.z, r[j].z); s.w = __fadd_rn(s.w, r[j].w);
-                    }
-                }
-            }
-        }
-    }
-    if (w == nullptr) {
-        s.x = __fmul_rn(s.x, inv_k); s.y = __fmul_rn(s.y, inv_k);
-        s.z = __fmul_rn(s.z, inv_k); s.w = __fmul_rn(s.w, inv_k);
-    }
-    mean[c] = s;
+    float s[4];
+    mean_rows<4, 8>(s, K, w, inv_k, [&](int i, float (&v)[4]) {
+        const float4 t = ld_stream(col + (int64_t)i * pvec);
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    });
+    mean[c] = make_float4(s[0], s[1], s[2], s[3]);
 }
 
-// Few workers (K <= 4): a float4 per row would leave too few bytes in flight per thread, so
-// one thread owns 8 columns (256-bit loads).  Same row order.  P mod 8 == 0, 32-byte aligned.
-template <int RC>
+// Few workers (K <= CAP <= 4): a float4 per row would leave too few bytes in flight per thread, so
+// one thread owns 8 columns (256-bit loads).  P mod 8 == 0, 32-byte aligned bases.
+template <int CAP>
 __global__ void __launch_bounds__(kThreads)
 mean_vec8(const float *__restrict__ snap, int K, int64_t P, const float *__restrict__ w,
           float *__restrict__ mean, float inv_k)
 {
     const int64_t c = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 8;
     if (c >= P) return;
-    f32x8 s;
-    for (int i0 = 0; i0 < K; i0 += RC) {
-        f32x8 r[RC];
+    float s[8];
+    mean_rows<8, CAP>(s, K, w, inv_k, [&](int i, float (&v)[8]) {
+        const f32x8 t = ld256_stream(snap + (int64_t)i * P + c);
 #pragma unroll
-        for (int j = 0; j < RC; ++j)
-            if (i0 + j < K) r[j] = ld256_stream(snap + (int64_t)(i0 + j) * P + c);
+        for (int q = 0; q < 8; ++q) v[q] = t.a[q];
+    });
+    f32x8 o;
 #pragma unroll
-        for (int j = 0; j < RC; ++j) {
-            const int i = i0 + j;
-            if (i < K) {
-                if (w != nullptr) {
-                    const float wi = __ldg(w + i);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        s.a[q] = (i == 0) ? __fmul_rn(wi, r[j].a[q]) : __fmaf_rn(wi, r[j].a[q], s.a[q]);
-                } else {
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) s.a[q] = (i == 0) ? r[j].a[q] : __fadd_rn(s.a[q], r[j].a[q]);
-                }
-            }
-        }
-    }
-    if (w == nullptr) {
-#pragma unroll
-        for (int q = 0; q < 8; ++q) s.a[q] = __fmul_rn(s.a[q], inv_k);
-    }
-    st256(mean + c, s);
+    for (int q = 0; q < 8; ++q) o.a[q] = s[q];
+    st256(mean + c, o);
 }
 
-// Any P / alignment: one thread per column, same row order.
+// Any P / alignment: one thread per column.
 __global__ void __launch_bounds__(kThreads)
 mean_scalar(const float *__restrict__ snap, int K, int64_t P, const float *__restrict__ w,
             float *__restrict__ mean, float inv_k)
 {
     const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (p >= P) return;
-    float s;
-    if (w != nullptr) {
-        s = __fmul_rn(__ldg(w), snap[p]);
-        for (int i = 1; i < K; ++i) s = __fmaf_rn(__ldg(w + i), snap[(int64_t)i * P + p], s);
-    } else {
-        s = snap[p];
-        for (int i = 1; i < K; ++i) s = __fadd_rn(s, snap[(int64_t)i * P + p]);
-        s = __fmul_rn(s, inv_k);
-    }
-    mean[p] = s;
+    float s[1];
+    mean_rows<1, 8>(s, K, w, inv_k, [&](int i, float (&v)[1]) { v[0] = snap[(int64_t)i * P + p]; });
+    mean[p] = s[0];
 }
 
 // ------------------------------------------------------------------------------------------ merge (line 6)

@@ -114,3 +114,13 @@ def test_vgg16_sized_sampled_columns_cross_the_2_31_flat_index(E):
     if free < 80e9:
         pytest.skip("not enough free HBM for the VGG16-sized state")
     run_fullsize(E, wl, rounds=5, n_random=2048)
+
+
+@pytest.mark.parametrize("K,logP,k", [(2, 24, 1), (8, 20, 8), (64, 20, 1), (32, 22, 8), (5, 21, 2)])
+def test_scaling_sweep_cells_sampled_columns(E, K, logP, k):
+    """Cells of the scaling sweep (P = 2^logP, K workers, k local steps per round, momentum 0.9):
+    sampled columns against the oracle plus the mean-preservation invariant, in the same launch
+    configuration the sweep times.  (K = 5 is not in the sweep: it exercises an odd worker count.)"""
+    from paper_1906_12043_b200.workloads import Workload
+    wl = Workload(f"sweep-K{K}-P2^{logP}-k{k}", K=K, P=1 << logP, k=k, rounds=3, lr=0.1, mu=0.9, wd=5e-4)
+    run_fullsize(E, wl, wl.rounds, n_random=1024)
