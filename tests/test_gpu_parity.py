@@ -403,6 +403,71 @@ def test_rounds_replayed_from_a_cuda_graph_match_eager_rounds(E):
         assert_bit_equal(cpu(graphed.get_momentum()), cpu(eager.get_momentum()), f"v after block {block}")
 
 
+@pytest.mark.parametrize("K,P,snapshot", [(3, 1001, 1), (4, 4100, 0), (2, 8 * 1000, 1), (16, 65_536 + 64, 1)])
+def test_bf16_shadow_tracks_the_master_copy_on_every_path(E, K, P, snapshot):
+    """With the bf16 shadow on, every kernel that writes x (local step, merge; vector and scalar
+    paths, both snapshot modes) also writes bf16(x): after each call the shadow equals the master
+    copy rounded to nearest even, and the fp32 results are unchanged by the option."""
+    rng = np.random.default_rng(P)
+    x0 = (rng.standard_normal(P) * 0.05).astype(np.float32)
+    eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
+    eng.set_option(E.OPT_SNAPSHOT, snapshot)
+    eng.set_option(E.OPT_BF16_SHADOW, 1)
+    eng.set_params(x0)
+    mir = OracleEngine(K, P, 0.1, 0.9, 5e-4, mode="mirror")
+    mir.set_params(x0)
+    side = torch.cuda.Stream()
+
+    def check(tag):
+        x = cpu(eng.get_params())
+        assert_bit_equal(x, mir.x, f"x {tag}")
+        assert_bit_equal(cpu(eng.bf16_shadow().float()), I.round_to_bf16(x), f"shadow {tag}")
+
+    check("after set_params")
+    for r in range(2):
+        eng.comm_begin(side)
+        mir.comm_begin()
+        for s in range(2):
+            g = (rng.standard_normal((K, P)) * 0.01).astype(np.float32)
+            eng.local_step(torch.from_numpy(g).cuda())
+            mir.local_step(g)
+            check(f"after step {r}.{s}")
+        eng.comm_end()
+        mir.comm_end()
+        check(f"after merge {r}")
+    X = (rng.standard_normal((K, P)) * 0.05).astype(np.float32)
+    eng.set_params_all(X)
+    mir.set_params_all(X)
+    check("after set_params_all")
+    eng.set_option(E.OPT_BF16_SHADOW, 0)
+    with pytest.raises(E.CocodError):
+        eng.bf16_shadow()
+
+
+def test_switching_the_compute_stream_keeps_work_ordered(E):
+    K, P = 4, 200_000
+    x0 = I.initial_point(P)
+    a, b = torch.cuda.Stream(), torch.cuda.Stream()
+    eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
+    mir = OracleEngine(K, P, 0.1, 0.9, 5e-4, mode="mirror")
+    eng.set_params(x0)
+    mir.set_params(x0)
+    side = torch.cuda.Stream()
+    gs = [torch.from_numpy(I.gradients(K, P, t)).cuda() for t in range(6)]
+    torch.cuda.synchronize()
+    for r, stream in enumerate([a, b, a]):
+        eng.set_stream(stream)                       # later work must wait for what the old stream still runs
+        eng.comm_begin(side)
+        mir.comm_begin()
+        for s in range(2):
+            eng.local_step(gs[2 * r + s])
+            mir.local_step(cpu(gs[2 * r + s]))
+        eng.comm_end()
+        mir.comm_end()
+    eng.sync()
+    assert_bit_equal(cpu(eng.get_params()), mir.x)
+
+
 def test_learning_rate_schedule_and_profile_records(E):
     K, P = 2, 4096
     eng = E.Engine(K, P, 0.1, 0.9, 0.0)
