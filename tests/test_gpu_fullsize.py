@@ -113,7 +113,7 @@ def test_vgg16_sized_sampled_columns_cross_the_2_31_flat_index(E):
     free, _ = torch.cuda.mem_get_info()
     if free < 80e9:
         pytest.skip("not enough free HBM for the VGG16-sized state")
-    run_fullsize(E, wl, rounds=5, n_random=2048)
+    run_fullsize(E, wl, wl.rounds, n_random=2048)          # the full 20 rounds of k = 4
 
 
 @pytest.mark.parametrize("K,logP,k", [(2, 24, 1), (8, 20, 8), (64, 20, 1), (32, 22, 8), (5, 21, 2)])
