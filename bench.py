@@ -63,10 +63,16 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.proc = None
+        ident = str(index)
+        try:        # nvidia-smi numbers GPUs physically; under CUDA_VISIBLE_DEVICES only the UUID is safe
+            import torch
+            ident = "GPU-" + str(torch.cuda.get_device_properties(index).uuid)
+        except Exception:
+            pass
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-i", str(index), "-lms", "100"],
+                 "-i", ident, "-lms", "100"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
