@@ -173,6 +173,63 @@ def test_shapes_spanning_tiles_and_ragged_tails(E, K, P, snapshot):
     assert_close_scaled(v, ref.v, 1e-5, "v vs ref")
 
 
+@pytest.mark.parametrize("seed", range(24))
+def test_random_configurations_match_the_mirror_bit_for_bit(E, seed):
+    """Randomised sweep over worker counts, sizes (aligned, ragged, tiny), periods, hyper-parameters,
+    batch-size weights, snapshot modes, side-stream choices and the bf16 shadow: the fp32 mirror must
+    be reproduced bit for bit and the reference within 1e-5."""
+    rng = np.random.default_rng(1000 + seed)
+    K = int(rng.choice([1, 2, 3, 4, 5, 7, 8, 9, 16, 17, 31, 40]))
+    P = int(rng.choice([1, 2, 5, 8, 12, 64, 100, 1000, 1024, 4096, 4100, 10_007, 65_536, 100_003]))
+    k, rounds = int(rng.integers(1, 5)), int(rng.integers(1, 4))
+    lr = float(rng.choice([0.01, 0.05, 0.1, 0.5]))
+    mu = float(rng.choice([0.0, 0.5, 0.9, 0.99]))
+    wd = float(rng.choice([0.0, 1e-4, 5e-4, 1e-2]))
+    M = rng.integers(1, 65, K).astype(float) if rng.random() < 0.5 else None
+    snapshot = int(rng.integers(0, 2))
+    side = str(rng.choice(["own", "same", "high"]))
+    shadow = bool(rng.random() < 0.3)
+    x0 = (rng.standard_normal(P) * 0.05).astype(np.float32)
+    G = (rng.standard_normal((k * rounds, K, P)) * 0.02).astype(np.float32)
+
+    eng = E.Engine(K, P, lr, mu, wd)
+    eng.set_option(E.OPT_SNAPSHOT, snapshot)
+    if shadow:
+        eng.set_option(E.OPT_BF16_SHADOW, 1)
+    if M is not None:
+        eng.set_batch_sizes(M)
+    eng.set_params(x0)
+    ref = OracleEngine(K, P, lr, mu, wd, mode="ref", batch_sizes=M)
+    mir = OracleEngine(K, P, lr, mu, wd, mode="mirror", batch_sizes=M)
+    ref.set_params(x0)
+    mir.set_params(x0)
+    side_stream = {"own": torch.cuda.Stream(), "same": torch.cuda.current_stream(),
+                   "high": torch.cuda.Stream(priority=-1)}[side]
+    keep = []
+    for r in range(rounds):
+        for o in (ref, mir):
+            o.comm_begin()
+        eng.comm_begin(side_stream)
+        for s in range(k):
+            g = G[r * k + s]
+            keep.append(torch.from_numpy(g).cuda())
+            eng.local_step(keep[-1])
+            ref.local_step(g)
+            mir.local_step(g)
+        eng.comm_end()
+        for o in (ref, mir):
+            o.comm_end()
+    what = f"K={K} P={P} k={k} rounds={rounds} lr={lr} mu={mu} wd={wd} weighted={M is not None} snapshot={snapshot} side={side} shadow={shadow}"
+    x, v = cpu(eng.get_params()), cpu(eng.get_momentum())
+    assert_bit_equal(x, mir.x, "x vs mirror: " + what)
+    assert_bit_equal(v, mir.v, "v vs mirror: " + what)
+    assert_bit_equal(cpu(eng.get_mean()), mir.mean, "mean vs mirror: " + what)
+    assert_close_scaled(x, ref.x, 1e-5, "x vs ref: " + what)
+    assert_close_scaled(v, ref.v, 1e-5, "v vs ref: " + what)
+    if shadow:
+        assert_bit_equal(cpu(eng.bf16_shadow().float()), I.round_to_bf16(x), "shadow: " + what)
+
+
 @pytest.mark.parametrize("side", ["own", "same", "high"])
 @pytest.mark.parametrize("weighted", [False, True])
 def test_side_stream_choices_and_weighted_mean(E, side, weighted):
