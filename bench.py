@@ -43,6 +43,8 @@ def parse():
     ap.add_argument("--ring", type=int, default=4, help="distinct gradient buffers cycled through")
     ap.add_argument("--graph", action="store_true",
                     help="replay the timed rounds from a CUDA graph of two rounds (launch-bound workloads)")
+    ap.add_argument("--fused", action="store_true",
+                    help="mlp workload: gradients and local step in one call (update inside the weight-gradient GEMMs)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-cols", type=int, default=1 << 20)
@@ -445,8 +447,11 @@ def run_mlp(args):
         eng.comm_begin(side)
         for _ in range(k):
             i = step_no[0] % ring_n
-            mg.grad(shadow, xs_d[i], ys_d[i], grads, loss)
-            eng.local_step(grads)
+            if args.fused:
+                mg.grad_step(eng, xs_d[i], ys_d[i], loss)
+            else:
+                mg.grad(shadow, xs_d[i], ys_d[i], grads, loss)
+                eng.local_step(grads)
             step_no[0] += 1
             if record:
                 losses.append(loss.clone())
@@ -506,8 +511,11 @@ def run_mlp(args):
             i = step_no[0] % ring_n
             x_dev.copy_(xs_h[i], non_blocking=True)
             y_dev.copy_(ys_h[i], non_blocking=True)
-            mg.grad(shadow, x_dev, y_dev, grads, loss)
-            eng.local_step(grads)
+            if args.fused:
+                mg.grad_step(eng, x_dev, y_dev, loss)
+            else:
+                mg.grad(shadow, x_dev, y_dev, grads, loss)
+                eng.local_step(grads)
             loss_h.copy_(loss, non_blocking=True)
             step_no[0] += 1
         eng.comm_end()
@@ -533,7 +541,8 @@ def run_mlp(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 contractions / f32 state",
         "data": "synthetic",
         "config": {"workload": "mlp", "K": K, "P": P_raw, "P_padded": P, "k": k, "lr": lr, "mu": mu, "wd": wd,
-                   "mlp": list(dims), "batch": B, "minibatch_ring": ring_n, "cuda_graph": bool(args.graph)},
+                   "mlp": list(dims), "batch": B, "minibatch_ring": ring_n, "cuda_graph": bool(args.graph),
+                   "fused_update": bool(args.fused)},
         "clocks": clocks, "gpu_launches": launches,
         "local_steps_per_s": k * args.steps / (ms * 1e-3), "ms_per_local_step": ms / (k * args.steps),
         "tensor_tflops": flops_step * k * args.steps / (ms * 1e-3) / 1e12,

@@ -58,6 +58,19 @@ int64_t cocod_mlp_param_count_unpadded(const cocod_mlp_handle *h);
 int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, const int32_t *labels,
                    float *grads, float *loss, cocod_stream_t stream);
 
+/* The same gradient pass fused with the engine's local step (Algorithm 1, Step II: gradient and
+ * update of one iteration in one call).  `engine` must have been created with
+ * K = the handle's K and P = cocod_mlp_param_count, with COCOD_OPT_BF16_SHADOW on (STATE otherwise):
+ * the gradients are computed from its bf16 copy of x.  For the two weight matrices W1 and W2
+ * (99.4 % of the parameters) the weight-gradient GEMMs apply the update d = g + wd x; v = mu v + d;
+ * x = x - lr v in their epilogue: the gradient tile never leaves the SM, x, v and the bf16 copy are
+ * read and written once.  The remaining tensors go through a small gradient buffer owned by the
+ * handle and the engine's ordinary update.  Results are bit-identical to cocod_mlp_grad followed by
+ * cocod_local_step.  Runs on the engine's compute stream; counts as one local step.
+ *   x, labels, loss: as for cocod_mlp_grad. */
+int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x, const int32_t *labels,
+                        float *loss);
+
 /* Synchronise `stream` and report whether any kernel of this handle gave up a wait. */
 int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream);
 

@@ -9,6 +9,7 @@
 // Ordering is by stream events only; no kernel spins on another and the host never blocks
 // inside a round.
 #include "cocod.h"
+#include "cocod_internal.h"
 #include "cocod_kernels.cuh"
 
 #include <algorithm>
@@ -50,6 +51,7 @@ struct cocod_engine {
     const float *snap = nullptr;       // where this round's stored copies live
     bool pending_flip = false;          // FLIP mode: x still lives in the stored-copy buffer
     bool mean_valid = false;
+    bool mean_captured = false;         // the last averaging was recorded into a CUDA graph, not executed
     int state = IDLE;
     int snapshot_mode = COCOD_SNAPSHOT_FLIP;
     cudaStream_t compute = nullptr, side = nullptr, copy = nullptr;
@@ -342,7 +344,7 @@ int cocod_destroy(cocod_handle *h)
 {
     if (!h) return COCOD_OK;
     cudaStreamSynchronize(h->compute);
-    cudaEventSynchronize(h->ev_mean);      // last work on the borrowed side stream (no-op if never recorded)
+    if (!h->mean_captured) cudaEventSynchronize(h->ev_mean);      // last work on the borrowed side stream
     if (h->copy) cudaStreamSynchronize(h->copy);
     cudaGetLastError();
     const int rc = h->cuda_error ? COCOD_ERR_CUDA : COCOD_OK;
@@ -425,6 +427,9 @@ int cocod_comm_begin(cocod_handle *h, cocod_stream_t side)
     }
     h->launches += nl;
     CK(h, cudaEventRecord(h->ev_mean, h->side));
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CK(h, cudaStreamIsCapturing(h->side, &cap));
+    h->mean_captured = (cap != cudaStreamCaptureStatusNone);      // a captured event cannot be waited on later
     h->mean_valid = true;
     h->state = IN_FLIGHT;
     return COCOD_OK;
@@ -579,7 +584,7 @@ int cocod_sync(cocod_handle *h)
 {
     if (!h) return COCOD_ERR_INVALID;
     fail(h, cudaStreamSynchronize(h->compute));
-    fail(h, cudaEventSynchronize(h->ev_mean));      // side-stream work (no-op if never recorded)
+    if (!h->mean_captured) fail(h, cudaEventSynchronize(h->ev_mean));      // side-stream work (no-op if never recorded)
     if (h->copy) fail(h, cudaStreamSynchronize(h->copy));
     return h->cuda_error ? COCOD_ERR_CUDA : COCOD_OK;
 }
@@ -685,6 +690,51 @@ int cocod_kernel_merge(float *x, const float *snap, const float *mean, int K, in
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ internal interface (cocod_internal.h)
+int cocod_internal_plan_step(cocod_handle *h, cocod_step_plan *plan)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!plan) return COCOD_ERR_INVALID;
+    plan->x_in = h->buf[h->cur];
+    plan->x_out = h->pending_flip ? h->buf[1 - h->cur] : h->buf[h->cur];
+    plan->v = h->v;
+    plan->shadow = h->shadow;
+    plan->lr = h->lr; plan->mu = h->mu; plan->wd = h->wd;
+    plan->K = h->K; plan->P = h->P;
+    plan->compute = h->compute;
+    return COCOD_OK;
+}
+
+int cocod_internal_step_segments(cocod_handle *h, const float *g, const int64_t *lo, const int64_t *hi, int nseg)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!g || !lo || !hi || nseg < 1 || nseg > 4) return COCOD_ERR_INVALID;
+    cocod::StepSegments seg{};
+    int64_t longest = 0;
+    for (int i = 0; i < nseg; ++i) {
+        if (lo[i] < 0 || hi[i] < lo[i] || hi[i] > h->P) return COCOD_ERR_INVALID;
+        seg.lo[i] = lo[i]; seg.hi[i] = hi[i];
+        longest = std::max(longest, hi[i] - lo[i]);
+    }
+    if (longest == 0) return COCOD_OK;
+    const float *x_in = h->buf[h->cur];
+    float *x_out = h->pending_flip ? h->buf[1 - h->cur] : h->buf[h->cur];
+    const unsigned gx = (unsigned)std::min<int64_t>((longest + cocod::kThreads - 1) / cocod::kThreads, 64);
+    cocod::local_step_segments<<<dim3(gx, (unsigned)nseg, (unsigned)h->K), cocod::kThreads, 0, h->compute>>>(
+        x_in, x_out, h->v, g, h->P, seg, h->lr, h->mu, h->wd, h->shadow);
+    CK(h, cudaGetLastError());
+    ++h->launches;
+    return COCOD_OK;
+}
+
+int cocod_internal_finish_step(cocod_handle *h, int kernels_launched)
+{
+    if (int rc = check_live(h)) return rc;
+    h->launches += kernels_launched;
+    finish_step(h);
+    return COCOD_OK;
+}
 
 // ------------------------------------------------------------------ allocation-free host-gradient step
 // Staging for cocod_kernel_local_step_host_noalloc.  In host code the name below is only a

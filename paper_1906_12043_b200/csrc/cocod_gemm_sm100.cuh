@@ -11,8 +11,11 @@
 //   * one elected thread issues tcgen05.mma (kind::f16, bf16 inputs, fp32 accumulation) on
 //     shared-memory descriptors; the 128 x 128 fp32 accumulator lives in TMEM (128 columns);
 //   * all four warps read the accumulator back with tcgen05.ld (32 lanes x 32 columns at a time)
-//     and run a fused epilogue: bias + ReLU or ReLU-mask with packed bf16 stores, or an fp32 store
-//     that goes through swizzled shared memory and TMA bulk stores (full 128-byte lines).
+//     and run a fused epilogue: bias + ReLU or ReLU-mask with packed bf16 stores, an fp32 store
+//     that goes through swizzled shared memory and TMA bulk stores (full 128-byte lines), or -- for
+//     weight gradients -- the momentum-SGD update itself: the matching x and v tiles are fetched by
+//     TMA while the MMAs run, updated in shared memory with the accumulator as the gradient, and
+//     stored back together with the bf16 copy of x, so the gradient never touches HBM.
 // Out-of-range rows / reduction columns are zero-filled by TMA, so M, N, K need not be
 // multiples of the tile; stores are predicated.
 //
@@ -23,6 +26,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+#include "cocod_kernels.cuh"
 
 namespace cocod {
 namespace gemm {
@@ -35,12 +40,21 @@ constexpr int MAX_STAGES = STAGES;
 // slack + a tail holding the barriers (256 B) and the bias tile (512 B)
 __host__ __device__ constexpr int ring_stages(int stages) { return stages < 2 ? 2 : stages; }
 __host__ __device__ constexpr int smem_bytes(int stages) { return ring_stages(stages) * STAGE_BYTES + 1024 + 1024; }
+// the update epilogue additionally keeps the x and v tiles (128 x 128 fp32 each)
+__host__ __device__ constexpr int smem_bytes_sgd(int stages) { return smem_bytes(stages) + 2 * BM * BN * 4; }
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Epilogue {
     EPI_F32 = 0,        // c[m][n] = acc                         (fp32, row stride ldc; TMA store if map_c_ok)
     EPI_BIAS_RELU = 1,  // o[m][n] = bf16(max(acc + bias[n], 0))
-    EPI_MASK = 2        // o[m][n] = bf16(acc * (mask[m][n] > 0))
+    EPI_MASK = 2,       // o[m][n] = bf16(acc * (mask[m][n] > 0))
+    EPI_SGD = 3         // g = acc: d = fma(wd, x, g); v = fma(mu, v, d); x = fma(-lr, v, x); shadow = bf16(x)
+};
+
+// Tensor maps of the update epilogue: fp32 [M][N] tiles of 32 columns x 128 rows (x read, x written,
+// v) and the bf16 copy of x in tiles of 64 columns x 128 rows; all with the 128-byte swizzle.
+struct SgdMaps {
+    CUtensorMap x_in, x_out, v, shadow;
 };
 
 struct Params {
@@ -55,6 +69,8 @@ struct Params {
     long long bias_worker_stride;
     const __nv_bfloat16 *mask;         // [M][N], row stride N
     long long mask_worker_stride;
+    float lr, mu, wd;                  // EPI_SGD
+    int has_shadow;                    // EPI_SGD: also write bf16(x)
     int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
@@ -193,19 +209,24 @@ __host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn)
 // Tensor maps: a K-major operand is {k (contiguous), rows, workers} with box {64, 128, 1}; an
 // MN-major operand is {m or n (contiguous), k, workers} with box {64, 64, 1} (two boxes per tile).
 // map_c (EPI_F32 only): {n (contiguous), m, workers} fp32 with box {32, 128, 1}, 128-byte swizzle.
-template <int EPI, bool A_MN, bool B_MN>
-__global__ void __launch_bounds__(128)
+// NT threads per CTA: 128 (every thread drains one accumulator row) or 256 (two threads share a row, each
+// draining 64 columns: used where the epilogue is long and only one CTA fits per SM).
+template <int EPI, bool A_MN, bool B_MN, int NT>
+__global__ void __launch_bounds__(NT)
 gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-          const __grid_constant__ CUtensorMap map_c, const Params p)
+          const __grid_constant__ CUtensorMap map_c, const __grid_constant__ SgdMaps sgd, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     if (threadIdx.x == 0) COCOD_TRACE(0);
     const int stages = p.stages;
-    uint8_t *tail = smem + ring_stages(stages) * STAGE_BYTES;
+    uint8_t *xs = smem + ring_stages(stages) * STAGE_BYTES;        // EPI_SGD: x tile, then v tile
+    uint8_t *vs = xs + BM * BN * 4;
+    uint8_t *tail = (EPI == EPI_SGD) ? vs + BM * BN * 4 : xs;
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_STAGES), accum = smem_u32(bars + 2 * MAX_STAGES);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 1);
+    const uint32_t aux = smem_u32(bars + 2 * MAX_STAGES + 1);      // EPI_SGD: x and v tiles have landed
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 2);
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
     float *sbias = reinterpret_cast<float *>(tail + 256);
@@ -245,6 +266,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum, 1);
+        mbar_init(aux, 1);
         abort[0] = 0;
         abort[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -252,6 +274,15 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // the first ring of copies starts now, under the rest of the set-up
         if (!p.debug_no_loads)
             for (; armed < nkb && armed < stages; ++armed) issue_loads(armed, armed);
+        if (EPI == EPI_SGD) {         // the tiles the update needs: in flight under the whole main loop
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&sgd.x_out) : "memory");
+            mbar_expect_tx(aux, 2 * BM * BN * 4);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                tma_load_3d(smem_u32(xs) + c * (BM * 128), &sgd.x_in, aux, n0 + c * 32, m0, wk);
+                tma_load_3d(smem_u32(vs) + c * (BM * 128), &sgd.v, aux, n0 + c * 32, m0, wk);
+            }
+        }
     }
     __syncwarp();
     if (warp == 0) {                  // warp-collective TMEM allocation
@@ -265,9 +296,11 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     if (threadIdx.x == 0) COCOD_TRACE(1);
 
     int failed = 0;
-    const int row = warp * 32 + lane;
+    constexpr int NCH = (NT == 256) ? 2 : 4;       // 32-column chunks drained by one thread
+    const int row = (warp & 3) * 32 + lane;        // accumulator row = TMEM lane (a warp reaches lanes 32 (w % 4) ..)
+    const int cbase = (warp >> 2) * NCH;           // first chunk of this thread
     const int m = m0 + row;
-    uint4 maskv[16];                  // EPI_MASK: this thread's 128 mask values, fetched while the MMAs run
+    uint4 maskv[NCH * 4];             // EPI_MASK: this thread's mask values, fetched while the MMAs run
     if (warp == 0 && lane == 0) {
         // ---- producer: the remaining k-blocks, each as soon as its stage is free again
         for (int kb = armed; kb < nkb && !p.debug_no_loads; ++kb) {
@@ -306,21 +339,22 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // ---- idle warps fetch what the epilogue needs besides the accumulator
         if (EPI == EPI_BIAS_RELU) {
             const __nv_bfloat16 *bias = p.bias + (long long)wk * p.bias_worker_stride;
-            for (int i = threadIdx.x - 64; i < BN; i += 64) sbias[i] = (n0 + i < p.N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
+            for (int i = threadIdx.x - 64; i < BN; i += NT - 64) sbias[i] = (n0 + i < p.N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
         }
     }
     if (EPI == EPI_MASK) {
-        const __nv_bfloat16 *mrow = p.mask + (long long)wk * p.mask_worker_stride + (long long)m * p.N + n0;
-        const bool vec = (m < p.M) && (n0 + BN <= p.N) && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0);
+        const int nm = n0 + cbase * 32;
+        const __nv_bfloat16 *mrow = p.mask + (long long)wk * p.mask_worker_stride + (long long)m * p.N + nm;
+        const bool vec = (m < p.M) && (nm + NCH * 32 <= p.N) && ((reinterpret_cast<uintptr_t>(mrow) & 15u) == 0);
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
+        for (int q = 0; q < NCH * 4; ++q) {
             if (vec) {
                 maskv[q] = *reinterpret_cast<const uint4 *>(mrow + q * 8);
             } else {
                 __align__(16) __nv_bfloat16 t[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
-                    t[e] = (m < p.M && n0 + q * 8 + e < p.N) ? mrow[q * 8 + e] : __float2bfloat16_rn(0.0f);
+                    t[e] = (m < p.M && nm + q * 8 + e < p.N) ? mrow[q * 8 + e] : __float2bfloat16_rn(0.0f);
                 maskv[q] = *reinterpret_cast<const uint4 *>(t);
             }
         }
@@ -329,26 +363,71 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     // ---- epilogue: every thread owns one accumulator row (TMEM lane) of the tile
     bool ok = mbar_wait(accum, 0, abort, limit + limit / 2);
+    if (EPI == EPI_SGD) {
+        const bool landed = mbar_wait(aux, 0, never, limit);      // issued copies must land in any case
+        ok = ok && landed;
+    }
     ok = __all_sync(0xffffffffu, ok);
     if (__syncthreads_and(ok ? 1 : 0)) {          // (also makes sbias visible)
         if (threadIdx.x == 0) COCOD_TRACE(4);
         tc_fence_after();
-        const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
-        uint32_t r[4][32];                         // the whole 128-column accumulator row
+        const uint32_t trow = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + cbase * 32;
+        uint32_t r[NCH][32];                       // this thread's part of the accumulator row
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(trow + c * 32, r[c]);
+        for (int cc = 0; cc < NCH; ++cc) tmem_ld32(trow + cc * 32, r[cc]);
         tmem_ld_wait();
-        if (EPI == EPI_F32) {
+        if (EPI == EPI_SGD) {
+            // gradient = accumulator; x and v tiles sit in shared memory in the TMA swizzle (16-byte piece
+            // j of row r at piece j ^ (r & 7)); the bf16 copy of x is staged in the idle ring.
+            uint8_t *ss = smem;
+#pragma unroll
+            for (int cc = 0; cc < NCH; ++cc) {
+                const int c = cbase + cc;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int off = c * (BM * 128) + row * 128 + ((j ^ (row & 7)) << 4);
+                    float4 xx = *reinterpret_cast<float4 *>(xs + off), vv = *reinterpret_cast<float4 *>(vs + off);
+                    const float4 gg = make_float4(__uint_as_float(r[cc][4 * j]), __uint_as_float(r[cc][4 * j + 1]),
+                                                  __uint_as_float(r[cc][4 * j + 2]), __uint_as_float(r[cc][4 * j + 3]));
+                    sgd_update(xx, vv, gg, p.lr, p.mu, p.wd);
+                    *reinterpret_cast<float4 *>(xs + off) = xx;
+                    *reinterpret_cast<float4 *>(vs + off) = vv;
+                    if (p.has_shadow) {
+                        const int nl = c * 32 + 4 * j, box = nl >> 6, piece = (nl & 63) >> 3, half = (nl >> 2) & 1;
+                        *reinterpret_cast<uint2 *>(ss + box * (BM * 128) + row * 128 + ((piece ^ (row & 7)) << 4) + half * 8) =
+                            make_uint2(pack_bf16x2(xx.x, xx.y), pack_bf16x2(xx.z, xx.w));
+                    }
+                }
+            }
+            fence_async_smem();
+            __syncthreads();
+            if (threadIdx.x == 0) COCOD_TRACE(6);
+            if (threadIdx.x == 0) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    if (n0 + c * 32 < p.N) {
+                        tma_store_3d(&sgd.x_out, smem_u32(xs) + c * (BM * 128), n0 + c * 32, m0, wk);
+                        tma_store_3d(&sgd.v, smem_u32(vs) + c * (BM * 128), n0 + c * 32, m0, wk);
+                    }
+                if (p.has_shadow) {
+#pragma unroll
+                    for (int b = 0; b < 2; ++b)
+                        if (n0 + b * 64 < p.N) tma_store_3d(&sgd.shadow, smem_base + b * (BM * 128), n0 + b * 64, m0, wk);
+                }
+                tma_store_commit();
+                tma_store_wait_read<0>();
+            }
+        } else if (EPI == EPI_F32) {
             if (p.map_c_ok) {
                 // stage the 128 x 128 fp32 tile in the (now idle) ring as four 128 x 32 sub-tiles with the
                 // 128-byte swizzle (16-byte piece j of row r sits at piece j ^ (r & 7)), then bulk-store them
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint8_t *tile = smem + c * (BM * 128);
+                for (int cc = 0; cc < NCH; ++cc) {
+                    uint8_t *tile = smem + (cbase + cc) * (BM * 128);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         *reinterpret_cast<uint4 *>(tile + row * 128 + ((j ^ (row & 7)) << 4)) =
-                            make_uint4(r[c][4 * j], r[c][4 * j + 1], r[c][4 * j + 2], r[c][4 * j + 3]);
+                            make_uint4(r[cc][4 * j], r[cc][4 * j + 1], r[cc][4 * j + 2], r[cc][4 * j + 3]);
                 }
                 fence_async_smem();
                 __syncthreads();
@@ -362,23 +441,24 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             } else if (m < p.M) {
                 float *dst = p.c + (long long)wk * p.c_worker_stride + (long long)m * p.ldc + n0;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int cc = 0; cc < NCH; ++cc)
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if (n0 + c * 32 + j < p.N) dst[c * 32 + j] = __uint_as_float(r[c][j]);
+                        if (n0 + (cbase + cc) * 32 + j < p.N) dst[(cbase + cc) * 32 + j] = __uint_as_float(r[cc][j]);
             }
         } else {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int cc = 0; cc < NCH; ++cc) {
+                const int c = cbase + cc;
                 const int nb = n0 + c * 32;
                 __align__(16) __nv_bfloat16 outv[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    float a = __uint_as_float(r[c][j]);
+                    float a = __uint_as_float(r[cc][j]);
                     if (EPI == EPI_BIAS_RELU) {
                         a = fmaxf(a + sbias[c * 32 + j], 0.0f);
                     } else {
-                        const __nv_bfloat16 *mk = reinterpret_cast<const __nv_bfloat16 *>(&maskv[c * 4 + (j >> 3)]);
+                        const __nv_bfloat16 *mk = reinterpret_cast<const __nv_bfloat16 *>(&maskv[cc * 4 + (j >> 3)]);
                         a = (__bfloat162float(mk[j & 7]) > 0.0f) ? a : 0.0f;
                     }
                     outv[j] = __float2bfloat16_rn(a);

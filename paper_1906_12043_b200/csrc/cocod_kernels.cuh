@@ -21,6 +21,7 @@
 
 namespace cocod {
 
+// (Non-template kernels are `static`: this header is included by both translation units of the library.)
 constexpr int kThreads = 256;
 
 // ------------------------------------------------------------------------------------------ loads / stores
@@ -123,13 +124,35 @@ local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__re
 }
 
 // Scalar path: misaligned pointers and the n mod 4 tail.  Elements [first, first + count).
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 local_step_scalar(const float *x_in, float *x_out, float *v, const float *__restrict__ g,
                   int64_t first, int64_t count, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < count; j += stride) {
         const int64_t e = first + j;
+        const float d = __fmaf_rn(wd, x_in[e], g[e]);
+        const float vn = __fmaf_rn(mu, v[e], d);
+        v[e] = vn;
+        const float xn = __fmaf_rn(-lr, vn, x_in[e]);
+        x_out[e] = xn;
+        if (shadow != nullptr) shadow[e] = __float2bfloat16_rn(xn);
+    }
+}
+
+// Same update on column ranges [lo[s], hi[s]) of every worker: grid (blocks, nseg, K).
+struct StepSegments {
+    int64_t lo[4], hi[4];
+};
+static __global__ void __launch_bounds__(kThreads)
+local_step_segments(const float *x_in, float *x_out, float *v, const float *__restrict__ g, int64_t P,
+                    StepSegments seg, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
+{
+    const int64_t lo = seg.lo[blockIdx.y], n = seg.hi[blockIdx.y] - lo;
+    const int64_t base = (int64_t)blockIdx.z * P + lo;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += stride) {
+        const int64_t e = base + j;
         const float d = __fmaf_rn(wd, x_in[e], g[e]);
         const float vn = __fmaf_rn(mu, v[e], d);
         v[e] = vn;
@@ -158,7 +181,7 @@ snapshot_vec4(const float4 *__restrict__ x, float4 *__restrict__ snap, int64_t n
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 snapshot_scalar(const float *__restrict__ x, float *__restrict__ snap, int64_t first, int64_t count)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
@@ -233,7 +256,7 @@ __device__ __forceinline__ void mean_rows(float (&s)[NV], int K, const float *__
 }
 
 // One thread owns one float4 of columns.  Needs P mod 4 == 0 and 16-byte aligned bases.
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__restrict__ w,
           float4 *__restrict__ mean, float inv_k)
 {
@@ -270,7 +293,7 @@ mean_vec8(const float *__restrict__ snap, int K, int64_t P, const float *__restr
 }
 
 // Any P / alignment: one thread per column.
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 mean_scalar(const float *__restrict__ snap, int K, int64_t P, const float *__restrict__ w,
             float *__restrict__ mean, float inv_k)
 {
@@ -353,7 +376,7 @@ merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, i
         }
 }
 
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 merge_scalar(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P,
              __nv_bfloat16 *__restrict__ shadow)
 {
@@ -369,7 +392,7 @@ merge_scalar(float *x, const float *snap, const float *__restrict__ mean, int K,
 }
 
 // Broadcast P values to K rows ("Initialize: x_i^0 = x_hat_0").
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 broadcast_rows(const float *__restrict__ x0, float *__restrict__ x, int K, int64_t P)
 {
     const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -379,7 +402,7 @@ broadcast_rows(const float *__restrict__ x0, float *__restrict__ x, int K, int64
 }
 
 // shadow[e] = bf16(x[e]) for a whole buffer (after the parameters were set from outside).
-__global__ void __launch_bounds__(kThreads)
+static __global__ void __launch_bounds__(kThreads)
 shadow_refresh(const float *__restrict__ x, __nv_bfloat16 *__restrict__ shadow, int64_t n)
 {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;

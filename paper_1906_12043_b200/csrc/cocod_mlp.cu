@@ -15,6 +15,7 @@
 //   dW1 = dz1^T x                     GEMM d_h x d_in x 128   A = dz1 read [k][m], B = x  read [k][n]   fp32 out
 #include "cocod_mlp.h"
 #include "cocod_gemm_sm100.cuh"
+#include "cocod_internal.h"
 
 #include <algorithm>
 #include <cstdio>
@@ -88,17 +89,21 @@ bool map_out(CUtensorMap *m, float *base, uint64_t cols, uint64_t rows, uint64_t
 
 template <int EPI, bool A_MN, bool B_MN>
 cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &c, const Params &p, int workers,
-                        cudaStream_t s)
+                        cudaStream_t s, const SgdMaps *sgd = nullptr)
 {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_bf16<EPI, A_MN, B_MN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             smem_bytes(MAX_STAGES));
+    static const SgdMaps no_sgd{};
+    constexpr int NT = (EPI == EPI_SGD) ? 256 : 128;      // the update epilogue is long and runs one CTA per SM
+    const int need = (EPI == EPI_SGD) ? smem_bytes_sgd(p.stages) : smem_bytes(p.stages);
+    static int configured = 0;
+    if (configured < need) {
+        const int cap = (EPI == EPI_SGD) ? smem_bytes_sgd(2) : smem_bytes(MAX_STAGES);
+        if (need > cap) return cudaErrorInvalidValue;
+        cudaError_t e = cudaFuncSetAttribute(gemm_bf16<EPI, A_MN, B_MN, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, cap);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured = cap;
     }
     const dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, workers);
-    gemm_bf16<EPI, A_MN, B_MN><<<grid, 128, smem_bytes(p.stages), s>>>(a, b, c, p);
+    gemm_bf16<EPI, A_MN, B_MN, NT><<<grid, NT, need, s>>>(a, b, c, sgd ? *sgd : no_sgd, p);
     return cudaGetLastError();
 }
 
@@ -319,6 +324,7 @@ struct cocod_mlp {
     bf16 *h1 = nullptr, *h2 = nullptr, *dz2 = nullptr, *dz1 = nullptr;
     float *dz3 = nullptr, *rowloss = nullptr;
     int *error_flag = nullptr;
+    float *gscratch = nullptr;          // K x P gradients of the fused path's small tensors (allocated on first use)
     // maps over scratch (fixed addresses): reduction-contiguous (k) and row-contiguous (mn) views
     CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
     long long launches = 0;
@@ -328,7 +334,7 @@ namespace {
 
 void mlp_free(cocod_mlp *h)
 {
-    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag};
+    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag, h->gscratch};
     for (void *p : ptrs) if (p) cudaFree(p);
     delete h;
 }
@@ -398,26 +404,38 @@ int64_t cocod_mlp_param_count(const cocod_mlp_handle *h) { return h ? h->P : -1;
 int64_t cocod_mlp_param_count_unpadded(const cocod_mlp_handle *h) { return h ? h->P_raw : -1; }
 int64_t cocod_mlp_launch_count(const cocod_mlp_handle *h) { return h ? h->launches : -1; }
 
-int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, const int32_t *labels, float *grads,
-                   float *loss, cocod_stream_t stream)
+}  // extern "C"
+
+namespace {
+
+// The whole gradient pass.  With fused == nullptr the weight gradients dW1, dW2 are written to `grads`;
+// otherwise their GEMMs apply the engine's local step in their epilogue (x, v and the bf16 copy of x
+// are updated in place, nothing is written to `grads` for W1 and W2).
+int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labels, float *grads, float *loss,
+             cudaStream_t s, const cocod_step_plan *fused)
 {
-    if (!h || !params_bf16 || !x || !labels || !grads || !loss) return COCOD_ERR_INVALID;
-    if ((reinterpret_cast<uintptr_t>(params_bf16) & 15u) || (reinterpret_cast<uintptr_t>(x) & 15u) ||
-        (reinterpret_cast<uintptr_t>(grads) & 15u))
-        return COCOD_ERR_INVALID;
-    cudaStream_t s = (cudaStream_t)stream;
-    const bf16 *prm = static_cast<const bf16 *>(params_bf16);
-    const bf16 *xin = static_cast<const bf16 *>(x);
     const int K = h->K, B = h->B, d_in = h->d_in, d_h = h->d_h, d_out = h->d_out;
     const long long P = h->P;
     const uint64_t uK = K, uB = B, uh = d_h, ui = d_in, uP = P;
     // maps over caller memory
-    CUtensorMap k_x, mn_x, k_w1, k_w2, mn_w2, c_w1, c_w2, none{};
+    CUtensorMap k_x, mn_x, k_w1, k_w2, mn_w2, c_w1{}, c_w2{}, none{};
     if (!map_k(&k_x, xin, ui, uB, uK, ui, uB * ui) || !map_mn(&mn_x, xin, ui, uB, uK, ui, uB * ui) ||
         !map_k(&k_w1, prm + h->oW1, ui, uh, uK, ui, uP) || !map_k(&k_w2, prm + h->oW2, uh, uh, uK, uh, uP) ||
-        !map_mn(&mn_w2, prm + h->oW2, uh, uh, uK, uh, uP) ||
-        !map_out(&c_w1, grads + h->oW1, ui, uh, uK, ui, uP) || !map_out(&c_w2, grads + h->oW2, uh, uh, uK, uh, uP))
+        !map_mn(&mn_w2, prm + h->oW2, uh, uh, uK, uh, uP))
         return COCOD_ERR_CUDA;
+    SgdMaps s_w1{}, s_w2{};
+    if (fused) {
+        float *xi = const_cast<float *>(fused->x_in);
+        bf16 *sh = fused->shadow;
+        bool ok = map_out(&s_w2.x_in, xi + h->oW2, uh, uh, uK, uh, uP) && map_out(&s_w2.x_out, fused->x_out + h->oW2, uh, uh, uK, uh, uP) &&
+                  map_out(&s_w2.v, fused->v + h->oW2, uh, uh, uK, uh, uP) &&
+                  map_out(&s_w1.x_in, xi + h->oW1, ui, uh, uK, ui, uP) && map_out(&s_w1.x_out, fused->x_out + h->oW1, ui, uh, uK, ui, uP) &&
+                  map_out(&s_w1.v, fused->v + h->oW1, ui, uh, uK, ui, uP);
+        if (ok && sh) ok = map_k(&s_w2.shadow, sh + h->oW2, uh, uh, uK, uh, uP) && map_k(&s_w1.shadow, sh + h->oW1, ui, uh, uK, ui, uP);
+        if (!ok) return COCOD_ERR_CUDA;
+    } else if (!map_out(&c_w1, grads + h->oW1, ui, uh, uK, ui, uP) || !map_out(&c_w2, grads + h->oW2, uh, uh, uK, uh, uP)) {
+        return COCOD_ERR_CUDA;
+    }
 #define LAUNCH_OK() do { if (cudaGetLastError() != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
 #define GEMM_OK(call) do { if ((call) != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
     Params p{};
@@ -432,7 +450,7 @@ int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, 
     GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, none, p, K, s)));
     // output layer, loss, dz3; then dz2, dW3, db3, db2
     head_logits<<<dim3(B / 8, K), 256, (size_t)d_out * d_h * sizeof(bf16), s>>>(h->h2, prm, P, h->oW3, h->ob3, labels,
-                                                                                h->dz3, h->rowloss, B, d_h, d_out);
+                                                                               h->dz3, h->rowloss, B, d_h, d_out);
     LAUNCH_OK();
     head_backward<<<dim3(d_h / 32, K), 128, 0, s>>>(h->h2, prm, h->dz3, h->rowloss, h->dz2, grads, loss, P, h->P_raw,
                                                     h->oW3, h->ob2, h->ob3, B, d_h, d_out);
@@ -450,13 +468,60 @@ int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, 
     Params r{};
     r.error_flag = h->error_flag;
     r.M = d_h; r.N = d_h; r.K = B; r.stages = stages_for(B);
-    r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
-    GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s)));
-    r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
-    GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s)));
+    if (fused) {
+        r.lr = fused->lr; r.mu = fused->mu; r.wd = fused->wd; r.has_shadow = fused->shadow != nullptr;
+        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2)));
+        r.N = d_in;
+        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1)));
+    } else {
+        r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s)));
+        r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s)));
+    }
 #undef LAUNCH_OK
 #undef GEMM_OK
     return COCOD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, const int32_t *labels, float *grads,
+                   float *loss, cocod_stream_t stream)
+{
+    if (!h || !params_bf16 || !x || !labels || !grads || !loss) return COCOD_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(params_bf16) & 15u) || (reinterpret_cast<uintptr_t>(x) & 15u) ||
+        (reinterpret_cast<uintptr_t>(grads) & 15u))
+        return COCOD_ERR_INVALID;
+    return run_grad(h, static_cast<const bf16 *>(params_bf16), static_cast<const bf16 *>(x), labels, grads, loss,
+                    (cudaStream_t)stream, nullptr);
+}
+
+int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x, const int32_t *labels, float *loss)
+{
+    if (!h || !engine || !x || !labels || !loss) return COCOD_ERR_INVALID;
+    if (reinterpret_cast<uintptr_t>(x) & 15u) return COCOD_ERR_INVALID;
+    cocod_step_plan plan{};
+    if (int rc = cocod_internal_plan_step(engine, &plan)) return rc;
+    if (plan.K != h->K || plan.P != h->P) return COCOD_ERR_INVALID;
+    if (!plan.shadow) return COCOD_ERR_STATE;            // the gradients are computed from the bf16 copy of x
+    if (!h->gscratch) {
+        if (cudaMalloc((void **)&h->gscratch, (size_t)h->K * h->P * sizeof(float)) != cudaSuccess) {
+            cudaGetLastError();
+            h->gscratch = nullptr;
+            return COCOD_ERR_OOM;
+        }
+    }
+    const long long before = h->launches;
+    if (int rc = run_grad(h, plan.shadow, static_cast<const bf16 *>(x), labels, h->gscratch, loss, plan.compute, &plan))
+        return rc;
+    // everything but W1 and W2: b1, then b2 | W3 | b3 | padding
+    const int64_t lo[2] = {h->ob1, h->ob2}, hi[2] = {h->oW2, h->P};
+    if (int rc = cocod_internal_step_segments(engine, h->gscratch, lo, hi, 2)) return rc;
+    (void)before;
+    return cocod_internal_finish_step(engine, 0);
 }
 
 int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream)

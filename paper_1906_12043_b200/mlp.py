@@ -17,6 +17,7 @@ SIGNATURES = {
     "cocod_mlp_param_count": (_i64, [_vp]),
     "cocod_mlp_param_count_unpadded": (_i64, [_vp]),
     "cocod_mlp_grad": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "cocod_mlp_grad_step": (_i, [_vp, _vp, _vp, _vp, _vp]),
     "cocod_mlp_check": (_i, [_vp, _vp]),
     "cocod_mlp_launch_count": (_i64, [_vp]),
     "cocod_gemm_wait_selftest": (_i, [_i, _vp]),
@@ -73,6 +74,20 @@ class MLPGrad:
                                       grads.data_ptr(), loss.data_ptr(), _cur_stream(stream))
         if rc != _E.OK:
             raise _E.CocodError(rc, "cocod_mlp_grad")
+
+    def grad_step(self, engine, x, labels, loss):
+        """Gradients and the engine's local step in one call (the update of W1 and W2 happens in the
+        epilogue of the weight-gradient GEMMs).  ``engine``: an Engine with K x P matching and the
+        bf16 shadow switched on.  Bit-identical to grad(...) followed by engine.local_step(grads)."""
+        import torch
+        K, B, d_in = self.K, self.batch, self.dims[0]
+        for t, dt, n, nm in ((x, torch.bfloat16, K * B * d_in, "x"), (labels, torch.int32, K * B, "labels"),
+                             (loss, torch.float32, K, "loss")):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == dt and t.numel() == n):
+                raise ValueError(f"{nm}: need a contiguous CUDA {dt} tensor of {n} elements")
+        rc = self._lib.cocod_mlp_grad_step(self._h, engine._h, x.data_ptr(), labels.data_ptr(), loss.data_ptr())
+        if rc != _E.OK:
+            raise _E.CocodError(rc, "cocod_mlp_grad_step")
 
     def check(self, stream=None):
         rc = self._lib.cocod_mlp_check(self._h, _cur_stream(stream))

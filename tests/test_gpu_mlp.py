@@ -295,3 +295,51 @@ def test_a_wait_that_nothing_satisfies_times_out_and_leaves_the_gpu_usable(M, E)
     M.gemm_bf16(bf16_tensor(A), bf16_tensor(A), C)
     np.testing.assert_allclose(cpu(C)[0], A[0].astype(np.float64) @ A[0].astype(np.float64).T, rtol=0, atol=1e-4)
     assert M.gemm_wait_selftest(20) == E.ERR_TIMEOUT     # and again
+
+
+@pytest.mark.parametrize("K,dims,wd", [(3, (200, 256, 256, 7), 5e-4), (16, I.MLP_DIMS, 0.0)])
+def test_fused_gradient_and_update_is_bit_identical_to_the_two_calls(M, E, K, dims, wd):
+    """cocod_mlp_grad_step (weight-gradient GEMMs apply the momentum update in their epilogue) against
+    cocod_mlp_grad followed by cocod_local_step: same x, v, bf16 copy and loss, bit for bit, through
+    rounds that include the buffer flip, in-place steps and merges."""
+    rng = np.random.default_rng(K)
+    k, rounds, lr, mu = 3, 2, 0.05, 0.9
+    mg = M.MLPGrad(K, 128, dims[0], dims[1], dims[3])
+    P, P_raw = mg.P, mg.P_raw
+    segs, _ = I.mlp_segments(dims)
+    x0 = np.zeros(P, np.float32)
+    for name, off, shape in segs:
+        n = int(np.prod(shape))
+        x0[off:off + n] = rng.standard_normal(n).astype(np.float32) * (1.0 / np.sqrt(shape[-1]) if name[0] == "W" else 0.1)
+    two, one = E.Engine(K, P, lr, mu, wd), E.Engine(K, P, lr, mu, wd)
+    for eng in (two, one):
+        eng.set_option(E.OPT_BF16_SHADOW, 1)
+        eng.set_params(x0)
+    side = torch.cuda.Stream(priority=-1)
+    grads = torch.empty((K, P), dtype=torch.float32, device="cuda")
+    loss2 = torch.empty(K, dtype=torch.float32, device="cuda")
+    loss1 = torch.empty(K, dtype=torch.float32, device="cuda")
+    for r in range(rounds):
+        two.comm_begin(side)
+        one.comm_begin(side)
+        for s in range(k):
+            t = r * k + s
+            X = bf16_tensor(np.stack([I.mlp_batch(w, t, 128, dims[0]) for w in range(K)]))
+            y = torch.from_numpy(rng.integers(0, dims[3], (K, 128)).astype(np.int32)).cuda()
+            mg.grad(two.bf16_shadow(), X, y, grads, loss2)
+            two.local_step(grads)
+            mg.grad_step(one, X, y, loss1)
+            what = f"round {r} step {s}"
+            assert torch.equal(loss1, loss2), what
+            assert torch.equal(one.get_params().view(torch.int32), two.get_params().view(torch.int32)), "x " + what
+            assert torch.equal(one.get_momentum().view(torch.int32), two.get_momentum().view(torch.int32)), "v " + what
+            assert torch.equal(one.bf16_shadow().view(torch.int16), two.bf16_shadow().view(torch.int16)), "shadow " + what
+        two.comm_end()
+        one.comm_end()
+        assert torch.equal(one.get_params().view(torch.int32), two.get_params().view(torch.int32)), f"x after merge {r}"
+    assert one.step_count == two.step_count == k * rounds
+    mg.check()
+    plain = E.Engine(K, P, lr, mu, wd)                    # without the bf16 copy there is nothing to compute from
+    with pytest.raises(E.CocodError) as e:
+        mg.grad_step(plain, X, y, loss1)
+    assert e.value.code == E.ERR_STATE
