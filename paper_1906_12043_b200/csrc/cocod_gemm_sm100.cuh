@@ -47,7 +47,7 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 enum Epilogue {
     EPI_F32 = 0,        // c[m][n] = acc                         (fp32, row stride ldc; TMA store if map_c_ok)
     EPI_BIAS_RELU = 1,  // o[m][n] = bf16(max(acc + bias[n], 0))
-    EPI_MASK = 2,       // o[m][n] = bf16(acc * (mask[m][n] > 0))
+    EPI_MASK = 2,       // o[m][n] = bf16(acc * (mask[m][n] > 0)); optionally colsum[n] = sum_m o[m][n] (M <= 128)
     EPI_SGD = 3         // g = acc: d = fma(wd, x, g); v = fma(mu, v, d); x = fma(-lr, v, x); shadow = bf16(x)
 };
 
@@ -69,6 +69,8 @@ struct Params {
     long long bias_worker_stride;
     const __nv_bfloat16 *mask;         // [M][N], row stride N
     long long mask_worker_stride;
+    float *colsum;                     // EPI_MASK, optional: [N] column sums of the bf16 output (needs M <= 128)
+    long long colsum_worker_stride;
     float lr, mu, wd;                  // EPI_SGD
     int has_shadow;                    // EPI_SGD: also write bf16(x)
     int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
@@ -463,6 +465,12 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     }
                     outv[j] = __float2bfloat16_rn(a);
                 }
+                if (EPI == EPI_MASK && p.colsum != nullptr) {       // stage the row for the column sums (padded rows)
+                    const uint4 *src = reinterpret_cast<const uint4 *>(outv);
+                    uint4 *stg = reinterpret_cast<uint4 *>(smem + row * 272 + c * 64);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) stg[j] = src[j];
+                }
                 if (m < p.M && nb < p.N) {
                     __nv_bfloat16 *dst = p.o + (long long)wk * p.o_worker_stride + (long long)m * p.N + nb;
                     if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
@@ -475,6 +483,18 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                             if (nb + j < p.N) dst[j] = outv[j];
                     }
                 }
+            }
+        }
+        if (EPI == EPI_MASK && p.colsum != nullptr) {
+            // the whole batch is in this tile: thread t adds column t over the rows, in row order
+            __syncthreads();
+            const int t = threadIdx.x;
+            if (t < BN && n0 + t < p.N) {
+                const int rows = (p.M - m0 < BM) ? (p.M - m0) : BM;
+                float acc = 0.0f;
+                for (int rr = 0; rr < rows; ++rr)
+                    acc += __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(smem + rr * 272 + t * 2));
+                p.colsum[(long long)wk * p.colsum_worker_stride + n0 + t] = acc;
             }
         }
     } else if (threadIdx.x == 0 && p.error_flag != nullptr) {

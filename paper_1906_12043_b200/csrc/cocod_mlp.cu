@@ -9,8 +9,8 @@
 //   h2 = bf16(relu(h1 W2^T + b2))     GEMM 128 x d_h x d_h    A = h1, B = W2           epilogue bias+ReLU
 //   logits = h2 W3^T + b3 ; loss ; dz3 = bf16((softmax - onehot)/batch)                CUDA cores
 //   dz2 = bf16((dz3 W3) * (h2 > 0)) ; dW3 = dz3^T h2 ; db3, db2 = column sums           CUDA cores
-//   dz1 = bf16((dz2 W2) * (h1 > 0))   GEMM 128 x d_h x d_h    A = dz2, B = W2 read [k][n]  epilogue mask
-//   db1 = column sums of dz1                                                           CUDA cores
+//   dz1 = bf16((dz2 W2) * (h1 > 0))   GEMM 128 x d_h x d_h    A = dz2, B = W2 read [k][n]  epilogue mask,
+//   db1 = column sums of dz1                                   (same epilogue: the batch is one tile)
 //   dW2 = dz2^T h1                    GEMM d_h x d_h x 128    A = dz2 read [k][m], B = h1 read [k][n]   fp32 out
 //   dW1 = dz1^T x                     GEMM d_h x d_in x 128   A = dz1 read [k][m], B = x  read [k][n]   fp32 out
 #include "cocod_mlp.h"
@@ -206,7 +206,7 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
               int B, int d_h, int d_out)
 {
     constexpr int NW = 4;                          // warps per CTA; warp wp owns samples wp, wp + 4, ...
-    __shared__ float sdz[128 * 16];
+    __shared__ __align__(16) float sdz[128 * 16];
     __shared__ float red[NW][16][33];
     __shared__ float colsum[NW][33];
     const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
@@ -241,11 +241,16 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
             if (b < B) {
                 const float h = hreg[q];
                 float a = 0.0f;
+                const float4 *d4 = reinterpret_cast<const float4 *>(sdz + b * 16);
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const float d = sdz[b * 16 + c];
-                    a = fmaf(d, w3[c], a);
-                    acc3[c] = fmaf(d, h, acc3[c]);
+                for (int c4 = 0; c4 < 4; ++c4) {
+                    const float4 dd = d4[c4];
+                    const float d[4] = {dd.x, dd.y, dd.z, dd.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        a = fmaf(d[e], w3[4 * c4 + e], a);
+                        acc3[4 * c4 + e] = fmaf(d[e], h, acc3[4 * c4 + e]);
+                    }
                 }
                 const bf16 v = __float2bfloat16_rn(h > 0.0f ? a : 0.0f);
                 dz2[((long long)w * B + b) * d_h + j] = v;
@@ -284,35 +289,6 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
             loss[w] = s / (float)B;
         }
         for (long long i = P_raw + threadIdx.x; i < P; i += 32 * NW) grads[(long long)w * P + i] = 0.0f;
-    }
-}
-
-// db1[j] = sum_b dz1[b][j].  One CTA = 32 hidden units; warp wp sums samples wp, wp + 8, ... (all its
-// loads in flight at once), then the 8 partial sums are added in warp order.  grid (d_h / 32, K).
-__global__ void __launch_bounds__(256)
-colsum_bf16(const bf16 *__restrict__ dz, float *__restrict__ grads, long long P, long long ob, int B, int d_h)
-{
-    __shared__ float part[8][33];
-    const int w = blockIdx.y, lane = threadIdx.x & 31, wp = threadIdx.x >> 5, j = blockIdx.x * 32 + lane;
-    const bf16 *col = dz + (long long)w * B * d_h + j;
-    float s = 0.0f;
-    for (int q0 = 0; q0 * 8 < B; q0 += 16) {
-        float t[16];
-#pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            const int b = wp + 8 * (q0 + q);
-            t[q] = (b < B && j < d_h) ? __bfloat162float(col[(long long)b * d_h]) : 0.0f;
-        }
-#pragma unroll
-        for (int q = 0; q < 16; ++q) s += t[q];
-    }
-    part[wp][lane] = s;
-    __syncthreads();
-    if (threadIdx.x < 32 && j < d_h) {
-        float r = 0.0f;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) r += part[q][threadIdx.x];
-        grads[(long long)w * P + ob + j] = r;
     }
 }
 
@@ -461,9 +437,8 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     q.M = B; q.N = d_h; q.K = d_h; q.stages = stages_for(d_h);
     q.o = h->dz1; q.o_worker_stride = (long long)B * d_h;
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
+    q.colsum = grads + h->ob1; q.colsum_worker_stride = P;      // db1 = column sums of dz1, from the same epilogue
     GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, none, q, K, s)));
-    colsum_bf16<<<dim3((d_h + 31) / 32, K), 256, 0, s>>>(h->dz1, grads, P, h->ob1, B, d_h);
-    LAUNCH_OK();
     // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
     Params r{};
     r.error_flag = h->error_flag;
