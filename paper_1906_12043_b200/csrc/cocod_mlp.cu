@@ -278,15 +278,25 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
         grads[(long long)w * P + ob2 + j0 + threadIdx.x] = s;
     }
     if (blockIdx.x == 0) {
-        if (threadIdx.x < d_out) {
-            float s = 0.0f;
-            for (int b = 0; b < B; ++b) s += sdz[b * 16 + threadIdx.x];
-            grads[(long long)w * P + ob3 + threadIdx.x] = s;
-        }
-        if (threadIdx.x == 32) {
-            float s = 0.0f;
-            for (int b = 0; b < B; ++b) s += rowloss[(long long)w * B + b];
-            loss[w] = s / (float)B;
+        // per-worker scalars: each by one warp, lane-strided partial sums then a fixed shuffle tree
+        if (wp == 0) {
+            for (int c = 0; c < d_out; ++c) {
+                float s = 0.0f;
+                for (int b = lane; b < B; b += 32) s += sdz[b * 16 + c];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                if (lane == 0) grads[(long long)w * P + ob3 + c] = s;
+            }
+        } else if (wp == 1) {
+            float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (lane + 32 * i < B) t[i] = rowloss[(long long)w * B + lane + 32 * i];
+            float s = (t[0] + t[1]) + (t[2] + t[3]);
+            for (int b = lane + 128; b < B; b += 32) s += rowloss[(long long)w * B + b];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane == 0) loss[w] = s / (float)B;
         }
         for (long long i = P_raw + threadIdx.x; i < P; i += 32 * NW) grads[(long long)w * P + i] = 0.0f;
     }
