@@ -564,6 +564,47 @@ def run_mlp(args):
     except OSError:
         pass
     flops_step = K * 2 * B * (2 * dims[0] * dims[1] + 3 * dims[1] * dims[2] + 3 * dims[2] * dims[3])
+    # roofline of the dominant kernel (the HBM-bound local step with bf16 shadow: 22 B per worker-parameter);
+    # this workload is launch-latency-bound, so the per-kernel events are taken in a short pass of their own
+    roofline = None
+    by = {}
+    if not args.fused:
+        eng.set_option(E.OPT_PROFILE, 1)
+        eng.profile_reset()
+        for _ in range(min(args.steps, 50)):
+            one_round()
+        by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+        eng.set_option(E.OPT_PROFILE, 0)
+    if by.get("local_step"):
+        iv = by["local_step"]
+        avg_ms = sum(b - a for a, b in iv) / len(iv)
+        hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+        gbs = 22.0 * K * P / (avg_ms * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": "local_step (with bf16 shadow)", "achieved": round(gbs, 1), "peak": hbm_peak,
+                    "unit": "GB/s", "frac": round(gbs / hbm_peak, 4), "traffic": None,
+                    "peak_kind": "measured" if "hbm_gbs" in peaks else "fallback",
+                    "algorithmic_bytes_per_launch": 22 * K * P, "avg_launch_ms": round(avg_ms, 5),
+                    "measured_in": "separate pass with per-kernel events"}
+    # the oracle beside it: one local step of two workers (numpy fp64 gradient + C update)
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        from oracle import mlp_oracle as MO
+        from oracle.cocod_oracle import OracleEngine
+        nw = 2
+        oe = OracleEngine(nw, P_raw, lr, mu, wd, mode="ref")
+        oe.set_params(x0[:P_raw])
+        Xo = [I.mlp_batch(w, 0) for w in range(nw)]
+        yo = [I.mlp_teacher_labels(Xo[w], teacher) for w in range(nw)]
+        t0 = time.perf_counter()
+        n_cpu = 0
+        while time.perf_counter() - t0 < 10.0:
+            g = np.stack([MO.loss_and_grad(oe.x[w], Xo[w], yo[w], dims, emulate_bf16=True)[1] for w in range(nw)])
+            oe.local_step(g)
+            n_cpu += 1
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": nw * P_raw * n_cpu / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                        "sample": f"{n_cpu} local steps of {nw} workers (numpy fp64 gradient with bf16 rounding points + "
+                                  f"reference-mode update), no averaging rounds"}
     print(json.dumps({
         "metric": METRIC, "value": K * P_raw * k * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps,
@@ -572,7 +613,7 @@ def run_mlp(args):
         "config": {"workload": "mlp", "K": K, "P": P_raw, "P_padded": P, "k": k, "lr": lr, "mu": mu, "wd": wd,
                    "mlp": list(dims), "batch": B, "minibatch_ring": ring_n, "cuda_graph": bool(args.graph),
                    "fused_update": bool(args.fused)},
-        "clocks": clocks, "gpu_launches": launches,
+        "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
         "local_steps_per_s": k * args.steps / (ms * 1e-3), "ms_per_local_step": ms / (k * args.steps),
         "tensor_tflops": flops_step * k * args.steps / (ms * 1e-3) / 1e12,
         "tensor_peak_tflops": peaks.get("bf16_tflops"),
