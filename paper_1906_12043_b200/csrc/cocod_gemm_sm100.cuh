@@ -227,8 +227,8 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     uint8_t *tail = (EPI == EPI_SGD) ? vs + BM * BN * 4 : xs;
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_STAGES), accum = smem_u32(bars + 2 * MAX_STAGES);
-    const uint32_t aux = smem_u32(bars + 2 * MAX_STAGES + 1);      // EPI_SGD: x and v tiles have landed
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 2);
+    const uint32_t aux = smem_u32(bars + 2 * MAX_STAGES + 1);      // EPI_SGD: four barriers, one per 32-column chunk of x and v
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 5);
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
     float *sbias = reinterpret_cast<float *>(tail + 256);
@@ -268,7 +268,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum, 1);
-        mbar_init(aux, 1);
+        for (int c = 0; c < 4; ++c) mbar_init(aux + 8 * c, 1);
         abort[0] = 0;
         abort[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -278,11 +278,11 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             for (; armed < nkb && armed < stages; ++armed) issue_loads(armed, armed);
         if (EPI == EPI_SGD) {         // the tiles the update needs: in flight under the whole main loop
             asm volatile("prefetch.tensormap [%0];" ::"l"(&sgd.x_out) : "memory");
-            mbar_expect_tx(aux, 2 * BM * BN * 4);
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                tma_load_3d(smem_u32(xs) + c * (BM * 128), &sgd.x_in, aux, n0 + c * 32, m0, wk);
-                tma_load_3d(smem_u32(vs) + c * (BM * 128), &sgd.v, aux, n0 + c * 32, m0, wk);
+                mbar_expect_tx(aux + 8 * c, 2 * BM * 128);
+                tma_load_3d(smem_u32(xs) + c * (BM * 128), &sgd.x_in, aux + 8 * c, n0 + c * 32, m0, wk);
+                tma_load_3d(smem_u32(vs) + c * (BM * 128), &sgd.v, aux + 8 * c, n0 + c * 32, m0, wk);
             }
         }
     }
@@ -365,9 +365,8 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
     // ---- epilogue: every thread owns one accumulator row (TMEM lane) of the tile
     bool ok = mbar_wait(accum, 0, abort, limit + limit / 2);
-    if (EPI == EPI_SGD) {
-        const bool landed = mbar_wait(aux, 0, never, limit);      // issued copies must land in any case
-        ok = ok && landed;
+    if (EPI == EPI_SGD && !ok) {                                  // issued copies must land in any case
+        for (int c = 0; c < 4; ++c) mbar_wait(aux + 8 * c, 0, never, limit);
     }
     ok = __all_sync(0xffffffffu, ok);
     if (__syncthreads_and(ok ? 1 : 0)) {          // (also makes sbias visible)
@@ -381,10 +380,17 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (EPI == EPI_SGD) {
             // gradient = accumulator; x and v tiles sit in shared memory in the TMA swizzle (16-byte piece
             // j of row r at piece j ^ (r & 7)); the bf16 copy of x is staged in the idle ring.
+            // Chunks are handed to the store engine one by one: the 128 threads that share a chunk
+            // meet on a named barrier and their first thread issues that chunk's bulk stores while the
+            // others already update the next chunk.
             uint8_t *ss = smem;
+            const int group = warp >> 2;                       // 128-thread group (NT == 256: two of them)
+            const bool leader = (threadIdx.x & 127) == 0;
+            bool landed = true;
 #pragma unroll
             for (int cc = 0; cc < NCH; ++cc) {
                 const int c = cbase + cc;
+                landed = mbar_wait(aux + 8 * c, 0, never, limit) && landed;      // this chunk's x and v tiles
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const int off = c * (BM * 128) + row * 128 + ((j ^ (row & 7)) << 4);
@@ -400,25 +406,21 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                             make_uint2(pack_bf16x2(xx.x, xx.y), pack_bf16x2(xx.z, xx.w));
                     }
                 }
-            }
-            fence_async_smem();
-            __syncthreads();
-            if (threadIdx.x == 0) COCOD_TRACE(6);
-            if (threadIdx.x == 0) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
+                fence_async_smem();
+                asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
+                if (leader) {
                     if (n0 + c * 32 < p.N) {
                         tma_store_3d(&sgd.x_out, smem_u32(xs) + c * (BM * 128), n0 + c * 32, m0, wk);
                         tma_store_3d(&sgd.v, smem_u32(vs) + c * (BM * 128), n0 + c * 32, m0, wk);
                     }
-                if (p.has_shadow) {
-#pragma unroll
-                    for (int b = 0; b < 2; ++b)
-                        if (n0 + b * 64 < p.N) tma_store_3d(&sgd.shadow, smem_base + b * (BM * 128), n0 + b * 64, m0, wk);
+                    // a 64-column box of the bf16 copy is complete after every second chunk
+                    if (p.has_shadow && (c & 1) && n0 + (c >> 1) * 64 < p.N)
+                        tma_store_3d(&sgd.shadow, smem_base + (c >> 1) * (BM * 128), n0 + (c >> 1) * 64, m0, wk);
+                    tma_store_commit();
                 }
-                tma_store_commit();
-                tma_store_wait_read<0>();
             }
+            if (leader) tma_store_wait_read<0>();              // shared memory must outlive the reads
+            if (!landed && p.error_flag != nullptr) atomicExch(p.error_flag, 4);
         } else if (EPI == EPI_F32) {
             if (p.map_c_ok) {
                 // stage the 128 x 128 fp32 tile in the (now idle) ring as four 128 x 32 sub-tiles with the
