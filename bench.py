@@ -323,6 +323,33 @@ def run_ours(args, wl):
     isolated = kernel_table(summarize_profile(eng.profile_records(), E.KERNEL_NAMES))
     eng.set_option(E.OPT_PROFILE, 0)
 
+    # ---- the paper's sequential counterparts on the same kernels: k local steps + blocking averaging
+    #      (Local-SGD) and k steps of gradient averaging (S-SGD); for context next to the decoupled round
+    def timed(fn, n):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        ev0.record(compute)
+        for _ in range(n):
+            fn()
+        ev1.record(compute)
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) / n
+
+    def local_sgd_round():
+        for _ in range(k):
+            eng.local_step(ring[step_no[0] % len(ring)])
+            step_no[0] += 1
+        eng.local_sgd_average()
+
+    def ssgd_round():
+        for _ in range(k):
+            eng.ssgd_step(ring[step_no[0] % len(ring)])
+            step_no[0] += 1
+
+    n_cmp = min(args.steps, 30)
+    schemes = {"cocod": ms / args.steps, "local_sgd": timed(local_sgd_round, n_cmp), "ssgd": timed(ssgd_round, n_cmp)}
+
     # ---- the same rounds replayed from a CUDA graph (extra figure; the contract value stays the eager one)
     graph_extra = None
     if graph is None and world == 1:
@@ -427,6 +454,7 @@ def run_ours(args, wl):
             "kernels_in_loop": in_loop, "kernels_isolated": isolated,
             "overlap_fraction": overlap, "ms_per_round_overlapped": ms / args.steps,
             "ms_per_round_serial": ms_serial, "cuda_graph_replay": graph_extra,
+            "ms_per_round_by_scheme": schemes,
             "hbm_gbs_whole_round": wl.bytes_per_round(args.snapshot == "copy") / (ms / args.steps * 1e-3) / 1e9,
         }
         print(json.dumps(line))

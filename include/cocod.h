@@ -103,6 +103,23 @@ int cocod_comm_begin(cocod_handle *h, cocod_stream_t side);
 int cocod_comm_end(cocod_handle *h);
 
 /* ---------------------------------------------------------------------------------------------
+ * The two sequential schemes the paper compares against (Section 2 and Section 4.2, time-speedup
+ * equations of S-SGD and Local-SGD), as calls on the same engine and kernels, so that the cost of
+ * NOT decoupling can be measured on identical code.
+ *
+ * Local-SGD: after k local steps every worker's model is replaced by the weighted mean of all
+ * models, sequentially: x^i <- sum_j (M_j / sum M) x^j.  On the compute stream, no side stream.
+ * Equals cocod_comm_begin + cocod_comm_end with no step in between.  STATE while a communication
+ * is in flight. */
+int cocod_local_sgd_average(cocod_handle *h);
+
+/* S-SGD: one synchronous step: the K workers' gradients are averaged (same weights), and every
+ * worker applies the same averaged gradient: g_bar = sum_j (M_j / sum M) g^j, then the local update
+ * with g_bar.  grads: device, K x P, borrowed.  On the compute stream.  STATE while a communication
+ * is in flight (the average-model buffer is used for g_bar; cocod_get_mean is invalid afterwards). */
+int cocod_ssgd_step(cocod_handle *h, const float *grads);
+
+/* ---------------------------------------------------------------------------------------------
  * Additions the five calls above need around them (initial point, results, schedule).      */
 
 /* Stream for local steps, stored copies and merges (borrowed).  Not while a communication is

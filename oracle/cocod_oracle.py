@@ -154,6 +154,30 @@ class OracleEngine:
             L.oracle_merge_mirror(self.K, self.P, _p(self.x), _p(self.snap), _p(self.mean))
         self.in_flight = False
 
+    # -- the sequential schemes the paper compares against (Section 2; Section 4.2)
+    def local_sgd_average(self) -> None:
+        """Local-SGD: every worker's model becomes the weighted mean of all models."""
+        if self.in_flight:
+            raise RuntimeError("communication in flight")
+        L = lib()
+        Mp = None if self.M is None else _p(self.M)
+        fn = {"ref": L.oracle_mean_ref, "mirror": L.oracle_mean_mirror, "f64": L.oracle_mean_f64}[self.mode]
+        fn(self.K, self.P, _p(self.x), Mp, _p(self.mean))
+        self.x[:] = self.mean[None, :]
+
+    def ssgd_step(self, g) -> None:
+        """S-SGD: the workers' gradients are averaged with the same weights and every worker applies
+        the averaged gradient (equivalent to one worker with the summed mini-batch)."""
+        if self.in_flight:
+            raise RuntimeError("communication in flight")
+        g = np.ascontiguousarray(g, self.dt)
+        L = lib()
+        Mp = None if self.M is None else _p(self.M)
+        gbar = np.zeros(self.P, self.dt)
+        fn = {"ref": L.oracle_mean_ref, "mirror": L.oracle_mean_mirror, "f64": L.oracle_mean_f64}[self.mode]
+        fn(self.K, self.P, _p(g), Mp, _p(gbar))
+        self.local_step(np.ascontiguousarray(np.tile(gbar, (self.K, 1))))
+
     def run(self, grad_fn, k: int, rounds: int, on_round=None) -> None:
         """The while loop of Algorithm 1 for whole rounds: ``grad_fn(tau)`` returns the
         K x P gradients of global local-step index tau = round * k + s."""

@@ -453,6 +453,60 @@ int cocod_comm_end(cocod_handle *h)
     return COCOD_OK;
 }
 
+int cocod_local_sgd_average(cocod_handle *h)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    int nl = 0;
+    {
+        Bracket br(h, h->compute, COCOD_KERNEL_MEAN);
+        CK(h, launch_mean(h->buf[h->cur], h->K, h->P, h->weighted ? h->w : nullptr, h->mean, h->compute, &nl));
+    }
+    // after the sequential mean nothing from the side stream is pending for this value
+    CK(h, cudaEventRecord(h->ev_mean, h->compute));
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CK(h, cudaStreamIsCapturing(h->compute, &cap));
+    h->mean_captured = (cap != cudaStreamCaptureStatusNone);
+    h->side = h->compute;
+    h->mean_valid = true;
+    cocod::broadcast_rows<<<grid_for(h->P, cocod::kThreads), cocod::kThreads, 0, h->compute>>>(
+        h->mean, h->buf[h->cur], h->K, h->P);
+    CK(h, cudaGetLastError());
+    h->launches += nl + 1;
+    return refresh_shadow(h);
+}
+
+int cocod_ssgd_step(cocod_handle *h, const float *grads)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!grads) return COCOD_ERR_INVALID;
+    if (h->state != IDLE) return COCOD_ERR_STATE;      // the average-model buffer holds the averaged gradient
+    using namespace cocod;
+    int nl = 0;
+    {
+        Bracket br(h, h->compute, COCOD_KERNEL_MEAN);
+        CK(h, launch_mean(grads, h->K, h->P, h->weighted ? h->w : nullptr, h->mean, h->compute, &nl));
+    }
+    h->mean_valid = false;                              // it is a gradient now, not an average model
+    float *x = h->buf[h->cur];
+    {
+        Bracket br(h, h->compute, COCOD_KERNEL_LOCAL_STEP);
+        if ((h->P % 4) == 0 && (h->shadow == nullptr || (reinterpret_cast<uintptr_t>(h->shadow) & 7u) == 0)) {
+            const int64_t pvec = h->P / 4;
+            local_step_shared_grad_vec4<<<dim3(grid_for(pvec, kThreads), (unsigned)h->K), kThreads, 0, h->compute>>>(
+                reinterpret_cast<const float4 *>(x), reinterpret_cast<float4 *>(x), reinterpret_cast<float4 *>(h->v),
+                reinterpret_cast<const float4 *>(h->mean), pvec, h->lr, h->mu, h->wd, h->shadow);
+        } else {
+            local_step_shared_grad_scalar<<<dim3(grid_for(h->P, kThreads), (unsigned)h->K), kThreads, 0, h->compute>>>(
+                x, x, h->v, h->mean, h->P, h->lr, h->mu, h->wd, h->shadow);
+        }
+        CK(h, cudaGetLastError());
+    }
+    h->launches += nl + 1;
+    ++h->steps;
+    return COCOD_OK;
+}
+
 int cocod_set_stream(cocod_handle *h, cocod_stream_t compute)
 {
     if (int rc = check_live(h)) return rc;

@@ -391,6 +391,37 @@ merge_scalar(float *x, const float *snap, const float *__restrict__ mean, int K,
     }
 }
 
+// Local step of every worker with ONE gradient vector shared by all (S-SGD: the averaged gradient):
+// grid (blocks over P / 4, K); gbar is read K times but stays in L2.  Same arithmetic as the local step.
+static __global__ void __launch_bounds__(kThreads)
+local_step_shared_grad_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__restrict__ gbar,
+                            int64_t pvec, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
+{
+    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= pvec) return;
+    const int64_t e = (int64_t)blockIdx.y * pvec + c;
+    float4 xx = x_in[e], vv = v[e];
+    const float4 gg = gbar[c];
+    sgd_update(xx, vv, gg, lr, mu, wd);
+    v[e] = vv;
+    x_out[e] = xx;
+    if (shadow != nullptr) st_shadow4(shadow + 4 * e, xx);
+}
+static __global__ void __launch_bounds__(kThreads)
+local_step_shared_grad_scalar(const float *x_in, float *x_out, float *v, const float *__restrict__ gbar, int64_t P,
+                              float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
+{
+    const int64_t p = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (p >= P) return;
+    const int64_t e = (int64_t)blockIdx.y * P + p;
+    const float d = __fmaf_rn(wd, x_in[e], gbar[p]);
+    const float vn = __fmaf_rn(mu, v[e], d);
+    v[e] = vn;
+    const float xn = __fmaf_rn(-lr, vn, x_in[e]);
+    x_out[e] = xn;
+    if (shadow != nullptr) shadow[e] = __float2bfloat16_rn(xn);
+}
+
 // Broadcast P values to K rows ("Initialize: x_i^0 = x_hat_0").
 static __global__ void __launch_bounds__(kThreads)
 broadcast_rows(const float *__restrict__ x0, float *__restrict__ x, int K, int64_t P)

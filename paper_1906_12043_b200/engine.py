@@ -29,6 +29,8 @@ SIGNATURES = {
     "cocod_local_step_host": (_i, [_vp, _vp]),
     "cocod_comm_begin": (_i, [_vp, _vp]),
     "cocod_comm_end": (_i, [_vp]),
+    "cocod_local_sgd_average": (_i, [_vp]),
+    "cocod_ssgd_step": (_i, [_vp, _vp]),
     "cocod_set_stream": (_i, [_vp, _vp]),
     "cocod_set_params": (_i, [_vp, _vp, _i]),
     "cocod_set_params_all": (_i, [_vp, _vp, _i]),
@@ -176,6 +178,17 @@ class Engine:
     def comm_end(self):
         """Line 6: x^i <- x_hat_t + (x^i - x_t^i)."""
         self._ck(self._lib.cocod_comm_end(self._h), "cocod_comm_end")
+
+    # -- the sequential schemes of the paper's comparison
+    def local_sgd_average(self):
+        """Local-SGD's blocking model averaging: every x^i <- weighted mean of all x^j."""
+        self._ck(self._lib.cocod_local_sgd_average(self._h), "cocod_local_sgd_average")
+
+    def ssgd_step(self, grads):
+        """S-SGD: average the K gradients, every worker applies the averaged gradient."""
+        if self._check_tensor(grads, self.K * self.P, "grads") != 0:
+            raise ValueError("grads must be a CUDA tensor")
+        self._ck(self._lib.cocod_ssgd_step(self._h, _ptr(grads)), "cocod_ssgd_step")
 
     # -- around it
     def set_stream(self, stream):

@@ -525,6 +525,53 @@ def test_switching_the_compute_stream_keeps_work_ordered(E):
     assert_bit_equal(cpu(eng.get_params()), mir.x)
 
 
+@pytest.mark.parametrize("K,P,weighted", [(4, 100_000, False), (5, 1001, True), (16, 65_536 + 8, True), (2, 7, False)])
+def test_sequential_schemes_local_sgd_and_ssgd(E, K, P, weighted):
+    """The two schemes the paper compares against, on the same kernels: Local-SGD (k local steps, then
+    blocking model averaging) and S-SGD (gradient averaging every step), against the oracle."""
+    rng = np.random.default_rng(K + P)
+    M = rng.integers(1, 9, K).astype(float) if weighted else None
+    x0 = (rng.standard_normal(P) * 0.05).astype(np.float32)
+    G = (rng.standard_normal((6, K, P)) * 0.02).astype(np.float32)
+    for scheme in ("local_sgd", "ssgd"):
+        eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
+        ref = OracleEngine(K, P, 0.1, 0.9, 5e-4, mode="ref", batch_sizes=M)
+        mir = OracleEngine(K, P, 0.1, 0.9, 5e-4, mode="mirror", batch_sizes=M)
+        if M is not None:
+            eng.set_batch_sizes(M)
+        eng.set_params(x0)
+        ref.set_params(x0)
+        mir.set_params(x0)
+        for t in range(6):
+            gd = torch.from_numpy(G[t]).cuda()
+            if scheme == "ssgd":
+                eng.ssgd_step(gd)
+                ref.ssgd_step(G[t])
+                mir.ssgd_step(G[t])
+            else:
+                eng.local_step(gd)
+                ref.local_step(G[t])
+                mir.local_step(G[t])
+                if t % 2 == 1:                     # period k = 2
+                    eng.local_sgd_average()
+                    ref.local_sgd_average()
+                    mir.local_sgd_average()
+        x, v = cpu(eng.get_params()), cpu(eng.get_momentum())
+        assert_bit_equal(x, mir.x, f"{scheme}: x vs mirror")
+        assert_bit_equal(v, mir.v, f"{scheme}: v vs mirror")
+        assert_close_scaled(x, ref.x, 1e-5, f"{scheme}: x vs ref")
+        if scheme == "ssgd":
+            for i in range(1, K):
+                assert_bit_equal(x[i], x[0], "replicas stay identical under S-SGD")
+        assert eng.step_count == 6
+    eng.comm_begin(torch.cuda.Stream())
+    with pytest.raises(E.CocodError):
+        eng.ssgd_step(gd)
+    with pytest.raises(E.CocodError):
+        eng.local_sgd_average()
+    eng.comm_end()
+
+
 def test_learning_rate_schedule_and_profile_records(E):
     K, P = 2, 4096
     eng = E.Engine(K, P, 0.1, 0.9, 0.0)

@@ -413,3 +413,52 @@ def test_state_machine_rejects_double_begin_and_end_without_begin():
     eng.comm_begin()
     with pytest.raises(RuntimeError):
         eng.comm_begin()
+
+
+# ----------------------------------------------------------------------------- the sequential schemes
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("weighted", [False, True])
+def test_ssgd_equals_one_worker_on_the_averaged_gradient(mode, weighted):
+    """S-SGD with K workers is single-worker momentum SGD driven by the weighted mean gradient (more
+    workers = a larger mini-batch); all replicas stay identical."""
+    rng = np.random.default_rng(21)
+    K, P, steps = 5, 27, 7
+    lr, mu, wd = np.float32(0.1), np.float32(0.9), np.float32(5e-4)
+    x0 = (rng.standard_normal(P) * 0.01).astype(np.float32)
+    G = rand_grads(rng, K, P, steps).astype(np.float32)
+    M = rng.integers(1, 6, K).astype(float) if weighted else None
+    w = np.full(K, 1 / K) if M is None else M / M.sum()
+    eng = OracleEngine(K, P, lr, mu, wd, mode=mode, batch_sizes=M)
+    eng.set_params(x0)
+    for t in range(steps):
+        eng.ssgd_step(G[t])
+    for i in range(1, K):
+        np.testing.assert_array_equal(eng.x[i], eng.x[0])
+    wx, wv = momentum_sgd_single(float(lr), float(mu), float(wd), x0, np.einsum("j,tjp->tp", w, G.astype(float)))
+    np.testing.assert_allclose(eng.x[0], wx, rtol=0, atol=tol(mode) * 0.05)
+    np.testing.assert_allclose(eng.v[0], wv, rtol=0, atol=tol(mode) * 0.05)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_local_sgd_average_is_the_zero_drift_merge(mode):
+    """Local-SGD's averaging step equals Step I + line 6 of Algorithm 1 with no local step in between,
+    and with k = 1 and plain SGD, Local-SGD and S-SGD produce the same models."""
+    rng = np.random.default_rng(22)
+    K, P = 4, 19
+    X = (rng.standard_normal((K, P)) * 0.1).astype(np.float32)
+    a = OracleEngine(K, P, 0.1, 0.0, 0.0, mode=mode)
+    b = OracleEngine(K, P, 0.1, 0.0, 0.0, mode=mode)
+    a.set_params_all(X)
+    b.set_params_all(X)
+    a.local_sgd_average()
+    b.comm_begin()
+    b.comm_end()
+    np.testing.assert_array_equal(a.x, b.x)
+    # k = 1, mu = wd = 0: average(x - lr g_i) = x - lr * mean(g)
+    g = (rng.standard_normal((K, P)) * 0.01).astype(np.float32)
+    c = OracleEngine(K, P, 0.1, 0.0, 0.0, mode=mode)
+    c.set_params_all(a.x)
+    a.local_step(g)
+    a.local_sgd_average()
+    c.ssgd_step(g)
+    np.testing.assert_allclose(a.x, c.x, rtol=0, atol=1e-15 if mode == "f64" else 5e-8)
