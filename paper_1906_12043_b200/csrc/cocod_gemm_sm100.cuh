@@ -423,25 +423,27 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             if (!landed && p.error_flag != nullptr) atomicExch(p.error_flag, 4);
         } else if (EPI == EPI_F32) {
             if (p.map_c_ok) {
-                // stage the 128 x 128 fp32 tile in the (now idle) ring as four 128 x 32 sub-tiles with the
-                // 128-byte swizzle (16-byte piece j of row r sits at piece j ^ (r & 7)), then bulk-store them
+                // stage the fp32 tile in the (now idle) ring as 128 x 32 sub-tiles with the 128-byte swizzle
+                // (16-byte piece j of row r sits at piece j ^ (r & 7)); each sub-tile is handed to the store
+                // engine as soon as the 128 threads sharing it have written it
+                const int group = warp >> 2;
+                const bool leader = (threadIdx.x & 127) == 0;
 #pragma unroll
                 for (int cc = 0; cc < NCH; ++cc) {
-                    uint8_t *tile = smem + (cbase + cc) * (BM * 128);
+                    const int c = cbase + cc;
+                    uint8_t *tile = smem + c * (BM * 128);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         *reinterpret_cast<uint4 *>(tile + row * 128 + ((j ^ (row & 7)) << 4)) =
                             make_uint4(r[cc][4 * j], r[cc][4 * j + 1], r[cc][4 * j + 2], r[cc][4 * j + 3]);
+                    fence_async_smem();
+                    asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
+                    if (leader && n0 + c * 32 < p.N) {
+                        tma_store_3d(&map_c, smem_base + c * (BM * 128), n0 + c * 32, m0, wk);
+                        tma_store_commit();
+                    }
                 }
-                fence_async_smem();
-                __syncthreads();
-                if (threadIdx.x == 0) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if (n0 + c * 32 < p.N) tma_store_3d(&map_c, smem_base + c * (BM * 128), n0 + c * 32, m0, wk);
-                    tma_store_commit();
-                    tma_store_wait_read<0>();      // shared memory must outlive the reads
-                }
+                if (leader) tma_store_wait_read<0>();      // shared memory must outlive the reads
             } else if (m < p.M) {
                 float *dst = p.c + (long long)wk * p.c_worker_stride + (long long)m * p.ldc + n0;
 #pragma unroll
