@@ -183,6 +183,73 @@ int cocod_profile_get(cocod_handle *h, int i, int *kind, float *start_ms, float 
 int64_t cocod_launch_count(const cocod_handle *h);
 
 /* ---------------------------------------------------------------------------------------------
+ * Workers spread over several GPUs, one process per GPU (the paper's own layout, Section 5.1: one
+ * worker per GPU, models averaged with an all-reduce).  Each process holds a contiguous block of
+ * the K_global workers in an engine of its own; Step II and line 6 stay local, only Step I's
+ * weighted mean x_hat_t = sum_i (M_i / sum_j M_j) x_t^i spans the GPUs.  Every process makes the
+ * same sequence of calls.  Two ways to complete the mean, both queued on the side stream:
+ *
+ *   all-reduce   cocod_comm_begin leaves this GPU's PARTIAL sum (its workers' terms, already
+ *                carrying the global weights) in the average buffer; the caller sums that buffer
+ *                over the processes in place (an all-reduce of P floats queued on the side stream,
+ *                e.g. NCCL), then calls cocod_comm_exchanged.
+ *   gather       after cocod_ipc_attach every GPU can address every GPU's buffers.  The caller
+ *                queues a barrier over the processes on the side stream (all stored copies exist),
+ *                calls cocod_comm_gather -- ONE kernel that reads the K_global stored copies of this
+ *                GPU's share of the columns straight from the GPUs holding them, sums them in
+ *                worker order (the same order as the single-GPU mean, so the result does not depend
+ *                on how the workers are spread) and stores the finished columns into every GPU's
+ *                average buffer -- queues a second barrier (all columns have arrived everywhere)
+ *                and calls cocod_comm_exchanged.
+ *
+ * cocod_comm_end is refused (STATE) until cocod_comm_exchanged has been called in that round.
+ * cocod_local_sgd_average and cocod_ssgd_step are not available on a sharded engine (STATE). */
+
+/* Declare this engine's K workers to be workers first .. first + K - 1 of K_global.  M_global:
+ * host, K_global positive finite mini-batch sizes of ALL workers, or NULL for equal sizes (this
+ * replaces cocod_set_batch_sizes on a sharded engine).  K_global = 0 returns the engine to the
+ * unsharded behaviour.  Errors: INVALID (range outside 0..K_global, K_global > 1024, bad M),
+ * STATE while a communication is in flight or peers are attached. */
+int cocod_set_shard(cocod_handle *h, int K_global, int first, const double *M_global);
+
+/* Device pointer of the average buffer (P floats, engine-owned, valid until cocod_destroy): the
+ * operand of the caller's all-reduce. */
+int cocod_mean_buffer(cocod_handle *h, float **out);
+
+/* The caller has queued, on the side stream given to cocod_comm_begin, everything that completes
+ * the average buffer; the engine marks that point of the side stream as "mean complete".
+ * Errors: STATE unless a communication of a sharded engine is in flight and not yet marked. */
+int cocod_comm_exchanged(cocod_handle *h);
+
+/* Addresses for the gather form.  cocod_ipc_export writes COCOD_IPC_EXPORT_BYTES bytes (host)
+ * describing this engine's buffers (inter-process memory handles of x, the stored copies and the
+ * average buffer, plus K, first, K_global and P for cross-checking).  The caller collects the
+ * blobs of all G processes in rank order (any host transport) and passes them to cocod_ipc_attach
+ * together with its own rank; the engine opens the other processes' buffers (they must be on GPUs
+ * with peer access to this one, or on this one) and builds its address tables.  The blobs must
+ * tile 0..K_global with equal P and K_global (INVALID otherwise; CUDA if a handle cannot be
+ * opened).  G is at most 64.  cocod_ipc_detach closes them again (also done by cocod_destroy);
+ * every process must detach before any process destroys its engine.  Requires cocod_set_shard
+ * first.  Not while a communication is in flight (STATE). */
+#define COCOD_IPC_EXPORT_BYTES 256
+int cocod_ipc_export(cocod_handle *h, void *out);
+int cocod_ipc_attach(cocod_handle *h, int G, int rank, const void *blobs);
+int cocod_ipc_detach(cocod_handle *h);
+
+/* Gather form of Step I's mean (see above): queue the gather kernel on the side stream.  STATE
+ * unless peers are attached and a communication is in flight whose mean has not been started. */
+int cocod_comm_gather(cocod_handle *h);
+
+/* The gather kernel on caller-owned buffers (no handle): rows = device array of K device pointers
+ * (row i = worker i's P stored values, in any allocation this GPU can address), outs = device
+ * array of G device pointers to P-float average buffers; columns [col_lo, col_hi) are averaged
+ * (weights w: device, K floats, or NULL for 1/K) and written to every outs[q].  vec4 != 0 selects the
+ * 128-bit path: the caller vouches that every row and output pointer is 16-byte aligned, and
+ * col_lo, col_hi must be multiples of 4 (INVALID otherwise). */
+int cocod_kernel_mean_gather(const float *const *rows, int K, int64_t col_lo, int64_t col_hi, const float *w,
+                             float *const *outs, int G, int vec4, cocod_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
  * The four kernels on caller-owned device buffers (no handle, no state): the same code the
  * engine launches, exposed for per-kernel measurement and tests.  All pointers: device, fp32.
  *   local_step: n = number of elements; x_out may equal x_in (in place).

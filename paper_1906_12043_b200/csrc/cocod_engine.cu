@@ -21,9 +21,12 @@
 #include <thread>
 #include <vector>
 
+#include <unistd.h>
+
 namespace {
 
 constexpr int kMaxWorkers = 1024;
+constexpr int kMaxRanks = 64;
 constexpr int kMaxProfile = 16384;
 constexpr int64_t kHostChunk = int64_t(1) << 24;   // elements per staged host->device chunk (64 MiB)
 constexpr int kHostSlots = 2;
@@ -56,6 +59,15 @@ struct cocod_engine {
     int snapshot_mode = COCOD_SNAPSHOT_FLIP;
     cudaStream_t compute = nullptr, side = nullptr, copy = nullptr;
     cudaEvent_t ev_snap = nullptr, ev_mean = nullptr, ev_tmp = nullptr;
+    // workers spread over several GPUs (K_global == 0: this engine holds all workers)
+    int K_global = 0, first = 0;
+    float *wg = nullptr;                // weights of all K_global workers (device), when batch sizes differ
+    bool mean_started = false;          // this round's kernel that fills the average buffer has been queued
+    bool exchanged = false;             // ... and the caller has marked the buffer complete
+    int G = 0, rank = 0;                // attached peers (G == 0: none)
+    void *opened[kMaxRanks][3] = {};    // peer buffers opened through inter-process handles (to be closed)
+    const float **rows_tab[2] = {nullptr, nullptr};   // device: row pointers of all K_global workers in buf[0] / buf[1]
+    float **outs_tab = nullptr;         // device: every GPU's average buffer
     // staging for host gradients
     float *stage[kHostSlots] = {nullptr, nullptr};
     cudaEvent_t ev_copied[kHostSlots] = {nullptr, nullptr}, ev_consumed[kHostSlots] = {nullptr, nullptr};
@@ -140,11 +152,11 @@ cudaError_t launch_snapshot(const float *x, float *snap, int64_t n, cudaStream_t
     return cudaGetLastError();
 }
 
-cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, float *mean, cudaStream_t s,
-                        int *n_launch)
+// inv_k: factor of the unweighted sum (1/K; 1/K_global for a partial sum over this GPU's workers)
+cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, float *mean, float inv_k,
+                        cudaStream_t s, int *n_launch)
 {
     using namespace cocod;
-    const float inv_k = 1.0f / (float)K;
     if (K <= 4 && (P % 8) == 0 && aligned32(snap) && aligned32(mean)) {
         const unsigned grid = grid_for(P / 8, kThreads);
         if (K <= 2) mean_vec8<2><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
@@ -155,6 +167,25 @@ cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, flo
             reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k);
     } else {
         mean_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
+    }
+    if (n_launch) ++*n_launch;
+    return cudaGetLastError();
+}
+
+// Average of columns [lo, hi) over rows held in separate allocations, written to G buffers.  vec4: the
+// caller vouches that all row and output pointers are 16-byte aligned and lo, hi are multiples of 4.
+cudaError_t launch_mean_gather(const float *const *rows, int K, int64_t lo, int64_t hi, const float *w,
+                               float *const *outs, int G, float inv_k, bool vec4, cudaStream_t s, int *n_launch)
+{
+    using namespace cocod;
+    if (hi <= lo) return cudaSuccess;
+    if (vec4) {
+        const int64_t c_lo = lo / 4, c_hi = hi / 4;
+        mean_gather_vec4<<<grid_for(c_hi - c_lo, kThreads), kThreads, 0, s>>>(
+            reinterpret_cast<const float4 *const *>(rows), K, c_lo, c_hi, w,
+            reinterpret_cast<float4 *const *>(outs), G, inv_k);
+    } else {
+        mean_gather_scalar<<<grid_for(hi - lo, kThreads), kThreads, 0, s>>>(rows, K, lo, hi, w, outs, G, inv_k);
     }
     if (n_launch) ++*n_launch;
     return cudaGetLastError();
@@ -224,9 +255,35 @@ int check_live(const cocod_engine *h)
     return COCOD_OK;
 }
 
+// Weights and scale of Step I's kernel: the whole mean, or this GPU's part of it with the global weights.
+inline const float *mean_weights(const cocod_engine *h)
+{
+    if (h->K_global > 0) return h->wg ? h->wg + h->first : nullptr;
+    return h->weighted ? h->w : nullptr;
+}
+inline float mean_scale(const cocod_engine *h)
+{
+    return 1.0f / (float)(h->K_global > 0 ? h->K_global : h->K);
+}
+
+void detach_peers(cocod_engine *h)
+{
+    for (int q = 0; q < kMaxRanks; ++q)
+        for (int b = 0; b < 3; ++b)
+            if (h->opened[q][b]) { cudaIpcCloseMemHandle(h->opened[q][b]); h->opened[q][b] = nullptr; }
+    for (int b = 0; b < 2; ++b)
+        if (h->rows_tab[b]) { cudaFree((void *)h->rows_tab[b]); h->rows_tab[b] = nullptr; }
+    if (h->outs_tab) { cudaFree((void *)h->outs_tab); h->outs_tab = nullptr; }
+    h->G = 0;
+    h->rank = 0;
+    cudaGetLastError();
+}
+
 void free_all(cocod_engine *h)
 {
     profile_clear(h);
+    detach_peers(h);
+    if (h->wg) cudaFree(h->wg);
     for (int i = 0; i < 2; ++i) if (h->buf[i]) cudaFree(h->buf[i]);
     if (h->v) cudaFree(h->v);
     if (h->mean) cudaFree(h->mean);
@@ -290,6 +347,17 @@ int step_range(cocod_engine *h, const float *g, int64_t off, int64_t len)
                                 h->shadow ? h->shadow + off : nullptr, h->compute, &nl));
     }
     h->launches += nl;
+    return COCOD_OK;
+}
+
+// The side stream's work so far completes the average buffer.
+int mark_mean_complete(cocod_engine *h)
+{
+    CK(h, cudaEventRecord(h->ev_mean, h->side));
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    CK(h, cudaStreamIsCapturing(h->side, &cap));
+    h->mean_captured = (cap != cudaStreamCaptureStatusNone);      // a captured event cannot be waited on later
+    h->mean_valid = true;
     return COCOD_OK;
 }
 
@@ -420,25 +488,63 @@ int cocod_comm_begin(cocod_handle *h, cocod_stream_t side)
         CK(h, cudaEventRecord(h->ev_snap, h->compute));
         CK(h, cudaStreamWaitEvent(h->side, h->ev_snap, 0));
     }
+    h->mean_started = false;
+    h->exchanged = false;
+    if (h->G > 0) {                 // gather form: the caller queues a barrier, then cocod_comm_gather
+        h->mean_valid = false;
+        h->state = IN_FLIGHT;
+        return COCOD_OK;
+    }
     int nl = 0;
     {
         Bracket br(h, h->side, COCOD_KERNEL_MEAN);
-        CK(h, launch_mean(h->snap, h->K, h->P, h->weighted ? h->w : nullptr, h->mean, h->side, &nl));
+        CK(h, launch_mean(h->snap, h->K, h->P, mean_weights(h), h->mean, mean_scale(h), h->side, &nl));
     }
     h->launches += nl;
-    CK(h, cudaEventRecord(h->ev_mean, h->side));
-    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-    CK(h, cudaStreamIsCapturing(h->side, &cap));
-    h->mean_captured = (cap != cudaStreamCaptureStatusNone);      // a captured event cannot be waited on later
-    h->mean_valid = true;
+    h->mean_started = true;
     h->state = IN_FLIGHT;
+    if (h->K_global > 0) {          // partial sum: complete only after the caller's all-reduce
+        h->mean_valid = false;
+        return COCOD_OK;
+    }
+    return mark_mean_complete(h);
+}
+
+int cocod_comm_gather(cocod_handle *h)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IN_FLIGHT || h->G == 0 || h->mean_started) return COCOD_ERR_STATE;
+    // this GPU's share of the columns (in float4 units when every row is 16-byte aligned)
+    const bool vec4 = (h->P % 4) == 0;
+    const int64_t units = vec4 ? h->P / 4 : h->P;
+    const int64_t base = units / h->G, rem = units % h->G;
+    const int64_t lo = h->rank * base + std::min<int64_t>(h->rank, rem);
+    const int64_t hi = lo + base + (h->rank < rem ? 1 : 0);
+    const int b = (h->snap == h->buf[0]) ? 0 : 1;
+    int nl = 0;
+    {
+        Bracket br(h, h->side, COCOD_KERNEL_MEAN);
+        CK(h, launch_mean_gather(h->rows_tab[b], h->K_global, vec4 ? lo * 4 : lo, vec4 ? hi * 4 : hi, h->wg,
+                                 h->outs_tab, h->G, mean_scale(h), vec4, h->side, &nl));
+    }
+    h->launches += nl;
+    h->mean_started = true;
     return COCOD_OK;
+}
+
+int cocod_comm_exchanged(cocod_handle *h)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IN_FLIGHT || h->K_global == 0 || !h->mean_started || h->exchanged) return COCOD_ERR_STATE;
+    h->exchanged = true;
+    return mark_mean_complete(h);
 }
 
 int cocod_comm_end(cocod_handle *h)
 {
     if (int rc = check_live(h)) return rc;
     if (h->state != IN_FLIGHT) return COCOD_ERR_STATE;
+    if (h->K_global > 0 && !h->exchanged) return COCOD_ERR_STATE;      // the mean over the GPUs is not complete
     if (h->side != h->compute) CK(h, cudaStreamWaitEvent(h->compute, h->ev_mean, 0));
     int nl = 0;
     {
@@ -456,11 +562,12 @@ int cocod_comm_end(cocod_handle *h)
 int cocod_local_sgd_average(cocod_handle *h)
 {
     if (int rc = check_live(h)) return rc;
-    if (h->state != IDLE) return COCOD_ERR_STATE;
+    if (h->state != IDLE || h->K_global > 0) return COCOD_ERR_STATE;
     int nl = 0;
     {
         Bracket br(h, h->compute, COCOD_KERNEL_MEAN);
-        CK(h, launch_mean(h->buf[h->cur], h->K, h->P, h->weighted ? h->w : nullptr, h->mean, h->compute, &nl));
+        CK(h, launch_mean(h->buf[h->cur], h->K, h->P, h->weighted ? h->w : nullptr, h->mean, 1.0f / (float)h->K,
+                          h->compute, &nl));
     }
     // after the sequential mean nothing from the side stream is pending for this value
     CK(h, cudaEventRecord(h->ev_mean, h->compute));
@@ -480,12 +587,13 @@ int cocod_ssgd_step(cocod_handle *h, const float *grads)
 {
     if (int rc = check_live(h)) return rc;
     if (!grads) return COCOD_ERR_INVALID;
-    if (h->state != IDLE) return COCOD_ERR_STATE;      // the average-model buffer holds the averaged gradient
+    if (h->state != IDLE || h->K_global > 0) return COCOD_ERR_STATE;   // the average buffer holds the averaged gradient
     using namespace cocod;
     int nl = 0;
     {
         Bracket br(h, h->compute, COCOD_KERNEL_MEAN);
-        CK(h, launch_mean(grads, h->K, h->P, h->weighted ? h->w : nullptr, h->mean, h->compute, &nl));
+        CK(h, launch_mean(grads, h->K, h->P, h->weighted ? h->w : nullptr, h->mean, 1.0f / (float)h->K, h->compute,
+                          &nl));
     }
     h->mean_valid = false;                              // it is a gradient now, not an average model
     float *x = h->buf[h->cur];
@@ -589,7 +697,7 @@ int cocod_set_lr(cocod_handle *h, float lr)
 int cocod_set_batch_sizes(cocod_handle *h, const double *M)
 {
     if (int rc = check_live(h)) return rc;
-    if (h->state != IDLE) return COCOD_ERR_STATE;
+    if (h->state != IDLE || h->K_global > 0) return COCOD_ERR_STATE;      // sharded: cocod_set_shard carries them
     if (!M) { h->weighted = false; return COCOD_OK; }
     double sum = 0.0;
     for (int i = 0; i < h->K; ++i) {
@@ -646,7 +754,7 @@ int cocod_sync(cocod_handle *h)
 int cocod_comm_wait(cocod_handle *h, int timeout_ms)
 {
     if (int rc = check_live(h)) return rc;
-    if (h->state != IN_FLIGHT) return COCOD_ERR_STATE;
+    if (h->state != IN_FLIGHT || (h->K_global > 0 && !h->exchanged)) return COCOD_ERR_STATE;
     const auto t0 = std::chrono::steady_clock::now();
     for (;;) {
         cudaError_t e = cudaEventQuery(h->ev_mean);
@@ -715,6 +823,164 @@ int cocod_profile_get(cocod_handle *h, int i, int *kind, float *start_ms, float 
     return COCOD_OK;
 }
 
+// ------------------------------------------------------------------ workers spread over several GPUs
+int cocod_set_shard(cocod_handle *h, int K_global, int first, const double *M_global)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IDLE || h->G > 0) return COCOD_ERR_STATE;
+    if (K_global == 0) {
+        h->K_global = 0; h->first = 0;
+        if (h->wg) { CK(h, cudaStreamSynchronize(h->compute)); cudaFree(h->wg); h->wg = nullptr; }
+        return COCOD_OK;
+    }
+    if (K_global < h->K || K_global > kMaxWorkers || first < 0 || first > K_global - h->K) return COCOD_ERR_INVALID;
+    float *wg = nullptr;
+    if (M_global) {
+        double sum = 0.0;
+        for (int i = 0; i < K_global; ++i) {
+            if (!(M_global[i] > 0.0) || !std::isfinite(M_global[i])) return COCOD_ERR_INVALID;
+            sum += M_global[i];
+        }
+        float w[kMaxWorkers];
+        for (int i = 0; i < K_global; ++i) w[i] = (float)(M_global[i] / sum);
+        if (cudaMalloc((void **)&wg, (size_t)K_global * sizeof(float)) != cudaSuccess) {
+            cudaGetLastError();
+            return COCOD_ERR_OOM;
+        }
+        cudaError_t e = cudaMemcpyAsync(wg, w, (size_t)K_global * sizeof(float), cudaMemcpyHostToDevice, h->compute);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(h->compute);      // w[] is a stack buffer
+        if (e != cudaSuccess) { cudaFree(wg); fail(h, e); return COCOD_ERR_CUDA; }
+    }
+    if (h->wg) { CK(h, cudaStreamSynchronize(h->compute)); cudaFree(h->wg); }
+    h->wg = wg;
+    h->K_global = K_global;
+    h->first = first;
+    return COCOD_OK;
+}
+
+int cocod_mean_buffer(cocod_handle *h, float **out)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!out) return COCOD_ERR_INVALID;
+    *out = h->mean;
+    return COCOD_OK;
+}
+
+namespace {
+// What one process tells the others about its engine (COCOD_IPC_EXPORT_BYTES bytes on the wire).
+struct IpcBlob {
+    uint32_t magic;
+    int32_t K, first, K_global, cur, pid;
+    int64_t P;
+    uint64_t ptr[3];                    // buf[0], buf[1], average buffer: usable as they are inside process `pid`
+    cudaIpcMemHandle_t mem[3];          // the same three for other processes
+};
+static_assert(sizeof(IpcBlob) <= COCOD_IPC_EXPORT_BYTES, "export blob too large");
+constexpr uint32_t kIpcMagic = 0xC0C0D5D1u;
+}  // namespace
+
+int cocod_ipc_export(cocod_handle *h, void *out)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!out) return COCOD_ERR_INVALID;
+    if (h->K_global == 0) return COCOD_ERR_STATE;
+    IpcBlob b{};
+    b.magic = kIpcMagic;
+    b.K = h->K; b.first = h->first; b.K_global = h->K_global; b.cur = h->cur; b.pid = (int32_t)getpid();
+    b.P = h->P;
+    float *ptrs[3] = {h->buf[0], h->buf[1], h->mean};
+    for (int i = 0; i < 3; ++i) {
+        b.ptr[i] = (uint64_t)reinterpret_cast<uintptr_t>(ptrs[i]);
+        CK(h, cudaIpcGetMemHandle(&b.mem[i], ptrs[i]));
+    }
+    std::memset(out, 0, COCOD_IPC_EXPORT_BYTES);
+    std::memcpy(out, &b, sizeof(b));
+    return COCOD_OK;
+}
+
+int cocod_ipc_attach(cocod_handle *h, int G, int rank, const void *blobs)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!blobs || G < 1 || G > kMaxRanks || rank < 0 || rank >= G) return COCOD_ERR_INVALID;
+    if (h->state != IDLE || h->K_global == 0 || h->G > 0) return COCOD_ERR_STATE;
+    std::vector<IpcBlob> all((size_t)G);
+    int next = 0;
+    for (int q = 0; q < G; ++q) {
+        std::memcpy(&all[q], (const unsigned char *)blobs + (size_t)q * COCOD_IPC_EXPORT_BYTES, sizeof(IpcBlob));
+        const IpcBlob &b = all[q];
+        if (b.magic != kIpcMagic || b.P != h->P || b.K_global != h->K_global || b.K < 1 || b.first != next ||
+            b.cur != h->cur)
+            return COCOD_ERR_INVALID;
+        next += b.K;
+    }
+    if (next != h->K_global || all[rank].K != h->K || all[rank].first != h->first ||
+        all[rank].ptr[0] != (uint64_t)reinterpret_cast<uintptr_t>(h->buf[0]) || all[rank].pid != (int32_t)getpid())
+        return COCOD_ERR_INVALID;
+    // addresses of every process's three buffers as seen from here
+    std::vector<float *> base((size_t)G * 3, nullptr);
+    for (int q = 0; q < G; ++q)
+        for (int i = 0; i < 3; ++i) {
+            if (all[q].pid == (int32_t)getpid()) {      // same process (also this engine itself): same address space
+                base[(size_t)q * 3 + i] = reinterpret_cast<float *>((uintptr_t)all[q].ptr[i]);
+                continue;
+            }
+            void *p = nullptr;
+            cudaError_t e = cudaIpcOpenMemHandle(&p, all[q].mem[i], cudaIpcMemLazyEnablePeerAccess);
+            if (e != cudaSuccess) { fail(h, e); cudaGetLastError(); detach_peers(h); return COCOD_ERR_CUDA; }
+            h->opened[q][i] = p;
+            base[(size_t)q * 3 + i] = static_cast<float *>(p);
+        }
+    std::vector<const float *> rows[2];
+    std::vector<float *> outs((size_t)G);
+    for (int b = 0; b < 2; ++b) rows[b].resize((size_t)h->K_global);
+    for (int q = 0; q < G; ++q) {
+        for (int r = 0; r < all[q].K; ++r)
+            for (int b = 0; b < 2; ++b) rows[b][(size_t)all[q].first + r] = base[(size_t)q * 3 + b] + (int64_t)r * h->P;
+        outs[q] = base[(size_t)q * 3 + 2];
+    }
+    cudaError_t e = cudaSuccess;
+    for (int b = 0; b < 2 && e == cudaSuccess; ++b) {
+        e = cudaMalloc((void **)&h->rows_tab[b], (size_t)h->K_global * sizeof(float *));
+        if (e == cudaSuccess)
+            e = cudaMemcpy((void *)h->rows_tab[b], rows[b].data(), (size_t)h->K_global * sizeof(float *),
+                           cudaMemcpyHostToDevice);
+    }
+    if (e == cudaSuccess) e = cudaMalloc((void **)&h->outs_tab, (size_t)G * sizeof(float *));
+    if (e == cudaSuccess) e = cudaMemcpy((void *)h->outs_tab, outs.data(), (size_t)G * sizeof(float *), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        const bool oom = (e == cudaErrorMemoryAllocation);
+        cudaGetLastError();
+        detach_peers(h);
+        if (oom) return COCOD_ERR_OOM;
+        fail(h, e);
+        return COCOD_ERR_CUDA;
+    }
+    h->G = G;
+    h->rank = rank;
+    return COCOD_OK;
+}
+
+int cocod_ipc_detach(cocod_handle *h)
+{
+    if (int rc = check_live(h)) return rc;
+    if (h->state != IDLE) return COCOD_ERR_STATE;
+    // peers may still be reading this GPU's buffers only until their own side streams are done; what
+    // this engine itself queued must be done before its mappings go away
+    CK(h, cudaStreamSynchronize(h->compute));
+    if (!h->mean_captured) CK(h, cudaEventSynchronize(h->ev_mean));
+    detach_peers(h);
+    return COCOD_OK;
+}
+
+int cocod_kernel_mean_gather(const float *const *rows, int K, int64_t col_lo, int64_t col_hi, const float *w,
+                             float *const *outs, int G, int vec4, cocod_stream_t stream)
+{
+    if (!rows || !outs || K < 1 || G < 1 || col_lo < 0 || col_hi < col_lo) return COCOD_ERR_INVALID;
+    if (vec4 && ((col_lo | col_hi) & 3)) return COCOD_ERR_INVALID;
+    return launch_mean_gather(rows, K, col_lo, col_hi, w, outs, G, 1.0f / (float)K, vec4 != 0, (cudaStream_t)stream,
+                              nullptr) == cudaSuccess ? COCOD_OK : COCOD_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------ stateless kernel entry points
 int cocod_kernel_local_step(const float *x_in, float *x_out, float *v, const float *g, int64_t n,
                             float lr, float mu, float wd, cocod_stream_t stream)
@@ -733,7 +999,8 @@ int cocod_kernel_snapshot(const float *x, float *snap, int64_t n, cocod_stream_t
 int cocod_kernel_mean(const float *snap, int K, int64_t P, const float *w, float *mean, cocod_stream_t stream)
 {
     if (!snap || !mean || K < 1 || P < 1) return COCOD_ERR_INVALID;
-    return launch_mean(snap, K, P, w, mean, (cudaStream_t)stream, nullptr) == cudaSuccess ? COCOD_OK : COCOD_ERR_CUDA;
+    return launch_mean(snap, K, P, w, mean, 1.0f / (float)K, (cudaStream_t)stream, nullptr) == cudaSuccess
+               ? COCOD_OK : COCOD_ERR_CUDA;
 }
 
 int cocod_kernel_merge(float *x, const float *snap, const float *mean, int K, int64_t P, cocod_stream_t stream)

@@ -304,6 +304,40 @@ mean_scalar(const float *__restrict__ snap, int K, int64_t P, const float *__res
     mean[p] = s[0];
 }
 
+// ------------------------------------------------------------------------------------------ average model over GPUs
+// Workers spread over several GPUs: row i of the stored copies is wherever rows[i] points (this GPU's
+// memory or a peer's, read over NVLink with ordinary loads), and the finished columns go to every
+// GPU's average buffer outs[0..G) with ordinary stores.  Each GPU runs this over its own share of the
+// columns [c_lo, c_hi), so every remote value crosses the link once.  Rows are summed in worker order
+// by the same mean_rows as above: the result is bit-identical to the single-GPU mean however the
+// workers are spread.  No waiting inside the kernel: the callers order it after "all stored copies
+// exist" and order the merges after "all GPUs' kernels are done" on the stream.
+static __global__ void __launch_bounds__(kThreads)
+mean_gather_vec4(const float4 *const *__restrict__ rows, int K, int64_t c_lo, int64_t c_hi,
+                 const float *__restrict__ w, float4 *const *__restrict__ outs, int G, float inv_k)
+{
+    const int64_t c = c_lo + (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= c_hi) return;
+    float s[4];
+    mean_rows<4, 8>(s, K, w, inv_k, [&](int i, float (&v)[4]) {
+        const float4 t = __ldcg(rows[i] + c);      // L2 only: each value is read once
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    });
+    const float4 o = make_float4(s[0], s[1], s[2], s[3]);
+    for (int q = 0; q < G; ++q) outs[q][c] = o;
+}
+
+static __global__ void __launch_bounds__(kThreads)
+mean_gather_scalar(const float *const *__restrict__ rows, int K, int64_t p_lo, int64_t p_hi,
+                   const float *__restrict__ w, float *const *__restrict__ outs, int G, float inv_k)
+{
+    const int64_t p = p_lo + (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (p >= p_hi) return;
+    float s[1];
+    mean_rows<1, 8>(s, K, w, inv_k, [&](int i, float (&v)[1]) { v[0] = __ldcg(rows[i] + p); });
+    for (int q = 0; q < G; ++q) outs[q][p] = s[0];
+}
+
 // ------------------------------------------------------------------------------------------ merge (line 6)
 // Same column ownership: the average is read once per column (4/K B per worker-parameter) and
 // reused for all K rows; RC rows (2 * RC loads) in flight per thread.  x may alias snap (a

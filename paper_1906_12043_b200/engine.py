@@ -14,6 +14,7 @@ LIB_PATH = os.path.join(_HERE, "libcocod.so")
 
 OK, ERR_INVALID, ERR_OOM, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
 NOALLOC_MAX_ELEMS = 4 * 1024 * 1024
+IPC_EXPORT_BYTES = 256
 OPT_SNAPSHOT, OPT_PROFILE, OPT_BF16_SHADOW = 1, 2, 3
 SNAPSHOT_COPY, SNAPSHOT_FLIP = 0, 1
 KERNEL_LOCAL_STEP, KERNEL_SNAPSHOT, KERNEL_MEAN, KERNEL_MERGE = 0, 1, 2, 3
@@ -51,6 +52,14 @@ SIGNATURES = {
     "cocod_profile_count": (_i, [_vp]),
     "cocod_profile_get": (_i, [_vp, _i, ctypes.POINTER(_i), ctypes.POINTER(_f), ctypes.POINTER(_f)]),
     "cocod_launch_count": (_i64, [_vp]),
+    "cocod_set_shard": (_i, [_vp, _i, _i, ctypes.POINTER(ctypes.c_double)]),
+    "cocod_mean_buffer": (_i, [_vp, ctypes.POINTER(_vp)]),
+    "cocod_comm_exchanged": (_i, [_vp]),
+    "cocod_ipc_export": (_i, [_vp, _vp]),
+    "cocod_ipc_attach": (_i, [_vp, _i, _i, _vp]),
+    "cocod_ipc_detach": (_i, [_vp]),
+    "cocod_comm_gather": (_i, [_vp]),
+    "cocod_kernel_mean_gather": (_i, [_vp, _i, _i64, _i64, _vp, _vp, _i, _i, _vp]),
     "cocod_kernel_local_step": (_i, [_vp, _vp, _vp, _vp, _i64, _f, _f, _f, _vp]),
     "cocod_kernel_snapshot": (_i, [_vp, _vp, _i64, _vp]),
     "cocod_kernel_mean": (_i, [_vp, _i, _i64, _vp, _vp, _vp]),
@@ -249,6 +258,46 @@ class Engine:
         arr = (ctypes.c_double * self.K)(*[float(m) for m in M])
         self._ck(self._lib.cocod_set_batch_sizes(self._h, arr), "cocod_set_batch_sizes")
 
+    # -- workers spread over several GPUs (one engine per process)
+    def set_shard(self, K_global: int, first: int, M_global=None):
+        """This engine's K workers are workers first .. first+K-1 of K_global; M_global: the
+        mini-batch sizes of ALL workers (None = equal).  K_global = 0 undoes it."""
+        arr = None
+        if M_global is not None:
+            if len(M_global) != K_global:
+                raise ValueError("need K_global batch sizes")
+            arr = (ctypes.c_double * K_global)(*[float(m) for m in M_global])
+        self._ck(self._lib.cocod_set_shard(self._h, int(K_global), int(first), arr), "cocod_set_shard")
+
+    def mean_buffer(self):
+        """The engine's average buffer as a torch CUDA tensor of P floats (a view, no copy): the
+        operand of the caller's all-reduce."""
+        import torch
+        ptr = _vp()
+        self._ck(self._lib.cocod_mean_buffer(self._h, ctypes.byref(ptr)), "cocod_mean_buffer")
+        return _device_view(ptr.value, (self.P,), torch.float32)
+
+    def comm_exchanged(self):
+        self._ck(self._lib.cocod_comm_exchanged(self._h), "cocod_comm_exchanged")
+
+    def ipc_export(self) -> bytes:
+        buf = ctypes.create_string_buffer(IPC_EXPORT_BYTES)
+        self._ck(self._lib.cocod_ipc_export(self._h, buf), "cocod_ipc_export")
+        return buf.raw
+
+    def ipc_attach(self, rank: int, blobs):
+        """blobs: the ipc_export() bytes of all processes in rank order."""
+        if any(len(b) != IPC_EXPORT_BYTES for b in blobs):
+            raise ValueError("every blob must be IPC_EXPORT_BYTES long")
+        raw = ctypes.create_string_buffer(b"".join(blobs), IPC_EXPORT_BYTES * len(blobs))
+        self._ck(self._lib.cocod_ipc_attach(self._h, len(blobs), int(rank), raw), "cocod_ipc_attach")
+
+    def ipc_detach(self):
+        self._ck(self._lib.cocod_ipc_detach(self._h), "cocod_ipc_detach")
+
+    def comm_gather(self):
+        self._ck(self._lib.cocod_comm_gather(self._h), "cocod_comm_gather")
+
     def set_option(self, option: int, value: int):
         self._ck(self._lib.cocod_set_option(self._h, option, value), "cocod_set_option")
 
@@ -312,6 +361,15 @@ def kernel_mean(snap, mean, w=None, stream=None):
     K, P = snap.shape
     s = _stream(stream) if stream is not None else torch.cuda.current_stream().cuda_stream
     _ck_rc(load().cocod_kernel_mean(_ptr(snap), K, P, _ptr(w), _ptr(mean), s), "cocod_kernel_mean")
+
+
+def kernel_mean_gather(rows, col_lo, col_hi, outs, w=None, vec4=True, stream=None):
+    """rows: int64 CUDA tensor of K device addresses (one per worker's P stored values); outs: int64
+    CUDA tensor of G device addresses of P-float average buffers."""
+    import torch
+    s = _stream(stream) if stream is not None else torch.cuda.current_stream().cuda_stream
+    _ck_rc(load().cocod_kernel_mean_gather(_ptr(rows), rows.numel(), int(col_lo), int(col_hi), _ptr(w), _ptr(outs),
+                                           outs.numel(), 1 if vec4 else 0, s), "cocod_kernel_mean_gather")
 
 
 def kernel_merge(x, snap, mean, stream=None):
