@@ -45,6 +45,12 @@ def parse():
                     help="replay the timed rounds from a CUDA graph of two rounds (launch-bound workloads)")
     ap.add_argument("--fused", action="store_true",
                     help="mlp workload: gradients and local step in one call (update inside the weight-gradient GEMMs)")
+    ap.add_argument("--shard", default="columns", choices=["columns", "workers"],
+                    help="N > 1: split the columns (default, no exchange) or the workers (the paper's layout: "
+                         "every rank holds K workers of K*N, Step I's mean spans the GPUs on the side stream)")
+    ap.add_argument("--exchange", default="allreduce", choices=["allreduce", "gather"],
+                    help="--shard workers: finish the mean with an all-reduce of P floats, or with the gather kernel "
+                         "over peer addresses")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample-cols", type=int, default=1 << 20)
@@ -654,6 +660,120 @@ def run_mlp(args):
     mg.destroy()
 
 
+# ---------------------------------------------------------------------------------------------- workers over GPUs
+def run_worker_sharded(args, wl):
+    """Every rank holds wl.K workers of K_global = wl.K * N (weak scaling in the workers, the paper's
+    layout).  Step II and the merge are local; Step I's mean over all K_global workers is completed on
+    the side stream by an all-reduce of P floats or by the gather kernel."""
+    import socket
+    import torch
+    import torch.distributed as dist
+    from paper_1906_12043_b200 import build, engine as E, inputs as I, workloads as W
+    from paper_1906_12043_b200.sharded import WorkerShardedEngine
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the engine has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if "MASTER_ADDR" not in os.environ:                 # plain `python bench.py`: a group of one
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(sk.getsockname()[1]))
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build()
+    dist.barrier()
+    E.load()
+    K, P, k = wl.K, wl.P, wl.k
+    K_global = K * world
+    hbm_peak, peak_kind = 6650.0, "fallback"
+    try:
+        hbm_peak, peak_kind = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["hbm_gbs"]), "measured"
+    except (OSError, KeyError):
+        pass
+    eng = WorkerShardedEngine(K_global, P, wl.lr, wl.mu, wl.wd, exchange=args.exchange, sync="stream")
+    x0 = torch.empty(P, dtype=torch.float32, device="cuda")
+    I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, 0, wl.sigma_x0)
+    eng.set_params(x0)
+    ring = []
+    for t in range(max(1, args.ring)):
+        g = torch.empty((K, P), dtype=torch.float32, device="cuda")
+        I.device_gradients_into(g, t, wl.sigma_g, first_worker=eng.first)
+        ring.append(g)
+    side = torch.cuda.Stream(priority=-1)
+    compute = torch.cuda.current_stream()
+    step_no = [0]
+
+    def one_round():
+        eng.comm_begin(side)
+        for _ in range(k):
+            eng.local_step(ring[step_no[0] % len(ring)])
+            step_no[0] += 1
+        eng.comm_end()
+
+    def barrier():
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        one_round()
+    eng.engine.set_option(E.OPT_PROFILE, 1)
+    eng.engine.profile_reset()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    launches0 = eng.engine.launch_count
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(compute)
+    for _ in range(args.steps):
+        one_round()
+    ev1.record(compute)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    launches = eng.engine.launch_count - launches0
+    by = summarize_profile(eng.engine.profile_records(), E.KERNEL_NAMES)
+    eng.engine.set_option(E.OPT_PROFILE, 0)
+    # what one GPU's mean kernel moves: its K stored copies -> P partial sums, or K_global rows of its
+    # share of the columns -> that share in every GPU's buffer
+    mean_bytes = (4 * K * P + 4 * P) if args.exchange == "allreduce" else (4 * K_global * P / world + 4 * P)
+    alg_bytes = {"local_step": W.BYTES_LOCAL_STEP * K * P, "mean": mean_bytes, "merge": W.bytes_merge(K) * K * P}
+    table = {}
+    for name, iv in by.items():
+        avg_ms = sum(b - a for a, b in iv) / len(iv)
+        gbs = alg_bytes[name] / (avg_ms * 1e-3) / 1e9
+        table[name] = {"launches": len(iv), "avg_ms": round(avg_ms, 5), "gbs": round(gbs, 1),
+                       "frac_of_peak": round(gbs / hbm_peak, 4)}
+    dom = table.get("local_step", {})
+    if rank == 0:
+        if world == 1:
+            link_bytes = 0
+        elif args.exchange == "allreduce":
+            link_bytes = 8 * P * (world - 1) / world
+        else:
+            link_bytes = 4 * P * (K_global - K) / world + 4 * P * (world - 1) / world
+        print(json.dumps({
+            "metric": METRIC, "value": world * K * P * k * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "K": K, "K_global": K_global, "P": P, "k": k, "lr": wl.lr, "mu": wl.mu,
+                       "wd": wl.wd, "snapshot": "flip", "gradient_ring": len(ring),
+                       "sharding": f"workers ({K} per GPU), mean over GPUs by {args.exchange} on the side stream",
+                       "l2": "inputs larger than L2" if K * P * 4 > 126e6 else "L2-resident workload: not an HBM number"},
+            "clocks": clocks, "e2e": None, "gpu_launches": launches,
+            "roofline": {"bound": "hbm", "kernel": "local_step", "achieved": dom.get("gbs"), "peak": hbm_peak,
+                         "unit": "GB/s", "frac": dom.get("frac_of_peak"), "traffic": None, "peak_kind": peak_kind,
+                         "algorithmic_bytes_per_launch": alg_bytes["local_step"], "avg_launch_ms": dom.get("avg_ms")},
+            "cpu_baseline": None, "kernels_in_loop": table, "overlap_fraction": overlap_fraction(by),
+            "link_bytes_per_round_per_gpu": link_bytes,
+        }))
+    eng.close()
+    dist.destroy_process_group()
+
+
 def run_sweep(args):
     """Timing-only sweep over (P, K, k).  Values do not affect timing, so each cell reuses one
     generated gradient buffer.  Cells whose four K x P buffers exceed 160 GB are skipped."""
@@ -738,6 +858,8 @@ def main():
         wl = replace(wl, name=wl.name + "-custom", K=args.K or wl.K, P=args.P or wl.P, k=args.k or wl.k)
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.shard == "workers":
+        run_worker_sharded(args, wl)
     else:
         run_ours(args, wl)
 

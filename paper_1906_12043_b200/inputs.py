@@ -223,12 +223,12 @@ def device_gaussian_into(out, seed: int, stream: int, worker: int, step: int, p0
 
 
 def device_gradients_into(g, step: int, sigma: float = 0.01, seed: int = GRAD_SEED,
-                          p0: int = 0) -> None:
+                          p0: int = 0, first_worker: int = 0) -> None:
     """Fill a K x P float32 CUDA tensor with the gradients of local step ``step``
-    (columns p0 .. p0+P-1 of the global vector)."""
+    (columns p0 .. p0+P-1 of the global vector, workers first_worker .. first_worker+K-1)."""
     K = g.shape[0]
     for w in range(K):
-        device_gaussian_into(g[w], seed, STREAM_GRAD, w, step, p0, sigma)
+        device_gaussian_into(g[w], seed, STREAM_GRAD, first_worker + w, step, p0, sigma)
 
 
 # ----------------------------------------------------------------------------- synthetic MLP workload
