@@ -144,6 +144,17 @@ template <int N> __device__ __forceinline__ void tma_store_wait_read()
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Programmatic dependent launch.  A kernel launched with the programmatic-serialization attribute may
+// become resident while its predecessor in the stream still runs; it must not touch anything the
+// predecessor (or, transitively, anything before it) writes until pdl_wait() has returned, which
+// happens once the predecessor grid has completed and its writes are visible.
+// pdl_launch_dependents() lets the successor's CTAs be scheduled as soon as every CTA of this grid has
+// called it (or exited): call it only after this CTA holds all the resources it will ever take
+// (shared memory, TMEM), so that a waiting successor can never hold something a CTA of this grid
+// still needs.  Both are no-ops for kernels launched without the attribute.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols)
 {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
@@ -273,6 +284,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         abort[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
+        pdl_wait();                   // everything above overlapped the previous kernel's tail
         // the first ring of copies starts now, under the rest of the set-up
         if (!p.debug_no_loads)
             for (; armed < nkb && armed < stages; ++armed) issue_loads(armed, armed);
@@ -296,6 +308,8 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     if (threadIdx.x == 0) COCOD_TRACE(1);
+    pdl_launch_dependents();          // this CTA holds its shared memory and TMEM: the next kernel may set up
+    pdl_wait();                       // (thread 0 has passed it already) before any thread reads global memory
 
     int failed = 0;
     constexpr int NCH = (NT == 256) ? 2 : 4;       // 32-column chunks drained by one thread

@@ -87,9 +87,25 @@ bool map_out(CUtensorMap *m, float *base, uint64_t cols, uint64_t rows, uint64_t
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Launch with the programmatic-serialization attribute: the kernel may become resident (and run the
+// part of its prologue that precedes pdl_wait()) while the previous kernel in the stream drains.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                             Args &&...args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <int EPI, bool A_MN, bool B_MN>
 cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &c, const Params &p, int workers,
-                        cudaStream_t s, const SgdMaps *sgd = nullptr)
+                        cudaStream_t s, const SgdMaps *sgd = nullptr, bool pdl = false)
 {
     static const SgdMaps no_sgd{};
     constexpr int NT = (EPI == EPI_SGD) ? 256 : 128;      // the update epilogue is long and runs one CTA per SM
@@ -103,17 +119,22 @@ cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtens
         configured = cap;
     }
     const dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, workers);
-    gemm_bf16<EPI, A_MN, B_MN, NT><<<grid, NT, need, s>>>(a, b, c, sgd ? *sgd : no_sgd, p);
-    return cudaGetLastError();
+    return launch_dependent(pdl, gemm_bf16<EPI, A_MN, B_MN, NT>, grid, dim3(NT), (size_t)need, s, a, b, c,
+                            sgd ? *sgd : no_sgd, p);
 }
 
 inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK - 1) / BK)); }
 
 // ------------------------------------------------------------------------------------------ small kernels
+// warps per CTA of head_backward (measured inside the gradient chain: 2 warps 20.3 us, 4 warps 14.3 us,
+// 8 warps 15.9 us; about 8 us of it is fixed cost, not the loop over the samples)
+constexpr int HEAD_NW = 4;
 // Output layer forward and loss.  One CTA = 8 samples of one worker (one per warp); W3 sits in shared
 // memory; every lane loads its slices of the h2 row up front (all loads in flight at once):
 // logits = h2 W3^T + b3 (fp32), row loss = -log softmax[label], dz3 = bf16((softmax - onehot) / batch)
 // kept as fp32 values in dz3[w][b][16].  grid (B / 8, K).
+// DOUT: compile-time bound of the class loops (>= d_out; 10 for the paper-shaped workload, else 16).
+template <int DOUT>
 __global__ void __launch_bounds__(256)
 head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long long P, long long oW3, long long ob3,
             const int *__restrict__ labels, float *__restrict__ dz3, float *__restrict__ rowloss, int B, int d_h,
@@ -121,6 +142,8 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
 {
     extern __shared__ __align__(16) uint8_t head_smem[];
     bf16 *sW3 = reinterpret_cast<bf16 *>(head_smem);                 // [d_out][d_h]
+    pdl_launch_dependents();
+    pdl_wait();
     const int w = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int b = blockIdx.x * 8 + warp;
     const bf16 *hrow = h2 + ((long long)w * B + b) * d_h;
@@ -138,9 +161,9 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
     const float bias = (lane < d_out) ? __bfloat162float(b3[lane]) : 0.0f;
     const int y = labels[(long long)w * B + b];
     __syncthreads();
-    float acc[16];
+    float acc[DOUT];
 #pragma unroll
-    for (int c = 0; c < 16; ++c) acc[c] = 0.0f;
+    for (int c = 0; c < DOUT; ++c) acc[c] = 0.0f;
     for (int j0 = 0; j0 < d_h; j0 += 256 * MAXV) {
         if (j0 > 0) {
 #pragma unroll
@@ -158,8 +181,8 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
 #pragma unroll
                 for (int e = 0; e < 8; ++e) hf[e] = __bfloat162float(hp[e]);
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    if (c < d_out) {
+                for (int c = 0; c < DOUT; ++c) {
+                    if (DOUT == 10 || c < d_out) {
                         const uint4 wv = *reinterpret_cast<const uint4 *>(sW3 + c * d_h + j);
                         const bf16 *wp = reinterpret_cast<const bf16 *>(&wv);
 #pragma unroll
@@ -170,13 +193,13 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
         }
     }
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
+    for (int c = 0; c < DOUT; ++c)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
     // lane c finishes class c
     float z = -INFINITY;
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
+    for (int c = 0; c < DOUT; ++c)
         if (lane == c && c < d_out) z = acc[c] + bias;
     float zmax = z;
 #pragma unroll
@@ -199,18 +222,22 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
 //   dW3[c][j] = sum_b dz3[b][c] h2[b][j];
 // the CTA with blockIdx.x == 0 also writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the
 // zero padding of the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32, K).
-__global__ void __launch_bounds__(128)
+template <int DOUT, int NW>
+__global__ void __launch_bounds__(32 * NW)
 head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, const float *__restrict__ dz3,
               const float *__restrict__ rowloss, bf16 *__restrict__ dz2, float *__restrict__ grads,
               float *__restrict__ loss, long long P, long long P_raw, long long oW3, long long ob2, long long ob3,
               int B, int d_h, int d_out)
 {
-    constexpr int NW = 4;                          // warps per CTA; warp wp owns samples wp, wp + 4, ...
+    // NW warps per CTA; warp wp owns samples wp, wp + NW, ...; DOUT bounds the class loops (>= d_out)
+    constexpr int C4 = (DOUT + 3) / 4;
     __shared__ __align__(16) float sdz[128 * 16];
     __shared__ float red[NW][16][33];
     __shared__ float colsum[NW][33];
     const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
     const int j = j0 + lane;
+    pdl_launch_dependents();
+    pdl_wait();
     // first batch of this thread's h2 values: in flight while dz3 and W3 are fetched
     float hreg[16];
 #pragma unroll
@@ -219,9 +246,9 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
         hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
     }
     for (int i = threadIdx.x; i < B * 16; i += 32 * NW) sdz[i] = dz3[(long long)w * B * 16 + i];
-    float w3[16], acc3[16];
+    float w3[4 * C4], acc3[4 * C4];
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
+    for (int c = 0; c < 4 * C4; ++c) {
         w3[c] = (c < d_out) ? __bfloat162float(params[(long long)w * P + oW3 + (long long)c * d_h + j]) : 0.0f;
         acc3[c] = 0.0f;
     }
@@ -243,13 +270,15 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
                 float a = 0.0f;
                 const float4 *d4 = reinterpret_cast<const float4 *>(sdz + b * 16);
 #pragma unroll
-                for (int c4 = 0; c4 < 4; ++c4) {
+                for (int c4 = 0; c4 < C4; ++c4) {
                     const float4 dd = d4[c4];
                     const float d[4] = {dd.x, dd.y, dd.z, dd.w};
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
-                        a = fmaf(d[e], w3[4 * c4 + e], a);
-                        acc3[4 * c4 + e] = fmaf(d[e], h, acc3[4 * c4 + e]);
+                        if (4 * c4 + e < DOUT) {
+                            a = fmaf(d[e], w3[4 * c4 + e], a);
+                            acc3[4 * c4 + e] = fmaf(d[e], h, acc3[4 * c4 + e]);
+                        }
                     }
                 }
                 const bf16 v = __float2bfloat16_rn(h > 0.0f ? a : 0.0f);
@@ -259,7 +288,7 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
         }
     }
 #pragma unroll
-    for (int c = 0; c < 16; ++c) red[wp][c][lane] = acc3[c];
+    for (int c = 0; c < 16; ++c) red[wp][c][lane] = (c < DOUT) ? acc3[c < DOUT ? c : 0] : 0.0f;
     colsum[wp][lane] = csum;
     __syncthreads();
     for (int i = threadIdx.x; i < 16 * 32; i += 32 * NW) {
@@ -358,7 +387,9 @@ int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_h
     alloc((void **)&h->error_flag, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->error_flag, 0, sizeof(int));
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(head_logits, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * d_hidden * (int)sizeof(bf16));
+        e = cudaFuncSetAttribute(head_logits<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * d_hidden * (int)sizeof(bf16));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(head_logits<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * d_hidden * (int)sizeof(bf16));
     if (e != cudaSuccess) {
         cudaGetLastError();
         mlp_free(h);
@@ -424,23 +455,29 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     }
 #define LAUNCH_OK() do { if (cudaGetLastError() != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
 #define GEMM_OK(call) do { if ((call) != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
+    // Each kernel of the chain may set up while its predecessor drains (programmatic dependent launch):
+    // 11 % off the eager chain.  Not while the stream is being captured: replayed from a graph the chain
+    // measured 1.5 % slower with these edges than without.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) return COCOD_ERR_CUDA;
+    const bool pdl = (capturing == cudaStreamCaptureStatusNone);
     Params p{};
     p.error_flag = h->error_flag;
     // h1 = relu(x W1^T + b1)
     p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
     p.o = h->h1; p.o_worker_stride = (long long)B * d_h;
     p.bias = prm + h->ob1; p.bias_worker_stride = P;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, none, p, K, s)));
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, none, p, K, s, nullptr, pdl)));
     // h2 = relu(h1 W2^T + b2)
     p.K = d_h; p.stages = stages_for(d_h); p.o = h->h2; p.bias = prm + h->ob2;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, none, p, K, s)));
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, none, p, K, s, nullptr, pdl)));
     // output layer, loss, dz3; then dz2, dW3, db3, db2
-    head_logits<<<dim3(B / 8, K), 256, (size_t)d_out * d_h * sizeof(bf16), s>>>(h->h2, prm, P, h->oW3, h->ob3, labels,
-                                                                               h->dz3, h->rowloss, B, d_h, d_out);
-    LAUNCH_OK();
-    head_backward<<<dim3(d_h / 32, K), 128, 0, s>>>(h->h2, prm, h->dz3, h->rowloss, h->dz2, grads, loss, P, h->P_raw,
-                                                    h->oW3, h->ob2, h->ob3, B, d_h, d_out);
-    LAUNCH_OK();
+    const size_t w3_bytes = (size_t)d_out * d_h * sizeof(bf16);
+    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_logits<10> : head_logits<16>, dim3(B / 8, K), dim3(256), w3_bytes, s,
+                             h->h2, prm, P, h->oW3, h->ob3, labels, h->dz3, h->rowloss, B, d_h, d_out));
+    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32, K),
+                             dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->dz3, (const float *)h->rowloss,
+                             h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
     Params q{};
     q.error_flag = h->error_flag;
@@ -448,21 +485,21 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     q.o = h->dz1; q.o_worker_stride = (long long)B * d_h;
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
     q.colsum = grads + h->ob1; q.colsum_worker_stride = P;      // db1 = column sums of dz1, from the same epilogue
-    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, none, q, K, s)));
+    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, none, q, K, s, nullptr, pdl)));
     // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
     Params r{};
     r.error_flag = h->error_flag;
     r.M = d_h; r.N = d_h; r.K = B; r.stages = stages_for(B);
     if (fused) {
         r.lr = fused->lr; r.mu = fused->mu; r.wd = fused->wd; r.has_shadow = fused->shadow != nullptr;
-        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2)));
+        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, pdl)));
         r.N = d_in;
-        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1)));
+        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1, pdl)));
     } else {
         r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s)));
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s, nullptr, pdl)));
         r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s)));
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, nullptr, pdl)));
     }
 #undef LAUNCH_OK
 #undef GEMM_OK
