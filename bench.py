@@ -469,6 +469,58 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_reference_mlp(args):
+    """Reference arm of the MLP workload: the oracle as it stands on the host cores.  A step is one round
+    (Step I, k x (numpy fp64 gradient with the bf16 rounding points + reference-mode update), line 6) of a
+    SAMPLE of two of the 16 workers."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import numpy as np
+    from oracle import mlp_oracle as MO
+    from oracle.cocod_oracle import OracleEngine
+    from paper_1906_12043_b200 import inputs as I
+    nw, k, lr, mu, wd = 2, args.k or 4, 0.05, 0.9, 0.0
+    dims = I.MLP_DIMS
+    x0 = I.mlp_init_params(I.MLP_STUDENT_SEED)
+    teacher = I.mlp_init_params(I.MLP_TEACHER_SEED)
+    P_raw = x0.size
+    oe = OracleEngine(nw, P_raw, lr, mu, wd, mode="ref")
+    oe.set_params(x0)
+    ring = max(k, 8)
+    Xo = [[I.mlp_batch(w, t) for w in range(nw)] for t in range(ring)]
+    yo = [[I.mlp_teacher_labels(Xo[t][w], teacher) for w in range(nw)] for t in range(ring)]
+    tau = [0]
+
+    def one_round():
+        oe.comm_begin()
+        for _ in range(k):
+            t = tau[0] % ring
+            g = np.stack([MO.loss_and_grad(oe.x[w], Xo[t][w], yo[t][w], dims, emulate_bf16=True)[1] for w in range(nw)])
+            oe.local_step(g)
+            tau[0] += 1
+        oe.comm_end()
+
+    for _ in range(args.warmup):
+        one_round()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_round()
+    dt = time.perf_counter() - t0
+    value = nw * P_raw * k * args.steps / dt
+    sample = (f"{nw} of 16 workers, {args.steps} rounds of k={k} local steps (numpy fp64 gradient with bf16 rounding "
+              f"points + reference-mode parameter path)")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 contractions / f32 state", "data": "synthetic",
+        "config": {"workload": "mlp", "K": 16, "P": P_raw, "k": k, "lr": lr, "mu": mu, "wd": wd, "mlp": list(dims),
+                   "batch": I.MLP_BATCH, "sampled_workers": nw},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
 def run_mlp(args):
     """End-to-end synthetic training: K = 16 workers each train the 784-1024-1024-10 ReLU MLP
     (bf16 weights, fp32 master copy and momentum) on minibatches of 128; gradients come from the
@@ -847,8 +899,7 @@ def main():
     from paper_1906_12043_b200.workloads import WORKLOADS
     if args.workload == "mlp":
         if args.impl == "reference":
-            print(json.dumps({"impl": "reference", "unavailable": "the oracle's MLP leg is timed by tests only; "
-                              "use the default workload for the reference arm"}))
+            run_reference_mlp(args)
             return
         run_mlp(args)
         return

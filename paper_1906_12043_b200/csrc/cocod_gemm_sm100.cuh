@@ -6,7 +6,7 @@
 // B is [N][K]) or "MN-major" (m resp. n is contiguous: A is [K][M], B is [K][N]); the tensor cores
 // read both forms from shared memory, so no operand is ever transposed in memory.  One CTA
 // computes one 128 x 128 tile of one worker:
-//   * operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
+//   * operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle; every CTA fetches its own tiles) into a
 //     shared-memory ring of up to 6 stages (32 KB each) guarded by mbarriers;
 //   * one elected thread issues tcgen05.mma (kind::f16, bf16 inputs, fp32 accumulation) on
 //     shared-memory descriptors; the 128 x 128 fp32 accumulator lives in TMEM (128 columns);
