@@ -121,7 +121,9 @@ def run_gpu_grad(M, K, dims, params, X, y):
 
 
 @pytest.mark.parametrize("K,dims,dyadic", [(2, (64, 128, 128, 10), False), (3, (200, 256, 256, 7), False),
-                                            (3, (200, 256, 256, 7), True), (16, I.MLP_DIMS, True)])
+                                            (3, (200, 256, 256, 7), True), (16, I.MLP_DIMS, True),
+                                            (2, (72, 384, 384, 10), True), (2, (72, 384, 384, 16), True),
+                                            (3, (64, 512, 512, 10), True), (2, (64, 512, 512, 3), False)])
 def test_batched_gradient_matches_the_oracle(M, K, dims, dyadic):
     params, X, y, P_raw = (make_dyadic_problem if dyadic else make_problem)(K, dims, seed=3)
     g, loss, mg = run_gpu_grad(M, K, dims, params, X, y)
