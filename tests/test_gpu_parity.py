@@ -157,7 +157,8 @@ def test_config1_full_vector_parity(E, snapshot):
 # ----------------------------------------------------------------------------- shapes: tiles, ragged tails, misaligned rows
 @pytest.mark.parametrize("K,P", [(1, 1), (1, 4099), (2, 8), (3, 7), (5, 1001), (2, 3), (16, 4096 + 4),
                                  (64, 1028), (7, 262_144 + 12), (33, 515), (128, 260),
-                                 (2, 4096 + 8), (3, 1024), (4, 100_000), (1, 2048), (9, 8 * 1000)])
+                                 (2, 4096 + 8), (3, 1024), (4, 100_000), (1, 2048), (9, 8 * 1000),
+                                 (1024, 40), (1024, 3)])          # the largest worker count the engine accepts
 @pytest.mark.parametrize("snapshot", [0, 1])
 def test_shapes_spanning_tiles_and_ragged_tails(E, K, P, snapshot):
     rng = np.random.default_rng(K * 1000 + P)
