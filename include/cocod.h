@@ -243,11 +243,12 @@ int cocod_comm_gather(cocod_handle *h);
 /* The gather kernel on caller-owned buffers (no handle): rows = device array of K device pointers
  * (row i = worker i's P stored values, in any allocation this GPU can address), outs = device
  * array of G device pointers to P-float average buffers; columns [col_lo, col_hi) are averaged
- * (weights w: device, K floats, or NULL for 1/K) and written to every outs[q].  vec4 != 0 selects the
- * 128-bit path: the caller vouches that every row and output pointer is 16-byte aligned, and
- * col_lo, col_hi must be multiples of 4 (INVALID otherwise). */
+ * (weights w: device, K floats, or NULL for 1/K) and written to every outs[q].  vec = 1, 4 or 8 is the
+ * number of columns per access: the caller vouches that every row and output pointer is aligned
+ * to 4 * vec bytes, and col_lo, col_hi must be multiples of vec (INVALID otherwise; 8 is used for
+ * K <= 4 only, larger K take the 4-column path). */
 int cocod_kernel_mean_gather(const float *const *rows, int K, int64_t col_lo, int64_t col_hi, const float *w,
-                             float *const *outs, int G, int vec4, cocod_stream_t stream);
+                             float *const *outs, int G, int vec, cocod_stream_t stream);
 
 /* ---------------------------------------------------------------------------------------------
  * The four kernels on caller-owned device buffers (no handle, no state): the same code the

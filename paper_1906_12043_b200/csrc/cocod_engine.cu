@@ -172,16 +172,21 @@ cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, flo
     return cudaGetLastError();
 }
 
-// Average of columns [lo, hi) over rows held in separate allocations, written to G buffers.  vec4: the
-// caller vouches that all row and output pointers are 16-byte aligned and lo, hi are multiples of 4.
+// Average of columns [lo, hi) over rows held in separate allocations, written to G buffers.  vec (1, 4 or 8):
+// the caller vouches that all row and output pointers are 4 * vec-byte aligned and lo, hi are multiples of vec.
 cudaError_t launch_mean_gather(const float *const *rows, int K, int64_t lo, int64_t hi, const float *w,
-                               float *const *outs, int G, float inv_k, bool vec4, cudaStream_t s, int *n_launch)
+                               float *const *outs, int G, float inv_k, int vec, cudaStream_t s, int *n_launch)
 {
     using namespace cocod;
     if (hi <= lo) return cudaSuccess;
-    if (vec4) {
+    if (vec == 8 && K <= 4) {           // few workers: 256-bit accesses keep enough bytes in flight
+        const int64_t c_lo = lo / 8, c_hi = hi / 8;
+        const unsigned grid = grid_for(c_hi - c_lo, kThreads);
+        if (K <= 2) mean_gather_vec8<2><<<grid, kThreads, 0, s>>>(rows, K, c_lo, c_hi, w, outs, G, inv_k);
+        else mean_gather_vec8<4><<<grid, kThreads, 0, s>>>(rows, K, c_lo, c_hi, w, outs, G, inv_k);
+    } else if (vec >= 4) {
         const int64_t c_lo = lo / 4, c_hi = hi / 4;
-        mean_gather_vec4<<<grid_for(c_hi - c_lo, kThreads), kThreads, 0, s>>>(
+        mean_gather_vec4<<<grid_for(c_hi - c_lo, kThreads), kThreads, (size_t)K * sizeof(float4 *), s>>>(
             reinterpret_cast<const float4 *const *>(rows), K, c_lo, c_hi, w,
             reinterpret_cast<float4 *const *>(outs), G, inv_k);
     } else {
@@ -514,9 +519,9 @@ int cocod_comm_gather(cocod_handle *h)
 {
     if (int rc = check_live(h)) return rc;
     if (h->state != IN_FLIGHT || h->G == 0 || h->mean_started) return COCOD_ERR_STATE;
-    // this GPU's share of the columns (in float4 units when every row is 16-byte aligned)
-    const bool vec4 = (h->P % 4) == 0;
-    const int64_t units = vec4 ? h->P / 4 : h->P;
+    // this GPU's share of the columns, in units of 8, 4 or 1 columns as the rows' alignment allows
+    const int vec = (h->P % 8) == 0 ? 8 : (h->P % 4) == 0 ? 4 : 1;
+    const int64_t units = h->P / vec;
     const int64_t base = units / h->G, rem = units % h->G;
     const int64_t lo = h->rank * base + std::min<int64_t>(h->rank, rem);
     const int64_t hi = lo + base + (h->rank < rem ? 1 : 0);
@@ -524,8 +529,8 @@ int cocod_comm_gather(cocod_handle *h)
     int nl = 0;
     {
         Bracket br(h, h->side, COCOD_KERNEL_MEAN);
-        CK(h, launch_mean_gather(h->rows_tab[b], h->K_global, vec4 ? lo * 4 : lo, vec4 ? hi * 4 : hi, h->wg,
-                                 h->outs_tab, h->G, mean_scale(h), vec4, h->side, &nl));
+        CK(h, launch_mean_gather(h->rows_tab[b], h->K_global, lo * vec, hi * vec, h->wg, h->outs_tab, h->G,
+                                 mean_scale(h), vec, h->side, &nl));
     }
     h->launches += nl;
     h->mean_started = true;
@@ -973,11 +978,12 @@ int cocod_ipc_detach(cocod_handle *h)
 }
 
 int cocod_kernel_mean_gather(const float *const *rows, int K, int64_t col_lo, int64_t col_hi, const float *w,
-                             float *const *outs, int G, int vec4, cocod_stream_t stream)
+                             float *const *outs, int G, int vec, cocod_stream_t stream)
 {
     if (!rows || !outs || K < 1 || G < 1 || col_lo < 0 || col_hi < col_lo) return COCOD_ERR_INVALID;
-    if (vec4 && ((col_lo | col_hi) & 3)) return COCOD_ERR_INVALID;
-    return launch_mean_gather(rows, K, col_lo, col_hi, w, outs, G, 1.0f / (float)K, vec4 != 0, (cudaStream_t)stream,
+    if (vec != 1 && vec != 4 && vec != 8) return COCOD_ERR_INVALID;
+    if ((col_lo % vec) || (col_hi % vec)) return COCOD_ERR_INVALID;
+    return launch_mean_gather(rows, K, col_lo, col_hi, w, outs, G, 1.0f / (float)K, vec, (cudaStream_t)stream,
                               nullptr) == cudaSuccess ? COCOD_OK : COCOD_ERR_CUDA;
 }
 

@@ -316,15 +316,41 @@ static __global__ void __launch_bounds__(kThreads)
 mean_gather_vec4(const float4 *const *__restrict__ rows, int K, int64_t c_lo, int64_t c_hi,
                  const float *__restrict__ w, float4 *const *__restrict__ outs, int G, float inv_k)
 {
+    // the row addresses once per CTA into shared memory (dynamic, K pointers): the 8 loads of a block of
+    // rows then depend on nothing but a shared-memory read
+    extern __shared__ const float4 *gather_rows[];
+    for (int i = threadIdx.x; i < K; i += kThreads) gather_rows[i] = rows[i];
+    __syncthreads();
     const int64_t c = c_lo + (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (c >= c_hi) return;
     float s[4];
     mean_rows<4, 8>(s, K, w, inv_k, [&](int i, float (&v)[4]) {
-        const float4 t = __ldcg(rows[i] + c);      // L2 only: each value is read once
+        const float4 t = __ldcs(gather_rows[i] + c);       // each value is read once
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     });
     const float4 o = make_float4(s[0], s[1], s[2], s[3]);
     for (int q = 0; q < G; ++q) outs[q][c] = o;
+}
+
+// Few workers (K <= CAP <= 4): 8 columns per thread with 256-bit accesses, as in mean_vec8.  32-byte aligned rows
+// and outputs, c_lo and c_hi in units of 8 columns.
+template <int CAP>
+__global__ void __launch_bounds__(kThreads)
+mean_gather_vec8(const float *const *__restrict__ rows, int K, int64_t c_lo, int64_t c_hi,
+                 const float *__restrict__ w, float *const *__restrict__ outs, int G, float inv_k)
+{
+    const int64_t c = c_lo + (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (c >= c_hi) return;
+    float s[8];
+    mean_rows<8, CAP>(s, K, w, inv_k, [&](int i, float (&v)[8]) {
+        const f32x8 t = ld256_stream(rows[i] + c * 8);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = t.a[q];
+    });
+    f32x8 o;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) o.a[q] = s[q];
+    for (int q = 0; q < G; ++q) st256(outs[q] + c * 8, o);
 }
 
 static __global__ void __launch_bounds__(kThreads)

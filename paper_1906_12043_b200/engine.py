@@ -363,13 +363,13 @@ def kernel_mean(snap, mean, w=None, stream=None):
     _ck_rc(load().cocod_kernel_mean(_ptr(snap), K, P, _ptr(w), _ptr(mean), s), "cocod_kernel_mean")
 
 
-def kernel_mean_gather(rows, col_lo, col_hi, outs, w=None, vec4=True, stream=None):
+def kernel_mean_gather(rows, col_lo, col_hi, outs, w=None, vec=4, stream=None):
     """rows: int64 CUDA tensor of K device addresses (one per worker's P stored values); outs: int64
-    CUDA tensor of G device addresses of P-float average buffers."""
+    CUDA tensor of G device addresses of P-float average buffers; vec: columns per access (1, 4, 8)."""
     import torch
     s = _stream(stream) if stream is not None else torch.cuda.current_stream().cuda_stream
     _ck_rc(load().cocod_kernel_mean_gather(_ptr(rows), rows.numel(), int(col_lo), int(col_hi), _ptr(w), _ptr(outs),
-                                           outs.numel(), 1 if vec4 else 0, s), "cocod_kernel_mean_gather")
+                                           outs.numel(), int(vec), s), "cocod_kernel_mean_gather")
 
 
 def kernel_merge(x, snap, mean, stream=None):

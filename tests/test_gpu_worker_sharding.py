@@ -65,12 +65,13 @@ def address_table(tensors):
 
 
 # ----------------------------------------------------------------------------- the gather kernel by itself
-@pytest.mark.parametrize("K,P,weighted,vec4", [
-    (1, 4096, False, True), (3, 4 * 1001, True, True), (8, 4 * 50_000, False, True),
-    (16, 4 * 50_001, False, True), (19, 4 * 7777, True, True), (16, 10_007, False, False),
-    (5, 999, True, False),
+@pytest.mark.parametrize("K,P,weighted,vec", [
+    (1, 4096, False, 4), (3, 4 * 1001, True, 4), (8, 4 * 50_000, False, 4),
+    (16, 4 * 50_001, False, 4), (19, 4 * 7777, True, 4), (16, 10_007, False, 1),
+    (5, 999, True, 1), (1, 8 * 999, False, 8), (2, 8 * 40_001, True, 8), (3, 8 * 5_000, False, 8),
+    (4, 8 * 30_000, True, 8), (16, 8 * 30_000, False, 8),
 ])
-def test_gather_kernel_equals_the_mirror_mean_with_rows_in_separate_allocations(E, K, P, weighted, vec4):
+def test_gather_kernel_equals_the_mirror_mean_with_rows_in_separate_allocations(E, K, P, weighted, vec):
     rng = np.random.default_rng(K * 1000 + P)
     S = (rng.standard_normal((K, P)) * 0.1).astype(np.float32)
     M = rng.integers(1, 9, K).astype(np.float64) * 32 if weighted else None
@@ -82,9 +83,9 @@ def test_gather_kernel_equals_the_mirror_mean_with_rows_in_separate_allocations(
     G = 3
     outs = [torch.full((P,), float("nan"), device="cuda") for _ in range(G)]
     w = None if M is None else torch.from_numpy((M / M.sum()).astype(np.float32)).cuda()
-    unit = 4 if vec4 else 1
+    unit = vec
     lo, hi = (P // 3) // unit * unit, (2 * P // 3) // unit * unit             # a share in the middle
-    E.kernel_mean_gather(address_table(rows), lo, hi, address_table(outs), w=w, vec4=vec4)
+    E.kernel_mean_gather(address_table(rows), lo, hi, address_table(outs), w=w, vec=vec)
     torch.cuda.synchronize()
     for q in range(G):
         got = cpu(outs[q])
@@ -94,13 +95,12 @@ def test_gather_kernel_equals_the_mirror_mean_with_rows_in_separate_allocations(
     for r in range(G):
         units = P // unit
         a, b = units * r // G * unit, (units * (r + 1) // G * unit if r < G - 1 else P)
-        if vec4:
-            b = b // 4 * 4
-        E.kernel_mean_gather(address_table(rows), a, b, address_table(outs), w=w, vec4=vec4)
+        b = b // unit * unit
+        E.kernel_mean_gather(address_table(rows), a, b, address_table(outs), w=w, vec=vec)
     torch.cuda.synchronize()
     assert_bit_equal(cpu(outs[1])[:P // unit * unit], expect[:P // unit * unit])
     with pytest.raises(E.CocodError) as e:
-        E.kernel_mean_gather(address_table(rows), 2, 8, address_table(outs), vec4=True)
+        E.kernel_mean_gather(address_table(rows), 2, 8, address_table(outs), vec=4)
     assert e.value.code == E.ERR_INVALID
 
 
