@@ -226,7 +226,9 @@ int cocod_comm_exchanged(cocod_handle *h);
  * average buffer, plus K, first, K_global and P for cross-checking).  The caller collects the
  * blobs of all G processes in rank order (any host transport) and passes them to cocod_ipc_attach
  * together with its own rank; the engine opens the other processes' buffers (they must be on GPUs
- * with peer access to this one, or on this one) and builds its address tables.  The blobs must
+ * with peer access to this one, or on this one) and builds its address tables.  Engines of the
+ * calling process itself are addressed directly, without a handle (if they sit on other GPUs, the
+ * caller has enabled peer access between the devices).  The blobs must
  * tile 0..K_global with equal P and K_global (INVALID otherwise; CUDA if a handle cannot be
  * opened).  G is at most 64.  cocod_ipc_detach closes them again (also done by cocod_destroy);
  * every process must detach before any process destroys its engine.  Requires cocod_set_shard
