@@ -298,11 +298,13 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             }
         }
     }
+    if (threadIdx.x == 0) COCOD_TRACE(6);
     __syncwarp();
     if (warp == 0) {                  // warp-collective TMEM allocation
         tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
         tmem_relinquish();
     }
+    if (threadIdx.x == 0) COCOD_TRACE(7);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
