@@ -46,8 +46,9 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Epilogue {
     EPI_F32 = 0,        // c[m][n] = acc                         (fp32, row stride ldc; TMA store if map_c_ok)
-    EPI_BIAS_RELU = 1,  // o[m][n] = bf16(max(acc + bias[n], 0))
-    EPI_MASK = 2,       // o[m][n] = bf16(acc * (mask[m][n] > 0)); optionally colsum[n] = sum_m o[m][n] (M <= 128)
+    EPI_BIAS_RELU = 1,  // o[m][n] = bf16(max(acc + bias[n], 0))          (o = the bf16 matrix map_c describes: boxes of
+    EPI_MASK = 2,       // o[m][n] = bf16(acc * (mask[m][n] > 0));         64 columns x 128 rows, 128-byte swizzle)
+                        // optionally colsum[n] = sum_m o[m][n] (M <= 128)
     EPI_SGD = 3         // g = acc: d = fma(wd, x, g); v = fma(mu, v, d); x = fma(-lr, v, x); shadow = bf16(x)
 };
 
@@ -63,8 +64,6 @@ struct Params {
     long long c_worker_stride;         // elements
     int ldc;
     int map_c_ok;                      // EPI_F32: map_c describes c, use TMA stores
-    __nv_bfloat16 *o;                  // bf16 output [M][N], row stride N
-    long long o_worker_stride;
     const __nv_bfloat16 *bias;         // [N]
     long long bias_worker_stride;
     const __nv_bfloat16 *mask;         // [M][N], row stride N
@@ -273,7 +272,8 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     if (threadIdx.x == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_b) : "memory");
-        if (EPI == EPI_F32 && p.map_c_ok) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+        if (EPI == EPI_BIAS_RELU || EPI == EPI_MASK || (EPI == EPI_F32 && p.map_c_ok))
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
         for (int s = 0; s < stages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
@@ -478,7 +478,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
             for (int cc = 0; cc < NCH; ++cc) {
                 const int c = cbase + cc;
-                const int nb = n0 + c * 32;
                 __align__(16) __nv_bfloat16 outv[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
@@ -491,37 +490,40 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     }
                     outv[j] = __float2bfloat16_rn(a);
                 }
-                if (EPI == EPI_MASK && p.colsum != nullptr) {       // stage the row for the column sums (padded rows)
+                // stage the bf16 row in the (now idle) ring in the TMA swizzle: 64-column boxes of 128-byte rows,
+                // 16-byte piece j of row r at piece j ^ (r & 7)
+                {
                     const uint4 *src = reinterpret_cast<const uint4 *>(outv);
-                    uint4 *stg = reinterpret_cast<uint4 *>(smem + row * 272 + c * 64);
+                    uint8_t *box = smem + (c >> 1) * (BM * 128) + row * 128;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) stg[j] = src[j];
-                }
-                if (m < p.M && nb < p.N) {
-                    __nv_bfloat16 *dst = p.o + (long long)wk * p.o_worker_stride + (long long)m * p.N + nb;
-                    if (nb + 32 <= p.N && ((reinterpret_cast<uintptr_t>(dst) & 15u) == 0)) {
-                        const uint4 *src = reinterpret_cast<const uint4 *>(outv);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) reinterpret_cast<uint4 *>(dst)[j] = src[j];
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (nb + j < p.N) dst[j] = outv[j];
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4 *>(box + ((((c & 1) * 4 + j) ^ (row & 7)) << 4)) = src[j];
                 }
             }
-        }
-        if (EPI == EPI_MASK && p.colsum != nullptr) {
-            // the whole batch is in this tile: thread t adds column t over the rows, in row order
+            // the tile leaves through two bulk stores (whole 128-byte lines; rows and columns beyond the
+            // matrix are clipped by the tensor map)
+            fence_async_smem();
             __syncthreads();
-            const int t = threadIdx.x;
-            if (t < BN && n0 + t < p.N) {
-                const int rows = (p.M - m0 < BM) ? (p.M - m0) : BM;
-                float acc = 0.0f;
-                for (int rr = 0; rr < rows; ++rr)
-                    acc += __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(smem + rr * 272 + t * 2));
-                p.colsum[(long long)wk * p.colsum_worker_stride + n0 + t] = acc;
+            if (threadIdx.x == 0) {
+#pragma unroll
+                for (int b = 0; b < BN / 64; ++b)
+                    if (n0 + b * 64 < p.N) tma_store_3d(&map_c, smem_base + b * (BM * 128), n0 + b * 64, m0, wk);
+                tma_store_commit();
             }
+            if (EPI == EPI_MASK && p.colsum != nullptr) {
+                // the whole batch is in this tile: thread t adds column t of the staged tile over the rows, in row order
+                const int t = threadIdx.x;
+                if (t < BN && n0 + t < p.N) {
+                    const int rows = (p.M - m0 < BM) ? (p.M - m0) : BM;
+                    const uint8_t *colp = smem + (t >> 6) * (BM * 128) + (t & 7) * 2;
+                    const int piece = (t & 63) >> 3;
+                    float acc = 0.0f;
+                    for (int rr = 0; rr < rows; ++rr)
+                        acc += __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(colp + rr * 128 + ((piece ^ (rr & 7)) << 4)));
+                    p.colsum[(long long)wk * p.colsum_worker_stride + n0 + t] = acc;
+                }
+            }
+            if (threadIdx.x == 0) tma_store_wait_read<0>();      // shared memory must outlive the reads
         }
     } else if (threadIdx.x == 0 && p.error_flag != nullptr) {
         atomicExch(p.error_flag, 1);

@@ -342,6 +342,7 @@ struct cocod_mlp {
     float *gscratch = nullptr;          // K x P gradients of the fused path's small tensors (allocated on first use)
     // maps over scratch (fixed addresses): reduction-contiguous (k) and row-contiguous (mn) views
     CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
+    CUtensorMap st_h2, st_dz1;          // store views (64 columns x 128 rows) of outputs that are not read that way
     long long launches = 0;
 };
 
@@ -400,7 +401,8 @@ int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_h
     // d_h; as a row-contiguous operand the reduction runs over the batch.
     bool ok = map_k(&h->k_h1, h->h1, uh, uB, uK, uh, uB * uh) && map_k(&h->k_dz2, h->dz2, uh, uB, uK, uh, uB * uh) &&
               map_mn(&h->mn_dz2, h->dz2, uh, uB, uK, uh, uB * uh) && map_mn(&h->mn_h1, h->h1, uh, uB, uK, uh, uB * uh) &&
-              map_mn(&h->mn_dz1, h->dz1, uh, uB, uK, uh, uB * uh);
+              map_mn(&h->mn_dz1, h->dz1, uh, uB, uK, uh, uB * uh) && map_k(&h->st_h2, h->h2, uh, uB, uK, uh, uB * uh) &&
+              map_k(&h->st_dz1, h->dz1, uh, uB, uK, uh, uB * uh);
     if (!ok) {
         mlp_free(h);
         return COCOD_ERR_CUDA;
@@ -465,12 +467,11 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     p.error_flag = h->error_flag;
     // h1 = relu(x W1^T + b1)
     p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
-    p.o = h->h1; p.o_worker_stride = (long long)B * d_h;
     p.bias = prm + h->ob1; p.bias_worker_stride = P;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, none, p, K, s, nullptr, pdl)));
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, nullptr, pdl)));
     // h2 = relu(h1 W2^T + b2)
-    p.K = d_h; p.stages = stages_for(d_h); p.o = h->h2; p.bias = prm + h->ob2;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, none, p, K, s, nullptr, pdl)));
+    p.K = d_h; p.stages = stages_for(d_h); p.bias = prm + h->ob2;
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, nullptr, pdl)));
     // output layer, loss, dz3; then dz2, dW3, db3, db2
     const size_t w3_bytes = (size_t)d_out * d_h * sizeof(bf16);
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_logits<10> : head_logits<16>, dim3(B / 8, K), dim3(256), w3_bytes, s,
@@ -482,10 +483,9 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     Params q{};
     q.error_flag = h->error_flag;
     q.M = B; q.N = d_h; q.K = d_h; q.stages = stages_for(d_h);
-    q.o = h->dz1; q.o_worker_stride = (long long)B * d_h;
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
     q.colsum = grads + h->ob1; q.colsum_worker_stride = P;      // db1 = column sums of dz1, from the same epilogue
-    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, none, q, K, s, nullptr, pdl)));
+    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
     // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
     Params r{};
     r.error_flag = h->error_flag;
