@@ -22,9 +22,10 @@ struct cocod_step_plan {
 int cocod_internal_plan_step(cocod_handle *h, cocod_step_plan *plan);
 
 // Run the engine's local-step arithmetic on up to `nseg` column ranges [lo, hi) of every worker
-// (gradients in a K x P matrix g), on the compute stream.  Used for the parameters a fused caller
-// does not update itself.
-int cocod_internal_step_segments(cocod_handle *h, const float *g, const int64_t *lo, const int64_t *hi, int nseg);
+// (gradients in a K x P matrix g), on `stream` (NULL = the compute stream; another stream must be ordered
+// against the compute stream by the caller).  Used for the parameters a fused caller does not update itself.
+int cocod_internal_step_segments(cocod_handle *h, const float *g, const int64_t *lo, const int64_t *hi, int nseg,
+                                 cudaStream_t stream);
 
 // Account for a completed local step (buffer flip, step counter).
 int cocod_internal_finish_step(cocod_handle *h, int kernels_launched);

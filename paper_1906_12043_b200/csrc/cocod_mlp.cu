@@ -344,6 +344,10 @@ struct cocod_mlp {
     CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
     CUtensorMap st_h2, st_dz1;          // store views (64 columns x 128 rows) of outputs that are not read that way
     long long launches = 0;
+    // second branch of the backward pass (dW2 beside dz1 -> dW1): a stream of the handle's own, forked from and
+    // joined to the caller's stream by events
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
 };
 
 namespace {
@@ -352,6 +356,9 @@ void mlp_free(cocod_mlp *h)
 {
     void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag, h->gscratch};
     for (void *p : ptrs) if (p) cudaFree(p);
+    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+    if (h->ev_join) cudaEventDestroy(h->ev_join);
+    if (h->side) cudaStreamDestroy(h->side);
     delete h;
 }
 
@@ -387,6 +394,9 @@ int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_h
     alloc((void **)&h->rowloss, (size_t)K * batch * sizeof(float));
     alloc((void **)&h->error_flag, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->error_flag, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(head_logits<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * d_hidden * (int)sizeof(bf16));
         if (e == cudaSuccess)
@@ -431,7 +441,7 @@ namespace {
 // otherwise their GEMMs apply the engine's local step in their epilogue (x, v and the bf16 copy of x
 // are updated in place, nothing is written to `grads` for W1 and W2).
 int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labels, float *grads, float *loss,
-             cudaStream_t s, const cocod_step_plan *fused)
+             cudaStream_t s, const cocod_step_plan *fused, cocod_handle *engine = nullptr)
 {
     const int K = h->K, B = h->B, d_in = h->d_in, d_h = h->d_h, d_out = h->d_out;
     const long long P = h->P;
@@ -485,17 +495,40 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     q.M = B; q.N = d_h; q.K = d_h; q.stages = stages_for(d_h);
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
     q.colsum = grads + h->ob1; q.colsum_worker_stride = P;      // db1 = column sums of dz1, from the same epilogue
-    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
     // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
     Params r{};
     r.error_flag = h->error_flag;
     r.M = d_h; r.N = d_h; r.K = B; r.stages = stages_for(B);
+    // Replayed from a CUDA graph, the backward pass of the gradient call runs as two branches (the handle's own
+    // stream, forked from and joined to the caller's stream by events): measured 89.1 -> 82.8 us for the chain.
+    // Queued eagerly the same fork costs more in event calls than it gains (93.0 -> 94.2 us), so it is used under
+    // stream capture only.
+    const bool fork = (capturing != cudaStreamCaptureStatusNone);
+    // everything but W1 and W2 (b1, then b2 | W3 | b3 | padding) is updated by the engine's own kernel
+    const int64_t seg_lo[2] = {h->ob1, h->ob2}, seg_hi[2] = {h->oW2, h->P};
     if (fused) {
+        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
         r.lr = fused->lr; r.mu = fused->mu; r.wd = fused->wd; r.has_shadow = fused->shadow != nullptr;
         GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, pdl)));
         r.N = d_in;
         GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1, pdl)));
+        // (the engine's small update beside these two kernels, on the second stream, was measured 7 us SLOWER)
+        if (int rc = cocod_internal_step_segments(engine, grads, seg_lo, seg_hi, 2, nullptr)) return rc;
+    } else if (fork) {
+        // dW2 needs only dz2 and h1: it runs beside dz1 -> dW1.  dz1 is queued first and keeps a ring of three
+        // stages here, so that a CTA of dW2 fits next to it on the same SM (2, 4 and 6 stages measured slower).
+        if (cudaEventRecord(h->ev_fork, s) != cudaSuccess) return COCOD_ERR_CUDA;
+        q.stages = std::min(q.stages, 3);
+        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, false)));
+        if (cudaStreamWaitEvent(h->side, h->ev_fork, 0) != cudaSuccess) return COCOD_ERR_CUDA;
+        r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, h->side, nullptr, false)));
+        if (cudaEventRecord(h->ev_join, h->side) != cudaSuccess) return COCOD_ERR_CUDA;
+        r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, nullptr, false)));
+        if (cudaStreamWaitEvent(s, h->ev_join, 0) != cudaSuccess) return COCOD_ERR_CUDA;
     } else {
+        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
         r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
         GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s, nullptr, pdl)));
         r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
@@ -537,11 +570,9 @@ int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x
         }
     }
     const long long before = h->launches;
-    if (int rc = run_grad(h, plan.shadow, static_cast<const bf16 *>(x), labels, h->gscratch, loss, plan.compute, &plan))
+    if (int rc = run_grad(h, plan.shadow, static_cast<const bf16 *>(x), labels, h->gscratch, loss, plan.compute, &plan,
+                          engine))
         return rc;
-    // everything but W1 and W2: b1, then b2 | W3 | b3 | padding
-    const int64_t lo[2] = {h->ob1, h->ob2}, hi[2] = {h->oW2, h->P};
-    if (int rc = cocod_internal_step_segments(engine, h->gscratch, lo, hi, 2)) return rc;
     (void)before;
     return cocod_internal_finish_step(engine, 0);
 }

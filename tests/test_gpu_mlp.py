@@ -345,3 +345,67 @@ def test_fused_gradient_and_update_is_bit_identical_to_the_two_calls(M, E, K, di
     with pytest.raises(E.CocodError) as e:
         mg.grad_step(plain, X, y, loss1)
     assert e.value.code == E.ERR_STATE
+
+
+@pytest.mark.parametrize("K,dims", [(3, (200, 256, 256, 7)), (16, I.MLP_DIMS)])
+def test_gradient_paths_replayed_from_a_cuda_graph_match_the_eager_calls(M, E, K, dims):
+    """Under stream capture the backward pass is queued as two branches on two streams (and without the
+    programmatic launch edges of the eager chain); replaying the graph must give the eager results bit for
+    bit, for the gradient call and for the fused gradient + update call, replay after replay."""
+    rng = np.random.default_rng(100 + K)
+    lr, mu, wd = 0.05, 0.9, 5e-4
+    mg = M.MLPGrad(K, 128, dims[0], dims[1], dims[3])
+    P = mg.P
+    segs, _ = I.mlp_segments(dims)
+    x0 = np.zeros(P, np.float32)
+    for name, off, shape in segs:
+        n = int(np.prod(shape))
+        x0[off:off + n] = rng.standard_normal(n).astype(np.float32) * (1.0 / np.sqrt(shape[-1]) if name[0] == "W" else 0.1)
+    X = bf16_tensor(np.stack([I.mlp_batch(w, 0, 128, dims[0]) for w in range(K)]))
+    y = torch.from_numpy(rng.integers(0, dims[3], (K, 128)).astype(np.int32)).cuda()
+    eager, replayed = E.Engine(K, P, lr, mu, wd), E.Engine(K, P, lr, mu, wd)
+    for eng in (eager, replayed):
+        eng.set_option(E.OPT_BF16_SHADOW, 1)
+        eng.set_params(x0)
+    # ---- gradient call
+    g_e = torch.empty((K, P), dtype=torch.float32, device="cuda")
+    l_e = torch.empty(K, dtype=torch.float32, device="cuda")
+    mg.grad(eager.bf16_shadow(), X, y, g_e, l_e)
+    g_g, l_g = torch.full_like(g_e, float("nan")), torch.full_like(l_e, float("nan"))
+    cap = torch.cuda.Stream()
+    with torch.cuda.stream(cap):
+        mg.grad(replayed.bf16_shadow(), X, y, g_g, l_g)          # warm-up outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=cap):
+        mg.grad(replayed.bf16_shadow(), X, y, g_g, l_g)
+    for _ in range(3):
+        g_g.fill_(float("nan"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(g_g.view(torch.int32), g_e.view(torch.int32))
+        assert torch.equal(l_g, l_e)
+    # ---- fused gradient + update: three steps eagerly, three replays of one captured step
+    l1 = torch.empty(K, dtype=torch.float32, device="cuda")
+    scratch = E.Engine(K, P, lr, mu, wd)                 # the handle's first fused call allocates: not under capture
+    scratch.set_option(E.OPT_BF16_SHADOW, 1)
+    scratch.set_params(x0)
+    mg.grad_step(scratch, X, y, l1)
+    scratch.sync()
+    scratch.destroy()
+    replayed.sync()
+    replayed.set_stream(cap)
+    step = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(step, stream=cap):
+        mg.grad_step(replayed, X, y, l_g)
+    for i in range(3):
+        mg.grad_step(eager, X, y, l1)
+        step.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(l_g, l1), f"loss, step {i}"
+        assert torch.equal(replayed.get_params().view(torch.int32), eager.get_params().view(torch.int32)), f"x, step {i}"
+        assert torch.equal(replayed.get_momentum().view(torch.int32), eager.get_momentum().view(torch.int32)), f"v, step {i}"
+        assert torch.equal(replayed.bf16_shadow().view(torch.int16), eager.bf16_shadow().view(torch.int16)), f"shadow, step {i}"
+    mg.check()
+    replayed.sync()
+    replayed.set_stream(torch.cuda.current_stream())
