@@ -499,8 +499,8 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     Params r{};
     r.error_flag = h->error_flag;
     r.M = d_h; r.N = d_h; r.K = B; r.stages = stages_for(B);
-    // Replayed from a CUDA graph, the backward pass of the gradient call runs as two branches (the handle's own
-    // stream, forked from and joined to the caller's stream by events): measured 89.1 -> 82.8 us for the chain.
+    // Replayed from a CUDA graph, the backward pass runs as two branches (the handle's own stream, forked from and
+    // joined to the caller's stream by events): measured 89.1 -> 82.8 us for the chain of the gradient call.
     // Queued eagerly the same fork costs more in event calls than it gains (93.0 -> 94.2 us), so it is used under
     // stream capture only.
     const bool fork = (capturing != cudaStreamCaptureStatusNone);
@@ -509,10 +509,21 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     if (fused) {
         GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
         r.lr = fused->lr; r.mu = fused->mu; r.wd = fused->wd; r.has_shadow = fused->shadow != nullptr;
-        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, pdl)));
-        r.N = d_in;
-        GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1, pdl)));
-        // (the engine's small update beside these two kernels, on the second stream, was measured 7 us SLOWER)
+        if (fork) {     // the two update kernels touch disjoint parameters: side by side, their last waves fill up
+            if (cudaEventRecord(h->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h->side, h->ev_fork, 0) != cudaSuccess)
+                return COCOD_ERR_CUDA;
+            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, false)));
+            r.N = d_in;
+            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, h->side, &s_w1, false)));
+            if (cudaEventRecord(h->ev_join, h->side) != cudaSuccess || cudaStreamWaitEvent(s, h->ev_join, 0) != cudaSuccess)
+                return COCOD_ERR_CUDA;
+        } else {
+            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, pdl)));
+            r.N = d_in;
+            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1, pdl)));
+        }
+        // (the engine's small update on the second stream gained nothing: beside both kernels it cost 7 us, behind
+        // the shorter one it changed nothing)
         if (int rc = cocod_internal_step_segments(engine, grads, seg_lo, seg_hi, 2, nullptr)) return rc;
     } else if (fork) {
         // dW2 needs only dz2 and h1: it runs beside dz1 -> dW1.  dz1 is queued first and keeps a ring of three
