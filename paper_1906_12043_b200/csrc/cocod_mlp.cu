@@ -220,8 +220,8 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
 // Everything downstream of dz3 that runs on CUDA cores, for 32 hidden units j and all 128 samples:
 //   dz2[b][j] = bf16((sum_c dz3[b][c] W3[c][j]) * (h2[b][j] > 0)),  db2[j] = sum_b dz2[b][j],
 //   dW3[c][j] = sum_b dz3[b][c] h2[b][j];
-// the CTA with blockIdx.x == 0 also writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the
-// zero padding of the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32, K).
+// one extra CTA per worker writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the zero padding of
+// the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32 + 1, K).
 template <int DOUT, int NW>
 __global__ void __launch_bounds__(32 * NW)
 head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, const float *__restrict__ dz3,
@@ -230,6 +230,7 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
               int B, int d_h, int d_out)
 {
     // NW warps per CTA; warp wp owns samples wp, wp + NW, ...; DOUT bounds the class loops (>= d_out)
+    static_assert(NW >= 2, "the scalar CTA uses two warps");
     constexpr int C4 = (DOUT + 3) / 4;
     __shared__ __align__(16) float sdz[128 * 16];
     __shared__ float red[NW][16][33];
@@ -238,6 +239,34 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
     const int j = j0 + lane;
     pdl_launch_dependents();
     pdl_wait();
+    if (blockIdx.x == gridDim.x - 1) {
+        // The extra CTA of every worker: the per-worker scalars db3[c] = sum_b dz3[b][c], loss = mean_b rowloss and
+        // the zero padding of the gradient, each by one warp (lane-strided partial sums, then a fixed shuffle tree).
+        // As an epilogue of one of the column CTAs this made that CTA the straggler of the kernel (2.3 us).
+        for (int i = threadIdx.x; i < B * 16; i += 32 * NW) sdz[i] = dz3[(long long)w * B * 16 + i];
+        __syncthreads();
+        if (wp == 0) {
+            for (int c = 0; c < d_out; ++c) {
+                float s = 0.0f;
+                for (int b = lane; b < B; b += 32) s += sdz[b * 16 + c];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                if (lane == 0) grads[(long long)w * P + ob3 + c] = s;
+            }
+        } else if (wp == 1) {
+            float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (lane + 32 * i < B) t[i] = rowloss[(long long)w * B + lane + 32 * i];
+            float s = (t[0] + t[1]) + (t[2] + t[3]);
+            for (int b = lane + 128; b < B; b += 32) s += rowloss[(long long)w * B + b];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            if (lane == 0) loss[w] = s / (float)B;
+        }
+        for (long long i = P_raw + threadIdx.x; i < P; i += 32 * NW) grads[(long long)w * P + i] = 0.0f;
+        return;
+    }
     // first batch of this thread's h2 values: in flight while dz3 and W3 are fetched
     float hreg[16];
 #pragma unroll
@@ -305,29 +334,6 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
 #pragma unroll
         for (int q = 0; q < NW; ++q) s += colsum[q][threadIdx.x];
         grads[(long long)w * P + ob2 + j0 + threadIdx.x] = s;
-    }
-    if (blockIdx.x == 0) {
-        // per-worker scalars: each by one warp, lane-strided partial sums then a fixed shuffle tree
-        if (wp == 0) {
-            for (int c = 0; c < d_out; ++c) {
-                float s = 0.0f;
-                for (int b = lane; b < B; b += 32) s += sdz[b * 16 + c];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-                if (lane == 0) grads[(long long)w * P + ob3 + c] = s;
-            }
-        } else if (wp == 1) {
-            float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (lane + 32 * i < B) t[i] = rowloss[(long long)w * B + lane + 32 * i];
-            float s = (t[0] + t[1]) + (t[2] + t[3]);
-            for (int b = lane + 128; b < B; b += 32) s += rowloss[(long long)w * B + b];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-            if (lane == 0) loss[w] = s / (float)B;
-        }
-        for (long long i = P_raw + threadIdx.x; i < P; i += 32 * NW) grads[(long long)w * P + i] = 0.0f;
     }
 }
 
@@ -486,7 +492,7 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     const size_t w3_bytes = (size_t)d_out * d_h * sizeof(bf16);
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_logits<10> : head_logits<16>, dim3(B / 8, K), dim3(256), w3_bytes, s,
                              h->h2, prm, P, h->oW3, h->ob3, labels, h->dz3, h->rowloss, B, d_h, d_out));
-    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32, K),
+    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
                              dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->dz3, (const float *)h->rowloss,
                              h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
