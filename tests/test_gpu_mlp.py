@@ -409,3 +409,13 @@ def test_gradient_paths_replayed_from_a_cuda_graph_match_the_eager_calls(M, E, K
     mg.check()
     replayed.sync()
     replayed.set_stream(torch.cuda.current_stream())
+
+
+def test_a_single_class_gives_zero_loss_and_zero_gradient(M):
+    """Degenerate output layer: with one class softmax is 1, the loss 0 and every gradient exactly 0."""
+    K, dims = 3, (72, 256, 256, 1)
+    params, X, y, P_raw = make_dyadic_problem(K, dims, seed=3)
+    g, loss, _ = run_gpu_grad(M, K, dims, params, X, y)
+    assert np.all(g == 0) and np.all(loss == 0)
+    ref_loss, ref_g = MO.loss_and_grad(params[0], X[0], y[0], dims, emulate_bf16=True)
+    assert ref_loss == 0 and np.all(ref_g == 0)
