@@ -64,10 +64,10 @@ int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, 
  * the gradients are computed from its bf16 copy of x.  For the two weight matrices W1 and W2
  * (99.4 % of the parameters) the weight-gradient GEMMs apply the update d = g + wd x; v = mu v + d;
  * x = x - lr v in their epilogue: the gradient tile never leaves the SM, x, v and the bf16 copy are
- * read and written once.  The remaining tensors go through a small gradient buffer owned by the
- * handle and the engine's ordinary update.  Results are bit-identical to cocod_mlp_grad followed by
- * cocod_local_step.  Runs on the engine's compute stream; counts as one local step.  The first call
- * on a handle allocates that gradient buffer (K x P floats): make it outside any stream capture.
+ * read and written once.  The remaining tensors (biases, W3) take the same update inside the kernels
+ * that produce their gradients, so no gradient is ever written to memory.  Results are bit-identical
+ * to cocod_mlp_grad followed by cocod_local_step.  Runs on the engine's compute stream; counts as
+ * one local step.
  *   x, labels, loss: as for cocod_mlp_grad. */
 int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x, const int32_t *labels,
                         float *loss);

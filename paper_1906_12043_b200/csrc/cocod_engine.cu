@@ -1033,30 +1033,6 @@ int cocod_internal_plan_step(cocod_handle *h, cocod_step_plan *plan)
     return COCOD_OK;
 }
 
-int cocod_internal_step_segments(cocod_handle *h, const float *g, const int64_t *lo, const int64_t *hi, int nseg,
-                                 cudaStream_t stream)
-{
-    if (int rc = check_live(h)) return rc;
-    if (!g || !lo || !hi || nseg < 1 || nseg > 4) return COCOD_ERR_INVALID;
-    cocod::StepSegments seg{};
-    int64_t longest = 0;
-    for (int i = 0; i < nseg; ++i) {
-        if (lo[i] < 0 || hi[i] < lo[i] || hi[i] > h->P) return COCOD_ERR_INVALID;
-        seg.lo[i] = lo[i]; seg.hi[i] = hi[i];
-        longest = std::max(longest, hi[i] - lo[i]);
-    }
-    if (longest == 0) return COCOD_OK;
-    const float *x_in = h->buf[h->cur];
-    float *x_out = h->pending_flip ? h->buf[1 - h->cur] : h->buf[h->cur];
-    const unsigned gx = (unsigned)std::min<int64_t>((longest + cocod::kThreads - 1) / cocod::kThreads, 64);
-    cocod::local_step_segments<<<dim3(gx, (unsigned)nseg, (unsigned)h->K), cocod::kThreads, 0,
-                                 stream ? stream : h->compute>>>(
-        x_in, x_out, h->v, g, h->P, seg, h->lr, h->mu, h->wd, h->shadow);
-    CK(h, cudaGetLastError());
-    ++h->launches;
-    return COCOD_OK;
-}
-
 int cocod_internal_finish_step(cocod_handle *h, int kernels_launched)
 {
     if (int rc = check_live(h)) return rc;

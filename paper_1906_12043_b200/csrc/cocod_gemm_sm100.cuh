@@ -58,6 +58,29 @@ struct SgdMaps {
     CUtensorMap x_in, x_out, v, shadow;
 };
 
+// Where a kernel that has just produced a gradient element applies the local step itself (fused gradient +
+// update call): pointers to the worker-major K x P state, already offset to the tensor's first element.
+// x_in == nullptr: no update, the gradient is written out instead.
+struct StepTarget {
+    const float *x_in;
+    float *x_out;
+    float *v;
+    __nv_bfloat16 *shadow;             // may be nullptr
+    long long worker_stride;           // P
+    float lr, mu, wd;
+};
+// d = fma(wd, x, g); v = fma(mu, v, d); x = fma(-lr, v, x); shadow = bf16(x)   (the engine's arithmetic)
+__device__ __forceinline__ void step_element(const StepTarget &t, long long idx, float g)
+{
+    const float x = t.x_in[idx];
+    const float d = __fmaf_rn(t.wd, x, g);
+    const float vn = __fmaf_rn(t.mu, t.v[idx], d);
+    t.v[idx] = vn;
+    const float xn = __fmaf_rn(-t.lr, vn, x);
+    t.x_out[idx] = xn;
+    if (t.shadow != nullptr) t.shadow[idx] = __float2bfloat16_rn(xn);
+}
+
 struct Params {
     int M, N, K;                       // per-worker problem
     float *c;                          // EPI_F32
@@ -70,6 +93,7 @@ struct Params {
     long long mask_worker_stride;
     float *colsum;                     // EPI_MASK, optional: [N] column sums of the bf16 output (needs M <= 128)
     long long colsum_worker_stride;
+    StepTarget colsum_step;            // ... or (x_in != nullptr) the local step of that [N] tensor, the sums as gradient
     float lr, mu, wd;                  // EPI_SGD
     int has_shadow;                    // EPI_SGD: also write bf16(x)
     int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
@@ -510,7 +534,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     if (n0 + b * 64 < p.N) tma_store_3d(&map_c, smem_base + b * (BM * 128), n0 + b * 64, m0, wk);
                 tma_store_commit();
             }
-            if (EPI == EPI_MASK && p.colsum != nullptr) {
+            if (EPI == EPI_MASK && (p.colsum != nullptr || p.colsum_step.x_in != nullptr)) {
                 // the whole batch is in this tile: thread t adds column t of the staged tile over the rows, in row order
                 const int t = threadIdx.x;
                 if (t < BN && n0 + t < p.N) {
@@ -520,7 +544,8 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     float acc = 0.0f;
                     for (int rr = 0; rr < rows; ++rr)
                         acc += __bfloat162float(*reinterpret_cast<const __nv_bfloat16 *>(colp + rr * 128 + ((piece ^ (rr & 7)) << 4)));
-                    p.colsum[(long long)wk * p.colsum_worker_stride + n0 + t] = acc;
+                    if (p.colsum_step.x_in != nullptr) step_element(p.colsum_step, (long long)wk * p.colsum_step.worker_stride + n0 + t, acc);
+                    else p.colsum[(long long)wk * p.colsum_worker_stride + n0 + t] = acc;
                 }
             }
             if (threadIdx.x == 0) tma_store_wait_read<0>();      // shared memory must outlive the reads

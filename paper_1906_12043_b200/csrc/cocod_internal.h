@@ -21,11 +21,5 @@ struct cocod_step_plan {
 // Describe the local step the engine would run now.  Fails like cocod_local_step would.
 int cocod_internal_plan_step(cocod_handle *h, cocod_step_plan *plan);
 
-// Run the engine's local-step arithmetic on up to `nseg` column ranges [lo, hi) of every worker
-// (gradients in a K x P matrix g), on `stream` (NULL = the compute stream; another stream must be ordered
-// against the compute stream by the caller).  Used for the parameters a fused caller does not update itself.
-int cocod_internal_step_segments(cocod_handle *h, const float *g, const int64_t *lo, const int64_t *hi, int nseg,
-                                 cudaStream_t stream);
-
 // Account for a completed local step (buffer flip, step counter).
 int cocod_internal_finish_step(cocod_handle *h, int kernels_launched);

@@ -140,28 +140,6 @@ local_step_scalar(const float *x_in, float *x_out, float *v, const float *__rest
     }
 }
 
-// Same update on column ranges [lo[s], hi[s]) of every worker: grid (blocks, nseg, K).
-struct StepSegments {
-    int64_t lo[4], hi[4];
-};
-static __global__ void __launch_bounds__(kThreads)
-local_step_segments(const float *x_in, float *x_out, float *v, const float *__restrict__ g, int64_t P,
-                    StepSegments seg, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
-{
-    const int64_t lo = seg.lo[blockIdx.y], n = seg.hi[blockIdx.y] - lo;
-    const int64_t base = (int64_t)blockIdx.z * P + lo;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; j < n; j += stride) {
-        const int64_t e = base + j;
-        const float d = __fmaf_rn(wd, x_in[e], g[e]);
-        const float vn = __fmaf_rn(mu, v[e], d);
-        v[e] = vn;
-        const float xn = __fmaf_rn(-lr, vn, x_in[e]);
-        x_out[e] = xn;
-        if (shadow != nullptr) shadow[e] = __float2bfloat16_rn(xn);
-    }
-}
-
 // ------------------------------------------------------------------------------------------ stored copy (Step I)
 template <int UNROLL>
 __global__ void __launch_bounds__(kThreads)

@@ -224,11 +224,14 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
 // the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32 + 1, K).
 template <int DOUT, int NW>
 __global__ void __launch_bounds__(32 * NW)
-head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, const float *__restrict__ dz3,
+head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__restrict__ dz3,
               const float *__restrict__ rowloss, bf16 *__restrict__ dz2, float *__restrict__ grads,
               float *__restrict__ loss, long long P, long long P_raw, long long oW3, long long ob2, long long ob3,
-              int B, int d_h, int d_out)
+              int B, int d_h, int d_out, const StepTarget step)
 {
+    // step.x_in != nullptr: instead of writing dW3, db2, db3 (and the zero padding) to `grads`, apply the local
+    // step to those parameters here (indices are flat positions in the K x P state).  Every CTA reads and
+    // updates only its own columns of W3, so the update cannot disturb another CTA's reads.
     // NW warps per CTA; warp wp owns samples wp, wp + NW, ...; DOUT bounds the class loops (>= d_out)
     static_assert(NW >= 2, "the scalar CTA uses two warps");
     constexpr int C4 = (DOUT + 3) / 4;
@@ -251,7 +254,10 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
                 for (int b = lane; b < B; b += 32) s += sdz[b * 16 + c];
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-                if (lane == 0) grads[(long long)w * P + ob3 + c] = s;
+                if (lane == 0) {
+                    if (step.x_in != nullptr) step_element(step, (long long)w * P + ob3 + c, s);
+                    else grads[(long long)w * P + ob3 + c] = s;
+                }
             }
         } else if (wp == 1) {
             float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -264,7 +270,10 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             if (lane == 0) loss[w] = s / (float)B;
         }
-        for (long long i = P_raw + threadIdx.x; i < P; i += 32 * NW) grads[(long long)w * P + i] = 0.0f;
+        for (long long i = P_raw + threadIdx.x; i < P; i += 32 * NW) {
+            if (step.x_in != nullptr) step_element(step, (long long)w * P + i, 0.0f);
+            else grads[(long long)w * P + i] = 0.0f;
+        }
         return;
     }
     // first batch of this thread's h2 values: in flight while dz3 and W3 are fetched
@@ -326,14 +335,18 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, cons
             float s = 0.0f;
 #pragma unroll
             for (int q = 0; q < NW; ++q) s += red[q][c][l];
-            grads[(long long)w * P + oW3 + (long long)c * d_h + j0 + l] = s;
+            const long long idx = (long long)w * P + oW3 + (long long)c * d_h + j0 + l;
+            if (step.x_in != nullptr) step_element(step, idx, s);
+            else grads[idx] = s;
         }
     }
     if (threadIdx.x < 32) {
         float s = 0.0f;
 #pragma unroll
         for (int q = 0; q < NW; ++q) s += colsum[q][threadIdx.x];
-        grads[(long long)w * P + ob2 + j0 + threadIdx.x] = s;
+        const long long idx = (long long)w * P + ob2 + j0 + threadIdx.x;
+        if (step.x_in != nullptr) step_element(step, idx, s);
+        else grads[idx] = s;
     }
 }
 
@@ -345,7 +358,6 @@ struct cocod_mlp {
     bf16 *h1 = nullptr, *h2 = nullptr, *dz2 = nullptr, *dz1 = nullptr;
     float *dz3 = nullptr, *rowloss = nullptr;
     int *error_flag = nullptr;
-    float *gscratch = nullptr;          // K x P gradients of the fused path's small tensors (allocated on first use)
     // maps over scratch (fixed addresses): reduction-contiguous (k) and row-contiguous (mn) views
     CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
     CUtensorMap st_h2, st_dz1;          // store views (64 columns x 128 rows) of outputs that are not read that way
@@ -360,7 +372,7 @@ namespace {
 
 void mlp_free(cocod_mlp *h)
 {
-    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag, h->gscratch};
+    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
@@ -447,7 +459,7 @@ namespace {
 // otherwise their GEMMs apply the engine's local step in their epilogue (x, v and the bf16 copy of x
 // are updated in place, nothing is written to `grads` for W1 and W2).
 int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labels, float *grads, float *loss,
-             cudaStream_t s, const cocod_step_plan *fused, cocod_handle *engine = nullptr)
+             cudaStream_t s, const cocod_step_plan *fused)
 {
     const int K = h->K, B = h->B, d_in = h->d_in, d_h = h->d_h, d_out = h->d_out;
     const long long P = h->P;
@@ -479,6 +491,13 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) return COCOD_ERR_CUDA;
     const bool pdl = (capturing == cudaStreamCaptureStatusNone);
+    // fused call: the small tensors (biases, W3, padding) take their local step inside the kernels that produce
+    // their gradients; otherwise those kernels write the gradients out
+    StepTarget small{};
+    if (fused) {
+        small.x_in = fused->x_in; small.x_out = fused->x_out; small.v = fused->v; small.shadow = fused->shadow;
+        small.worker_stride = P; small.lr = fused->lr; small.mu = fused->mu; small.wd = fused->wd;
+    }
     Params p{};
     p.error_flag = h->error_flag;
     // h1 = relu(x W1^T + b1)
@@ -494,13 +513,20 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
                              h->h2, prm, P, h->oW3, h->ob3, labels, h->dz3, h->rowloss, B, d_h, d_out));
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
                              dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->dz3, (const float *)h->rowloss,
-                             h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out));
+                             h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out, small));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
     Params q{};
     q.error_flag = h->error_flag;
     q.M = B; q.N = d_h; q.K = d_h; q.stages = stages_for(d_h);
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
-    q.colsum = grads + h->ob1; q.colsum_worker_stride = P;      // db1 = column sums of dz1, from the same epilogue
+    // db1 = column sums of dz1, from the same epilogue
+    if (!fused) {
+        q.colsum = grads + h->ob1; q.colsum_worker_stride = P;
+    } else {                                                      // ... applied to b1 on the spot
+        q.colsum_step = small;
+        q.colsum_step.x_in += h->ob1; q.colsum_step.x_out += h->ob1; q.colsum_step.v += h->ob1;
+        if (q.colsum_step.shadow) q.colsum_step.shadow += h->ob1;
+    }
     // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
     Params r{};
     r.error_flag = h->error_flag;
@@ -510,8 +536,6 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     // Queued eagerly the same fork costs more in event calls than it gains (93.0 -> 94.2 us), so it is used under
     // stream capture only.
     const bool fork = (capturing != cudaStreamCaptureStatusNone);
-    // everything but W1 and W2 (b1, then b2 | W3 | b3 | padding) is updated by the engine's own kernel
-    const int64_t seg_lo[2] = {h->ob1, h->ob2}, seg_hi[2] = {h->oW2, h->P};
     if (fused) {
         GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
         r.lr = fused->lr; r.mu = fused->mu; r.wd = fused->wd; r.has_shadow = fused->shadow != nullptr;
@@ -528,9 +552,6 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
             r.N = d_in;
             GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1, pdl)));
         }
-        // (the engine's small update on the second stream gained nothing: beside both kernels it cost 7 us, behind
-        // the shorter one it changed nothing)
-        if (int rc = cocod_internal_step_segments(engine, grads, seg_lo, seg_hi, 2, nullptr)) return rc;
     } else if (fork) {
         // dW2 needs only dz2 and h1: it runs beside dz1 -> dW1.  dz1 is queued first and keeps a ring of three
         // stages here, so that a CTA of dW2 fits next to it on the same SM (2, 4 and 6 stages measured slower).
@@ -579,18 +600,9 @@ int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x
     if (int rc = cocod_internal_plan_step(engine, &plan)) return rc;
     if (plan.K != h->K || plan.P != h->P) return COCOD_ERR_INVALID;
     if (!plan.shadow) return COCOD_ERR_STATE;            // the gradients are computed from the bf16 copy of x
-    if (!h->gscratch) {
-        if (cudaMalloc((void **)&h->gscratch, (size_t)h->K * h->P * sizeof(float)) != cudaSuccess) {
-            cudaGetLastError();
-            h->gscratch = nullptr;
-            return COCOD_ERR_OOM;
-        }
-    }
-    const long long before = h->launches;
-    if (int rc = run_grad(h, plan.shadow, static_cast<const bf16 *>(x), labels, h->gscratch, loss, plan.compute, &plan,
-                          engine))
+    // no gradient buffer: every tensor takes its local step inside the kernel that produces its gradient
+    if (int rc = run_grad(h, plan.shadow, static_cast<const bf16 *>(x), labels, nullptr, loss, plan.compute, &plan))
         return rc;
-    (void)before;
     return cocod_internal_finish_step(engine, 0);
 }
 

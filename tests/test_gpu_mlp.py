@@ -387,12 +387,6 @@ def test_gradient_paths_replayed_from_a_cuda_graph_match_the_eager_calls(M, E, K
         assert torch.equal(l_g, l_e)
     # ---- fused gradient + update: three steps eagerly, three replays of one captured step
     l1 = torch.empty(K, dtype=torch.float32, device="cuda")
-    scratch = E.Engine(K, P, lr, mu, wd)                 # the handle's first fused call allocates: not under capture
-    scratch.set_option(E.OPT_BF16_SHADOW, 1)
-    scratch.set_params(x0)
-    mg.grad_step(scratch, X, y, l1)
-    scratch.sync()
-    scratch.destroy()
     replayed.sync()
     replayed.set_stream(cap)
     step = torch.cuda.CUDAGraph()
