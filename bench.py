@@ -615,24 +615,45 @@ def run_mlp(args):
         eng.set_stream(compute)
     final_loss = float(loss.mean().item())
 
-    # end to end: minibatches and labels start in pinned host memory, the loss comes back every step
-    x_dev, y_dev = torch.empty_like(xs_d[0]), torch.empty_like(ys_d[0])
+    # end to end: minibatches and labels start in pinned host memory, the loss comes back every step.  The upload
+    # of step t + 1 (copy stream, two device buffers) runs under the kernels of step t.
+    copy_stream = torch.cuda.Stream()
+    x_buf = [torch.empty_like(xs_d[0]) for _ in range(2)]
+    y_buf = [torch.empty_like(ys_d[0]) for _ in range(2)]
+    ev_up = [torch.cuda.Event() for _ in range(2)]
+    ev_used = [torch.cuda.Event() for _ in range(2)]
     loss_h = torch.empty(K, dtype=torch.float32, pin_memory=True)
     n_e2e = max(1, min(args.steps, 50))
+    up_no = [0]
+
+    def upload():
+        slot, i = up_no[0] % 2, up_no[0] % ring_n
+        with torch.cuda.stream(copy_stream):
+            if up_no[0] >= 2:
+                copy_stream.wait_event(ev_used[slot])          # the kernels that read this buffer are done
+            x_buf[slot].copy_(xs_h[i], non_blocking=True)
+            y_buf[slot].copy_(ys_h[i], non_blocking=True)
+            ev_up[slot].record(copy_stream)
+        up_no[0] += 1
+
+    torch.cuda.synchronize()
+    upload()
+    host_step = [0]
 
     def one_round_host():
         eng.comm_begin(side)
         for _ in range(k):
-            i = step_no[0] % ring_n
-            x_dev.copy_(xs_h[i], non_blocking=True)
-            y_dev.copy_(ys_h[i], non_blocking=True)
+            slot = host_step[0] % 2
+            upload()                                           # next step's inputs
+            compute.wait_event(ev_up[slot])
             if args.fused:
-                mg.grad_step(eng, x_dev, y_dev, loss)
+                mg.grad_step(eng, x_buf[slot], y_buf[slot], loss)
             else:
-                mg.grad(shadow, x_dev, y_dev, grads, loss)
+                mg.grad(shadow, x_buf[slot], y_buf[slot], grads, loss)
                 eng.local_step(grads)
+            ev_used[slot].record(compute)
             loss_h.copy_(loss, non_blocking=True)
-            step_no[0] += 1
+            host_step[0] += 1
         eng.comm_end()
 
     for _ in range(2):
