@@ -485,12 +485,14 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     }
 #define LAUNCH_OK() do { if (cudaGetLastError() != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
 #define GEMM_OK(call) do { if ((call) != cudaSuccess) return COCOD_ERR_CUDA; ++h->launches; } while (0)
-    // Each kernel of the chain may set up while its predecessor drains (programmatic dependent launch):
-    // 11 % off the eager chain.  Not while the stream is being captured: replayed from a graph the chain
-    // measured 1.5 % slower with these edges than without.
+    // Each kernel of the chain may set up while its predecessor drains (programmatic dependent launch): 11 % off
+    // the eager chain.  Under stream capture only the two forward GEMMs keep these edges: measured edge by edge in a
+    // replayed graph, they gain 1.1 and 0.8 us there, while the edges into the two output-layer kernels and into the
+    // backward GEMMs cost 1.5 - 2.7 us each.
     cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) return COCOD_ERR_CUDA;
     const bool pdl = (capturing == cudaStreamCaptureStatusNone);
+    const bool pdl_fwd = true;
     // fused call: the small tensors (biases, W3, padding) take their local step inside the kernels that produce
     // their gradients; otherwise those kernels write the gradients out
     StepTarget small{};
@@ -503,10 +505,10 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     // h1 = relu(x W1^T + b1)
     p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
     p.bias = prm + h->ob1; p.bias_worker_stride = P;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, nullptr, pdl)));
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, nullptr, pdl_fwd)));
     // h2 = relu(h1 W2^T + b2)
     p.K = d_h; p.stages = stages_for(d_h); p.bias = prm + h->ob2;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, nullptr, pdl)));
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, nullptr, pdl_fwd)));
     // output layer, loss, dz3; then dz2, dW3, db3, db2
     const size_t w3_bytes = (size_t)d_out * d_h * sizeof(bf16);
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_logits<10> : head_logits<16>, dim3(B / 8, K), dim3(256), w3_bytes, s,
