@@ -129,6 +129,7 @@ inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK -
 // warps per CTA of head_backward (measured inside the gradient chain: 2 warps 20.3 us, 4 warps 14.3 us,
 // 8 warps 15.9 us; about 8 us of it is fixed cost, not the loop over the samples)
 constexpr int HEAD_NW = 4;
+constexpr int HEAD_COLS = 64;       // hidden units per CTA of head_backward: two adjacent ones per thread
 // Output layer forward and loss.  One CTA = 8 samples of one worker (one per warp); W3 sits in shared
 // memory; every lane loads its slices of the h2 row up front (all loads in flight at once):
 // logits = h2 W3^T + b3 (fp32), row loss = -log softmax[label], dz3 = bf16((softmax - onehot) / batch)
@@ -217,11 +218,11 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
     if (lane == 0) rowloss[(long long)w * B + b] = -logf(py);
 }
 
-// Everything downstream of dz3 that runs on CUDA cores, for 32 hidden units j and all 128 samples:
+// Everything downstream of dz3 that runs on CUDA cores, for 64 hidden units j and all 128 samples:
 //   dz2[b][j] = bf16((sum_c dz3[b][c] W3[c][j]) * (h2[b][j] > 0)),  db2[j] = sum_b dz2[b][j],
 //   dW3[c][j] = sum_b dz3[b][c] h2[b][j];
 // one extra CTA per worker writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the zero padding of
-// the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32 + 1, K).
+// the gradient.  Fixed summation orders (deterministic).  grid (d_h / 64 + 1, K).
 template <int DOUT, int NW>
 __global__ void __launch_bounds__(32 * NW)
 head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__restrict__ dz3,
@@ -236,10 +237,10 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
     static_assert(NW >= 2, "the scalar CTA uses two warps");
     constexpr int C4 = (DOUT + 3) / 4;
     __shared__ __align__(16) float sdz[128 * 16];
-    __shared__ float red[NW][16][33];
-    __shared__ float colsum[NW][33];
-    const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
-    const int j = j0 + lane;
+    __shared__ float red[NW][16][HEAD_COLS + 2];
+    __shared__ float colsum[NW][HEAD_COLS + 2];
+    const int w = blockIdx.y, j0 = blockIdx.x * HEAD_COLS, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+    const int j = j0 + 2 * lane;
     pdl_launch_dependents();
     pdl_wait();
     if (blockIdx.x == gridDim.x - 1) {
@@ -276,36 +277,41 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
         }
         return;
     }
-    // first batch of this thread's h2 values: in flight while dz3 and W3 are fetched
-    float hreg[16];
+    // first batch of this thread's h2 values (two adjacent hidden units per thread: 128-byte lines per warp):
+    // in flight while dz3 and W3 are fetched
+    float2 hreg[16];
 #pragma unroll
     for (int q = 0; q < 16; ++q) {
         const int b = wp + NW * q;
-        hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
+        hreg[q] = (b < B) ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(h2 + ((long long)w * B + b) * d_h + j))
+                          : make_float2(0.0f, 0.0f);
     }
     for (int i = threadIdx.x; i < B * 16; i += 32 * NW) sdz[i] = dz3[(long long)w * B * 16 + i];
-    float w3[4 * C4], acc3[4 * C4];
+    float2 w3[4 * C4], acc3[4 * C4];
 #pragma unroll
     for (int c = 0; c < 4 * C4; ++c) {
-        w3[c] = (c < d_out) ? __bfloat162float(params[(long long)w * P + oW3 + (long long)c * d_h + j]) : 0.0f;
-        acc3[c] = 0.0f;
+        w3[c] = (c < d_out) ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(
+                                  params + (long long)w * P + oW3 + (long long)c * d_h + j))
+                            : make_float2(0.0f, 0.0f);
+        acc3[c] = make_float2(0.0f, 0.0f);
     }
     __syncthreads();
-    float csum = 0.0f;
+    float2 csum = make_float2(0.0f, 0.0f);
     for (int q0 = 0; q0 * NW < B; q0 += 16) {
         if (q0 > 0) {
 #pragma unroll
             for (int q = 0; q < 16; ++q) {
                 const int b = wp + NW * (q0 + q);
-                hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
+                hreg[q] = (b < B) ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(h2 + ((long long)w * B + b) * d_h + j))
+                                  : make_float2(0.0f, 0.0f);
             }
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const int b = wp + NW * (q0 + q);
             if (b < B) {
-                const float h = hreg[q];
-                float a = 0.0f;
+                const float2 h = hreg[q];
+                float2 a = make_float2(0.0f, 0.0f);
                 const float4 *d4 = reinterpret_cast<const float4 *>(sdz + b * 16);
 #pragma unroll
                 for (int c4 = 0; c4 < C4; ++c4) {
@@ -314,23 +320,31 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         if (4 * c4 + e < DOUT) {
-                            a = fmaf(d[e], w3[4 * c4 + e], a);
-                            acc3[4 * c4 + e] = fmaf(d[e], h, acc3[4 * c4 + e]);
+                            a.x = fmaf(d[e], w3[4 * c4 + e].x, a.x);
+                            a.y = fmaf(d[e], w3[4 * c4 + e].y, a.y);
+                            acc3[4 * c4 + e].x = fmaf(d[e], h.x, acc3[4 * c4 + e].x);
+                            acc3[4 * c4 + e].y = fmaf(d[e], h.y, acc3[4 * c4 + e].y);
                         }
                     }
                 }
-                const bf16 v = __float2bfloat16_rn(h > 0.0f ? a : 0.0f);
-                dz2[((long long)w * B + b) * d_h + j] = v;
-                csum += __bfloat162float(v);
+                const __nv_bfloat162 v = __floats2bfloat162_rn(h.x > 0.0f ? a.x : 0.0f, h.y > 0.0f ? a.y : 0.0f);
+                *reinterpret_cast<__nv_bfloat162 *>(dz2 + ((long long)w * B + b) * d_h + j) = v;
+                const float2 vf = __bfloat1622float2(v);
+                csum.x += vf.x;
+                csum.y += vf.y;
             }
         }
     }
 #pragma unroll
-    for (int c = 0; c < 16; ++c) red[wp][c][lane] = (c < DOUT) ? acc3[c < DOUT ? c : 0] : 0.0f;
-    colsum[wp][lane] = csum;
+    for (int c = 0; c < 16; ++c) {
+        red[wp][c][2 * lane] = (c < DOUT) ? acc3[c < DOUT ? c : 0].x : 0.0f;
+        red[wp][c][2 * lane + 1] = (c < DOUT) ? acc3[c < DOUT ? c : 0].y : 0.0f;
+    }
+    colsum[wp][2 * lane] = csum.x;
+    colsum[wp][2 * lane + 1] = csum.y;
     __syncthreads();
-    for (int i = threadIdx.x; i < 16 * 32; i += 32 * NW) {
-        const int c = i >> 5, l = i & 31;
+    for (int i = threadIdx.x; i < 16 * HEAD_COLS; i += 32 * NW) {
+        const int c = i / HEAD_COLS, l = i % HEAD_COLS;
         if (c < d_out) {
             float s = 0.0f;
 #pragma unroll
@@ -340,7 +354,7 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
             else grads[idx] = s;
         }
     }
-    if (threadIdx.x < 32) {
+    if (threadIdx.x < HEAD_COLS) {
         float s = 0.0f;
 #pragma unroll
         for (int q = 0; q < NW; ++q) s += colsum[q][threadIdx.x];
@@ -513,7 +527,7 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     const size_t w3_bytes = (size_t)d_out * d_h * sizeof(bf16);
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_logits<10> : head_logits<16>, dim3(B / 8, K), dim3(256), w3_bytes, s,
                              h->h2, prm, P, h->oW3, h->ob3, labels, h->dz3, h->rowloss, B, d_h, d_out));
-    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
+    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / HEAD_COLS + 1, K),
                              dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->dz3, (const float *)h->rowloss,
                              h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out, small));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
