@@ -152,6 +152,14 @@ def test_config1_full_vector_parity(E, snapshot):
                              snapshot=snapshot, check_round=check)
     assert_bit_equal(cpu(eng.get_mean()), mir.mean, "last average model")
     print("config1 worst scaled errors (x, v) by round:", worst)
+    # context figures after the full run: plain relative error (unscaled, so elements near zero dominate) and the
+    # distance to the fp32 mirror in units in the last place
+    x = cpu(eng.get_params()).astype(np.float64)
+    rel = np.abs(x - ref.x) / np.maximum(np.abs(ref.x.astype(np.float64)), 1e-300)
+    ulps = np.abs(cpu(eng.get_params()).view(np.int32).astype(np.int64) - mir.x.view(np.int32).astype(np.int64))
+    print(f"config1 after the run: max relative error {rel.max():.3e}, 99.99th percentile {np.quantile(rel, 0.9999):.3e}, "
+          f"max distance to the mirror {int(ulps.max())} ulp")
+    assert ulps.max() == 0 and np.quantile(rel, 0.9999) < 1e-3
 
 
 # ----------------------------------------------------------------------------- shapes: tiles, ragged tails, misaligned rows
