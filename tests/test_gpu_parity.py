@@ -657,3 +657,18 @@ def test_buffers_next_to_engine_inputs_are_untouched(E):
     eng.sync()
     assert torch.isnan(big[:pad]).all() and torch.isnan(big[pad + K * P:]).all()
     assert torch.isfinite(eng.get_params()).all()
+
+
+def test_a_request_beyond_the_device_memory_fails_cleanly(E):
+    """cocod_create with buffers that cannot exist (256 GB each): out-of-memory error code, nothing leaked,
+    and the device is as usable as before."""
+    free_before = torch.cuda.mem_get_info()[0]
+    with pytest.raises(E.CocodError) as e:
+        E.Engine(16, 4_000_000_000, 0.1, 0.9, 0.0)
+    assert e.value.code == E.ERR_OOM
+    assert abs(torch.cuda.mem_get_info()[0] - free_before) < (64 << 20)
+    eng = E.Engine(2, 1024, 0.1, 0.0, 0.0)
+    eng.set_params(np.ones(1024, np.float32))
+    eng.local_step(torch.ones(2, 1024, device="cuda"))
+    assert np.allclose(cpu(eng.get_params()), 0.9)
+    eng.destroy()
