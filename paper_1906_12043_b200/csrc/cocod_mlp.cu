@@ -15,6 +15,7 @@
 //   dW1 = dz1^T x                     GEMM d_h x d_in x 128   A = dz1 read [k][m], B = x  read [k][n]   fp32 out
 #include "cocod_mlp.h"
 #include "cocod_gemm_sm100.cuh"
+#include "cocod_gemm_update_sm100.cuh"
 #include "cocod_internal.h"
 
 #include <algorithm>
@@ -121,6 +122,23 @@ cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtens
     const dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, workers);
     return launch_dependent(pdl, gemm_bf16<EPI, A_MN, B_MN, NT>, grid, dim3(NT), (size_t)need, s, a, b, c,
                             sgd ? *sgd : no_sgd, p);
+}
+
+// The persistent gradient + update kernel over the tiles of up to two weight matrices.
+cudaError_t launch_update(const UpdateProblem &p0, const UpdateProblem &p1, const UpdateParams &q, cudaStream_t s, bool pdl)
+{
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_update_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM);
+        if (e != cudaSuccess) { sms = 0; return e; }
+    }
+    const int total = p0.tiles + p1.tiles;
+    if (total <= 0) return cudaSuccess;
+    return launch_dependent(pdl, gemm_update_persistent, dim3(std::min(total, sms)), dim3(UPD_THREADS), (size_t)UPD_SMEM, s,
+                            p0, p1, q);
 }
 
 inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK - 1) / BK)); }
@@ -554,6 +572,22 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     const bool fork = (capturing != cudaStreamCaptureStatusNone);
     if (fused) {
         GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
+        if (B <= 2 * BK) {
+            // one persistent kernel walks the tiles of W2 and then of W1 (loads of a tile under the update and the
+            // store drain of the tile before it)
+            UpdateProblem u2{}, u1{};
+            u2.a = h->mn_dz2; u2.b = h->mn_h1; u2.x_in = s_w2.x_in; u2.x_out = s_w2.x_out; u2.v = s_w2.v;
+            u2.shadow = s_w2.shadow; u2.has_shadow = fused->shadow != nullptr;
+            u2.M = d_h; u2.N = d_h; u2.tiles_m = (d_h + BM - 1) / BM; u2.tiles_n = (d_h + BN - 1) / BN;
+            u2.tiles = K * u2.tiles_m * u2.tiles_n;
+            u1.a = h->mn_dz1; u1.b = mn_x; u1.x_in = s_w1.x_in; u1.x_out = s_w1.x_out; u1.v = s_w1.v;
+            u1.shadow = s_w1.shadow; u1.has_shadow = fused->shadow != nullptr;
+            u1.M = d_h; u1.N = d_in; u1.tiles_m = (d_h + BM - 1) / BM; u1.tiles_n = (d_in + BN - 1) / BN;
+            u1.tiles = K * u1.tiles_m * u1.tiles_n;
+            UpdateParams uq{};
+            uq.K = B; uq.lr = fused->lr; uq.mu = fused->mu; uq.wd = fused->wd; uq.error_flag = h->error_flag;
+            GEMM_OK(launch_update(u2, u1, uq, s, pdl));
+        } else {
         r.lr = fused->lr; r.mu = fused->mu; r.wd = fused->wd; r.has_shadow = fused->shadow != nullptr;
         if (fork) {     // the two update kernels touch disjoint parameters: side by side, their last waves fill up
             if (cudaEventRecord(h->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h->side, h->ev_fork, 0) != cudaSuccess)
@@ -567,6 +601,7 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
             GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, pdl)));
             r.N = d_in;
             GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1, pdl)));
+        }
         }
     } else if (fork) {
         // dW2 needs only dz2 and h1: it runs beside dz1 -> dW1.  dz1 is queued first and keeps a ring of three
