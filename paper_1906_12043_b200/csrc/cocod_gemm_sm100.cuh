@@ -40,22 +40,13 @@ constexpr int MAX_STAGES = STAGES;
 // slack + a tail holding the barriers (256 B) and the bias tile (512 B)
 __host__ __device__ constexpr int ring_stages(int stages) { return stages < 2 ? 2 : stages; }
 __host__ __device__ constexpr int smem_bytes(int stages) { return ring_stages(stages) * STAGE_BYTES + 1024 + 1024; }
-// the update epilogue additionally keeps the x and v tiles (128 x 128 fp32 each)
-__host__ __device__ constexpr int smem_bytes_sgd(int stages) { return smem_bytes(stages) + 2 * BM * BN * 4; }
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Epilogue {
     EPI_F32 = 0,        // c[m][n] = acc                         (fp32, row stride ldc; TMA store if map_c_ok)
     EPI_BIAS_RELU = 1,  // o[m][n] = bf16(max(acc + bias[n], 0))          (o = the bf16 matrix map_c describes: boxes of
-    EPI_MASK = 2,       // o[m][n] = bf16(acc * (mask[m][n] > 0));         64 columns x 128 rows, 128-byte swizzle)
+    EPI_MASK = 2        // o[m][n] = bf16(acc * (mask[m][n] > 0));         64 columns x 128 rows, 128-byte swizzle)
                         // optionally colsum[n] = sum_m o[m][n] (M <= 128)
-    EPI_SGD = 3         // g = acc: d = fma(wd, x, g); v = fma(mu, v, d); x = fma(-lr, v, x); shadow = bf16(x)
-};
-
-// Tensor maps of the update epilogue: fp32 [M][N] tiles of 32 columns x 128 rows (x read, x written,
-// v) and the bf16 copy of x in tiles of 64 columns x 128 rows; all with the 128-byte swizzle.
-struct SgdMaps {
-    CUtensorMap x_in, x_out, v, shadow;
 };
 
 // Where a kernel that has just produced a gradient element applies the local step itself (fused gradient +
@@ -94,8 +85,6 @@ struct Params {
     float *colsum;                     // EPI_MASK, optional: [N] column sums of the bf16 output (needs M <= 128)
     long long colsum_worker_stride;
     StepTarget colsum_step;            // ... or (x_in != nullptr) the local step of that [N] tensor, the sums as gradient
-    float lr, mu, wd;                  // EPI_SGD
-    int has_shadow;                    // EPI_SGD: also write bf16(x)
     int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
@@ -245,23 +234,19 @@ __host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn)
 // Tensor maps: a K-major operand is {k (contiguous), rows, workers} with box {64, 128, 1}; an
 // MN-major operand is {m or n (contiguous), k, workers} with box {64, 64, 1} (two boxes per tile).
 // map_c (EPI_F32 only): {n (contiguous), m, workers} fp32 with box {32, 128, 1}, 128-byte swizzle.
-// NT threads per CTA: 128 (every thread drains one accumulator row) or 256 (two threads share a row, each
-// draining 64 columns: used where the epilogue is long and only one CTA fits per SM).
+// NT threads per CTA: 128 (every thread drains one accumulator row; 256 would let two threads share a row).
 template <int EPI, bool A_MN, bool B_MN, int NT>
 __global__ void __launch_bounds__(NT)
 gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-          const __grid_constant__ CUtensorMap map_c, const __grid_constant__ SgdMaps sgd, const Params p)
+          const __grid_constant__ CUtensorMap map_c, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     if (threadIdx.x == 0) COCOD_TRACE(0);
     const int stages = p.stages;
-    uint8_t *xs = smem + ring_stages(stages) * STAGE_BYTES;        // EPI_SGD: x tile, then v tile
-    uint8_t *vs = xs + BM * BN * 4;
-    uint8_t *tail = (EPI == EPI_SGD) ? vs + BM * BN * 4 : xs;
+    uint8_t *tail = smem + ring_stages(stages) * STAGE_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(tail);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + MAX_STAGES), accum = smem_u32(bars + 2 * MAX_STAGES);
-    const uint32_t aux = smem_u32(bars + 2 * MAX_STAGES + 1);      // EPI_SGD: four barriers, one per 32-column chunk of x and v
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * MAX_STAGES + 5);
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
@@ -303,7 +288,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum, 1);
-        for (int c = 0; c < 4; ++c) mbar_init(aux + 8 * c, 1);
         abort[0] = 0;
         abort[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -312,15 +296,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // the first ring of copies starts now, under the rest of the set-up
         if (!p.debug_no_loads)
             for (; armed < nkb && armed < stages; ++armed) issue_loads(armed, armed);
-        if (EPI == EPI_SGD) {         // the tiles the update needs: in flight under the whole main loop
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&sgd.x_out) : "memory");
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                mbar_expect_tx(aux + 8 * c, 2 * BM * 128);
-                tma_load_3d(smem_u32(xs) + c * (BM * 128), &sgd.x_in, aux + 8 * c, n0 + c * 32, m0, wk);
-                tma_load_3d(smem_u32(vs) + c * (BM * 128), &sgd.v, aux + 8 * c, n0 + c * 32, m0, wk);
-            }
-        }
     }
     if (threadIdx.x == 0) COCOD_TRACE(6);
     __syncwarp();
@@ -411,9 +386,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     // ---- epilogue: every thread owns one accumulator row (TMEM lane) of the tile
     bool ok = mbar_wait(accum, 0, abort, limit + limit / 2);
 
-    if (EPI == EPI_SGD && !ok) {                                  // issued copies must land in any case
-        for (int c = 0; c < 4; ++c) mbar_wait(aux + 8 * c, 0, never, limit);
-    }
     ok = __all_sync(0xffffffffu, ok);
     if (__syncthreads_and(ok ? 1 : 0)) {          // (also makes sbias visible)
         if (threadIdx.x == 0) COCOD_TRACE(4);
@@ -423,51 +395,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
         for (int cc = 0; cc < NCH; ++cc) tmem_ld32(trow + cc * 32, r[cc]);
         tmem_ld_wait();
-        if (EPI == EPI_SGD) {
-            // gradient = accumulator; x and v tiles sit in shared memory in the TMA swizzle (16-byte piece
-            // j of row r at piece j ^ (r & 7)); the bf16 copy of x is staged in the idle ring.
-            // Chunks are handed to the store engine one by one: the 128 threads that share a chunk
-            // meet on a named barrier and their first thread issues that chunk's bulk stores while the
-            // others already update the next chunk.
-            uint8_t *ss = smem;
-            const int group = warp >> 2;                       // 128-thread group (NT == 256: two of them)
-            const bool leader = (threadIdx.x & 127) == 0;
-            bool landed = true;
-#pragma unroll
-            for (int cc = 0; cc < NCH; ++cc) {
-                const int c = cbase + cc;
-                landed = mbar_wait(aux + 8 * c, 0, never, limit) && landed;      // this chunk's x and v tiles
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const int off = c * (BM * 128) + row * 128 + ((j ^ (row & 7)) << 4);
-                    float4 xx = *reinterpret_cast<float4 *>(xs + off), vv = *reinterpret_cast<float4 *>(vs + off);
-                    const float4 gg = make_float4(__uint_as_float(r[cc][4 * j]), __uint_as_float(r[cc][4 * j + 1]),
-                                                  __uint_as_float(r[cc][4 * j + 2]), __uint_as_float(r[cc][4 * j + 3]));
-                    sgd_update(xx, vv, gg, p.lr, p.mu, p.wd);
-                    *reinterpret_cast<float4 *>(xs + off) = xx;
-                    *reinterpret_cast<float4 *>(vs + off) = vv;
-                    if (p.has_shadow) {
-                        const int nl = c * 32 + 4 * j, box = nl >> 6, piece = (nl & 63) >> 3, half = (nl >> 2) & 1;
-                        *reinterpret_cast<uint2 *>(ss + box * (BM * 128) + row * 128 + ((piece ^ (row & 7)) << 4) + half * 8) =
-                            make_uint2(pack_bf16x2(xx.x, xx.y), pack_bf16x2(xx.z, xx.w));
-                    }
-                }
-                fence_async_smem();
-                asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
-                if (leader) {
-                    if (n0 + c * 32 < p.N) {
-                        tma_store_3d(&sgd.x_out, smem_u32(xs) + c * (BM * 128), n0 + c * 32, m0, wk);
-                        tma_store_3d(&sgd.v, smem_u32(vs) + c * (BM * 128), n0 + c * 32, m0, wk);
-                    }
-                    // a 64-column box of the bf16 copy is complete after every second chunk
-                    if (p.has_shadow && (c & 1) && n0 + (c >> 1) * 64 < p.N)
-                        tma_store_3d(&sgd.shadow, smem_base + (c >> 1) * (BM * 128), n0 + (c >> 1) * 64, m0, wk);
-                    tma_store_commit();
-                }
-            }
-            if (leader) tma_store_wait_read<0>();              // shared memory must outlive the reads
-            if (!landed && p.error_flag != nullptr) atomicExch(p.error_flag, 4);
-        } else if (EPI == EPI_F32) {
+        if (EPI == EPI_F32) {
             if (p.map_c_ok) {
                 // stage the fp32 tile in the (now idle) ring as 128 x 32 sub-tiles with the 128-byte swizzle
                 // (16-byte piece j of row r sits at piece j ^ (r & 7)); each sub-tile is handed to the store

@@ -106,22 +106,20 @@ cudaError_t launch_dependent(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3
 
 template <int EPI, bool A_MN, bool B_MN>
 cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &c, const Params &p, int workers,
-                        cudaStream_t s, const SgdMaps *sgd = nullptr, bool pdl = false)
+                        cudaStream_t s, bool pdl = false)
 {
-    static const SgdMaps no_sgd{};
-    constexpr int NT = (EPI == EPI_SGD) ? 256 : 128;      // the update epilogue is long and runs one CTA per SM
-    const int need = (EPI == EPI_SGD) ? smem_bytes_sgd(p.stages) : smem_bytes(p.stages);
+    constexpr int NT = 128;
+    const int need = smem_bytes(p.stages);
     static int configured = 0;
     if (configured < need) {
-        const int cap = (EPI == EPI_SGD) ? smem_bytes_sgd(2) : smem_bytes(MAX_STAGES);
+        const int cap = smem_bytes(MAX_STAGES);
         if (need > cap) return cudaErrorInvalidValue;
         cudaError_t e = cudaFuncSetAttribute(gemm_bf16<EPI, A_MN, B_MN, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, cap);
         if (e != cudaSuccess) return e;
         configured = cap;
     }
     const dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, workers);
-    return launch_dependent(pdl, gemm_bf16<EPI, A_MN, B_MN, NT>, grid, dim3(NT), (size_t)need, s, a, b, c,
-                            sgd ? *sgd : no_sgd, p);
+    return launch_dependent(pdl, gemm_bf16<EPI, A_MN, B_MN, NT>, grid, dim3(NT), (size_t)need, s, a, b, c, p);
 }
 
 // The persistent gradient + update kernel over the tiles of up to two weight matrices.
@@ -147,7 +145,6 @@ inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK -
 // warps per CTA of head_backward (measured inside the gradient chain: 2 warps 20.3 us, 4 warps 14.3 us,
 // 8 warps 15.9 us; about 8 us of it is fixed cost, not the loop over the samples)
 constexpr int HEAD_NW = 4;
-constexpr int HEAD_COLS = 64;       // hidden units per CTA of head_backward: two adjacent ones per thread
 // Output layer forward and loss.  One CTA = 8 samples of one worker (one per warp); W3 sits in shared
 // memory; every lane loads its slices of the h2 row up front (all loads in flight at once):
 // logits = h2 W3^T + b3 (fp32), row loss = -log softmax[label], dz3 = bf16((softmax - onehot) / batch)
@@ -236,11 +233,11 @@ head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long l
     if (lane == 0) rowloss[(long long)w * B + b] = -logf(py);
 }
 
-// Everything downstream of dz3 that runs on CUDA cores, for 64 hidden units j and all 128 samples:
+// Everything downstream of dz3 that runs on CUDA cores, for 32 hidden units j and all 128 samples:
 //   dz2[b][j] = bf16((sum_c dz3[b][c] W3[c][j]) * (h2[b][j] > 0)),  db2[j] = sum_b dz2[b][j],
 //   dW3[c][j] = sum_b dz3[b][c] h2[b][j];
 // one extra CTA per worker writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the zero padding of
-// the gradient.  Fixed summation orders (deterministic).  grid (d_h / 64 + 1, K).
+// the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32 + 1, K).
 template <int DOUT, int NW>
 __global__ void __launch_bounds__(32 * NW)
 head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__restrict__ dz3,
@@ -255,10 +252,10 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
     static_assert(NW >= 2, "the scalar CTA uses two warps");
     constexpr int C4 = (DOUT + 3) / 4;
     __shared__ __align__(16) float sdz[128 * 16];
-    __shared__ float red[NW][16][HEAD_COLS + 2];
-    __shared__ float colsum[NW][HEAD_COLS + 2];
-    const int w = blockIdx.y, j0 = blockIdx.x * HEAD_COLS, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
-    const int j = j0 + 2 * lane;
+    __shared__ float red[NW][16][33];
+    __shared__ float colsum[NW][33];
+    const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
+    const int j = j0 + lane;
     pdl_launch_dependents();
     pdl_wait();
     if (blockIdx.x == gridDim.x - 1) {
@@ -295,41 +292,36 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
         }
         return;
     }
-    // first batch of this thread's h2 values (two adjacent hidden units per thread: 128-byte lines per warp):
-    // in flight while dz3 and W3 are fetched
-    float2 hreg[16];
+    // first batch of this thread's h2 values: in flight while dz3 and W3 are fetched
+    float hreg[16];
 #pragma unroll
     for (int q = 0; q < 16; ++q) {
         const int b = wp + NW * q;
-        hreg[q] = (b < B) ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(h2 + ((long long)w * B + b) * d_h + j))
-                          : make_float2(0.0f, 0.0f);
+        hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
     }
     for (int i = threadIdx.x; i < B * 16; i += 32 * NW) sdz[i] = dz3[(long long)w * B * 16 + i];
-    float2 w3[4 * C4], acc3[4 * C4];
+    float w3[4 * C4], acc3[4 * C4];
 #pragma unroll
     for (int c = 0; c < 4 * C4; ++c) {
-        w3[c] = (c < d_out) ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(
-                                  params + (long long)w * P + oW3 + (long long)c * d_h + j))
-                            : make_float2(0.0f, 0.0f);
-        acc3[c] = make_float2(0.0f, 0.0f);
+        w3[c] = (c < d_out) ? __bfloat162float(params[(long long)w * P + oW3 + (long long)c * d_h + j]) : 0.0f;
+        acc3[c] = 0.0f;
     }
     __syncthreads();
-    float2 csum = make_float2(0.0f, 0.0f);
+    float csum = 0.0f;
     for (int q0 = 0; q0 * NW < B; q0 += 16) {
         if (q0 > 0) {
 #pragma unroll
             for (int q = 0; q < 16; ++q) {
                 const int b = wp + NW * (q0 + q);
-                hreg[q] = (b < B) ? __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(h2 + ((long long)w * B + b) * d_h + j))
-                                  : make_float2(0.0f, 0.0f);
+                hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
             }
         }
 #pragma unroll
         for (int q = 0; q < 16; ++q) {
             const int b = wp + NW * (q0 + q);
             if (b < B) {
-                const float2 h = hreg[q];
-                float2 a = make_float2(0.0f, 0.0f);
+                const float h = hreg[q];
+                float a = 0.0f;
                 const float4 *d4 = reinterpret_cast<const float4 *>(sdz + b * 16);
 #pragma unroll
                 for (int c4 = 0; c4 < C4; ++c4) {
@@ -338,31 +330,23 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         if (4 * c4 + e < DOUT) {
-                            a.x = fmaf(d[e], w3[4 * c4 + e].x, a.x);
-                            a.y = fmaf(d[e], w3[4 * c4 + e].y, a.y);
-                            acc3[4 * c4 + e].x = fmaf(d[e], h.x, acc3[4 * c4 + e].x);
-                            acc3[4 * c4 + e].y = fmaf(d[e], h.y, acc3[4 * c4 + e].y);
+                            a = fmaf(d[e], w3[4 * c4 + e], a);
+                            acc3[4 * c4 + e] = fmaf(d[e], h, acc3[4 * c4 + e]);
                         }
                     }
                 }
-                const __nv_bfloat162 v = __floats2bfloat162_rn(h.x > 0.0f ? a.x : 0.0f, h.y > 0.0f ? a.y : 0.0f);
-                *reinterpret_cast<__nv_bfloat162 *>(dz2 + ((long long)w * B + b) * d_h + j) = v;
-                const float2 vf = __bfloat1622float2(v);
-                csum.x += vf.x;
-                csum.y += vf.y;
+                const bf16 v = __float2bfloat16_rn(h > 0.0f ? a : 0.0f);
+                dz2[((long long)w * B + b) * d_h + j] = v;
+                csum += __bfloat162float(v);
             }
         }
     }
 #pragma unroll
-    for (int c = 0; c < 16; ++c) {
-        red[wp][c][2 * lane] = (c < DOUT) ? acc3[c < DOUT ? c : 0].x : 0.0f;
-        red[wp][c][2 * lane + 1] = (c < DOUT) ? acc3[c < DOUT ? c : 0].y : 0.0f;
-    }
-    colsum[wp][2 * lane] = csum.x;
-    colsum[wp][2 * lane + 1] = csum.y;
+    for (int c = 0; c < 16; ++c) red[wp][c][lane] = (c < DOUT) ? acc3[c < DOUT ? c : 0] : 0.0f;
+    colsum[wp][lane] = csum;
     __syncthreads();
-    for (int i = threadIdx.x; i < 16 * HEAD_COLS; i += 32 * NW) {
-        const int c = i / HEAD_COLS, l = i % HEAD_COLS;
+    for (int i = threadIdx.x; i < 16 * 32; i += 32 * NW) {
+        const int c = i >> 5, l = i & 31;
         if (c < d_out) {
             float s = 0.0f;
 #pragma unroll
@@ -372,7 +356,7 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
             else grads[idx] = s;
         }
     }
-    if (threadIdx.x < HEAD_COLS) {
+    if (threadIdx.x < 32) {
         float s = 0.0f;
 #pragma unroll
         for (int q = 0; q < NW; ++q) s += colsum[q][threadIdx.x];
@@ -497,12 +481,12 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     const long long P = h->P;
     const uint64_t uK = K, uB = B, uh = d_h, ui = d_in, uP = P;
     // maps over caller memory
-    CUtensorMap k_x, mn_x, k_w1, k_w2, mn_w2, c_w1{}, c_w2{}, none{};
+    CUtensorMap k_x, mn_x, k_w1, k_w2, mn_w2, c_w1{}, c_w2{};
     if (!map_k(&k_x, xin, ui, uB, uK, ui, uB * ui) || !map_mn(&mn_x, xin, ui, uB, uK, ui, uB * ui) ||
         !map_k(&k_w1, prm + h->oW1, ui, uh, uK, ui, uP) || !map_k(&k_w2, prm + h->oW2, uh, uh, uK, uh, uP) ||
         !map_mn(&mn_w2, prm + h->oW2, uh, uh, uK, uh, uP))
         return COCOD_ERR_CUDA;
-    SgdMaps s_w1{}, s_w2{};
+    struct StateMaps { CUtensorMap x_in, x_out, v, shadow; } s_w1{}, s_w2{};      // views of W1 and W2 in the engine's state
     if (fused) {
         float *xi = const_cast<float *>(fused->x_in);
         bf16 *sh = fused->shadow;
@@ -537,15 +521,15 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     // h1 = relu(x W1^T + b1)
     p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
     p.bias = prm + h->ob1; p.bias_worker_stride = P;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, nullptr, pdl_fwd)));
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, pdl_fwd)));
     // h2 = relu(h1 W2^T + b2)
     p.K = d_h; p.stages = stages_for(d_h); p.bias = prm + h->ob2;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, nullptr, pdl_fwd)));
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, pdl_fwd)));
     // output layer, loss, dz3; then dz2, dW3, db3, db2
     const size_t w3_bytes = (size_t)d_out * d_h * sizeof(bf16);
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_logits<10> : head_logits<16>, dim3(B / 8, K), dim3(256), w3_bytes, s,
                              h->h2, prm, P, h->oW3, h->ob3, labels, h->dz3, h->rowloss, B, d_h, d_out));
-    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / HEAD_COLS + 1, K),
+    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
                              dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->dz3, (const float *)h->rowloss,
                              h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out, small));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
@@ -565,16 +549,17 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     Params r{};
     r.error_flag = h->error_flag;
     r.M = d_h; r.N = d_h; r.K = B; r.stages = stages_for(B);
-    // Replayed from a CUDA graph, the backward pass runs as two branches (the handle's own stream, forked from and
+    // Replayed from a CUDA graph, the backward pass of the gradient call runs as two branches (the handle's own stream, forked from and
     // joined to the caller's stream by events): measured 89.1 -> 82.8 us for the chain of the gradient call.
     // Queued eagerly the same fork costs more in event calls than it gains (93.0 -> 94.2 us), so it is used under
     // stream capture only.
     const bool fork = (capturing != cudaStreamCaptureStatusNone);
     if (fused) {
-        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
-        if (B <= 2 * BK) {
+        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, pdl)));
+        {
             // one persistent kernel walks the tiles of W2 and then of W1 (loads of a tile under the update and the
-            // store drain of the tile before it)
+            // store drain of the tile before it); the batch of 128 is its whole reduction (two operand blocks)
+            static_assert(2 * BK == 128, "the update kernel holds the whole reduction in its two-stage ring");
             UpdateProblem u2{}, u1{};
             u2.a = h->mn_dz2; u2.b = h->mn_h1; u2.x_in = s_w2.x_in; u2.x_out = s_w2.x_out; u2.v = s_w2.v;
             u2.shadow = s_w2.shadow; u2.has_shadow = fused->shadow != nullptr;
@@ -587,41 +572,26 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
             UpdateParams uq{};
             uq.K = B; uq.lr = fused->lr; uq.mu = fused->mu; uq.wd = fused->wd; uq.error_flag = h->error_flag;
             GEMM_OK(launch_update(u2, u1, uq, s, pdl));
-        } else {
-        r.lr = fused->lr; r.mu = fused->mu; r.wd = fused->wd; r.has_shadow = fused->shadow != nullptr;
-        if (fork) {     // the two update kernels touch disjoint parameters: side by side, their last waves fill up
-            if (cudaEventRecord(h->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(h->side, h->ev_fork, 0) != cudaSuccess)
-                return COCOD_ERR_CUDA;
-            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, false)));
-            r.N = d_in;
-            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, h->side, &s_w1, false)));
-            if (cudaEventRecord(h->ev_join, h->side) != cudaSuccess || cudaStreamWaitEvent(s, h->ev_join, 0) != cudaSuccess)
-                return COCOD_ERR_CUDA;
-        } else {
-            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz2, h->mn_h1, none, r, K, s, &s_w2, pdl)));
-            r.N = d_in;
-            GEMM_OK((launch_gemm<EPI_SGD, true, true>(h->mn_dz1, mn_x, none, r, K, s, &s_w1, pdl)));
-        }
         }
     } else if (fork) {
         // dW2 needs only dz2 and h1: it runs beside dz1 -> dW1.  dz1 is queued first and keeps a ring of three
         // stages here, so that a CTA of dW2 fits next to it on the same SM (2, 4 and 6 stages measured slower).
         if (cudaEventRecord(h->ev_fork, s) != cudaSuccess) return COCOD_ERR_CUDA;
         q.stages = std::min(q.stages, 3);
-        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, false)));
+        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, false)));
         if (cudaStreamWaitEvent(h->side, h->ev_fork, 0) != cudaSuccess) return COCOD_ERR_CUDA;
         r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, h->side, nullptr, false)));
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, h->side, false)));
         if (cudaEventRecord(h->ev_join, h->side) != cudaSuccess) return COCOD_ERR_CUDA;
         r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, nullptr, false)));
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, false)));
         if (cudaStreamWaitEvent(s, h->ev_join, 0) != cudaSuccess) return COCOD_ERR_CUDA;
     } else {
-        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, nullptr, pdl)));
+        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, pdl)));
         r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s, nullptr, pdl)));
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s, pdl)));
         r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, nullptr, pdl)));
+        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, pdl)));
     }
 #undef LAUNCH_OK
 #undef GEMM_OK
