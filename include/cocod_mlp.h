@@ -96,6 +96,13 @@ int cocod_gemm_bf16(const void *A, const void *B, float *C, int M, int N, int K,
  * and the CUDA context stays usable.  (COCOD_OK would mean the wait did not run out.) */
 int cocod_gemm_wait_selftest(int wait_ms, cocod_stream_t stream);
 
+/* The same self-test for the persistent gradient + update kernel of cocod_mlp_grad_step: one CTA
+ * with three tiles whose copies are never issued.  The thread that issues the tensor-core
+ * instructions gives up after wait_ms, the other roles see that and walk through their remaining
+ * tiles without touching memory (every barrier still sees all of its threads), tensor memory is
+ * released, COCOD_ERR_TIMEOUT is returned and the context stays usable. */
+int cocod_gemm_update_wait_selftest(int wait_ms, cocod_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -38,6 +38,7 @@ struct UpdateParams {
     float lr, mu, wd;
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
+    int debug_no_loads;                // self-test: the producer issues nothing, so the waits run out
 };
 
 constexpr int UPD_THREADS = 320;       // producer warp, MMA warp, 8 update warps
@@ -119,7 +120,7 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
     if (warp == 0 && lane == 0) {
         // ---- producer
         int i = 0, issued_ops = 0, issued_xv = 0;      // tiles whose operand / x-v copies have been issued
-        for (int t = blockIdx.x; t < total && !failed; t += gridDim.x, ++i) {
+        for (int t = blockIdx.x; t < total && !failed && !q.debug_no_loads; t += gridDim.x, ++i) {
             const UpdateProblem *P; int wk, m0, n0;
             decode(t, P, wk, m0, n0);
             for (int kb = 0; kb < nkb; ++kb) {

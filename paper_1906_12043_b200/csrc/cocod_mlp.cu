@@ -711,4 +711,40 @@ int cocod_gemm_wait_selftest(int wait_ms, cocod_stream_t stream)
     return f ? COCOD_ERR_TIMEOUT : COCOD_OK;
 }
 
+int cocod_gemm_update_wait_selftest(int wait_ms, cocod_stream_t stream)
+{
+    if (wait_ms < 1 || wait_ms > 2000) return COCOD_ERR_INVALID;
+    static bf16 *ops = nullptr;
+    static float *state = nullptr;
+    static int *flag = nullptr;
+    if (!ops) {
+        if (cudaMalloc((void **)&ops, 128 * 128 * sizeof(bf16)) != cudaSuccess) return COCOD_ERR_OOM;
+        if (cudaMalloc((void **)&state, 128 * 128 * sizeof(float)) != cudaSuccess) return COCOD_ERR_OOM;
+        if (cudaMalloc((void **)&flag, sizeof(int)) != cudaSuccess) return COCOD_ERR_OOM;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(flag, 0, sizeof(int), s) != cudaSuccess) return COCOD_ERR_CUDA;
+    // three tiles for one CTA: nothing is ever copied, so the maps only have to exist
+    UpdateProblem u{}, none{};
+    if (!map_mn(&u.a, ops, 128, 128, 1, 128, 128 * 128) || !map_mn(&u.b, ops, 128, 128, 1, 128, 128 * 128) ||
+        !map_out(&u.x_in, state, 128, 128, 1, 128, 128 * 128) || !map_out(&u.x_out, state, 128, 128, 1, 128, 128 * 128) ||
+        !map_out(&u.v, state, 128, 128, 1, 128, 128 * 128))
+        return COCOD_ERR_CUDA;
+    u.has_shadow = 0; u.M = 128; u.N = 128; u.tiles_m = 1; u.tiles_n = 1; u.tiles = 3;
+    UpdateParams q{};
+    q.K = 128; q.lr = 0.1f; q.mu = 0.9f; q.wd = 0.0f; q.error_flag = flag;
+    q.wait_ns = (unsigned long long)wait_ms * 1000000ull;
+    q.debug_no_loads = 1;
+    if (cudaFuncSetAttribute(gemm_update_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    if (launch_dependent(false, gemm_update_persistent, dim3(1), dim3(UPD_THREADS), (size_t)UPD_SMEM, s, u, none, q) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    int f = 0;
+    if (cudaMemcpyAsync(&f, flag, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    return f ? COCOD_ERR_TIMEOUT : COCOD_OK;
+}
+
+
 }  // extern "C"

@@ -21,6 +21,7 @@ SIGNATURES = {
     "cocod_mlp_check": (_i, [_vp, _vp]),
     "cocod_mlp_launch_count": (_i64, [_vp]),
     "cocod_gemm_wait_selftest": (_i, [_i, _vp]),
+    "cocod_gemm_update_wait_selftest": (_i, [_i, _vp]),
     "cocod_gemm_bf16": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i64, _i64, _i64, _vp]),
 }
 
@@ -121,6 +122,11 @@ def gemm_bf16(A, B, C, a_rows_contiguous=False, b_rows_contiguous=False, stream=
                                 B.stride(0), C.stride(0), _cur_stream(stream))
     if rc != _E.OK:
         raise _E.CocodError(rc, "cocod_gemm_bf16")
+
+
+def gemm_update_wait_selftest(wait_ms: int = 50, stream=None) -> int:
+    """The bounded-wait self-test of the persistent gradient + update kernel (ERR_TIMEOUT is the expected code)."""
+    return int(load().cocod_gemm_update_wait_selftest(int(wait_ms), _cur_stream(stream)))
 
 
 def gemm_wait_selftest(wait_ms: int = 50, stream=None) -> int:

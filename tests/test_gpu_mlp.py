@@ -297,6 +297,13 @@ def test_a_wait_that_nothing_satisfies_times_out_and_leaves_the_gpu_usable(M, E)
     M.gemm_bf16(bf16_tensor(A), bf16_tensor(A), C)
     np.testing.assert_allclose(cpu(C)[0], A[0].astype(np.float64) @ A[0].astype(np.float64).T, rtol=0, atol=1e-4)
     assert M.gemm_wait_selftest(20) == E.ERR_TIMEOUT     # and again
+    # the persistent gradient + update kernel: its tensor-core thread gives up, the other roles walk through
+    # their remaining tiles without touching memory, and the fused path still works afterwards
+    assert M.gemm_update_wait_selftest(50) == E.ERR_TIMEOUT
+    assert M.gemm_update_wait_selftest(20) == E.ERR_TIMEOUT
+    C.zero_()
+    M.gemm_bf16(bf16_tensor(A), bf16_tensor(A), C)
+    np.testing.assert_allclose(cpu(C)[0], A[0].astype(np.float64) @ A[0].astype(np.float64).T, rtol=0, atol=1e-4)
 
 
 @pytest.mark.parametrize("K,dims,wd", [(3, (200, 256, 256, 7), 5e-4), (16, I.MLP_DIMS, 0.0)])
