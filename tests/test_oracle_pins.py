@@ -462,3 +462,109 @@ def test_local_sgd_average_is_the_zero_drift_merge(mode):
     a.local_sgd_average()
     c.ssgd_step(g)
     np.testing.assert_allclose(a.x, c.x, rtol=0, atol=1e-15 if mode == "f64" else 5e-8)
+
+
+# ----------------------------------------------------------------------------- Step I's mean over many workers
+# The fp32 "mirror" sums the workers in blocks of 8 rows (pairwise tree inside a block, block sums accumulated in
+# order, a ragged last block); the cases below hold that path -- and the plain loops of the other two modes -- to
+# exact rational arithmetic and to an error bound, at worker counts with 2 to 125 blocks and every kind of tail.
+MANY_K = [9, 15, 16, 17, 64, 1000]
+
+
+def exact_weighted_mean(X, M=None):
+    """Step I's x_hat = sum_i (M_i / sum_j M_j) x^i in exact rational arithmetic (scalar loops)."""
+    K, P = X.shape
+    tot = Fraction(K) if M is None else sum(Fraction(float(m)) for m in M)
+    w = [Fraction(1) / tot if M is None else Fraction(float(M[i])) / tot for i in range(K)]
+    return [sum(w[i] * Fraction(float(X[i, p])) for i in range(K)) for p in range(P)]
+
+
+def mean_of(mode, X, M=None):
+    K, P = X.shape
+    eng = OracleEngine(K, P, 0.1, 0.0, 0.0, mode=mode, batch_sizes=M)
+    eng.set_params_all(X)
+    eng.comm_begin()
+    return eng
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("K", MANY_K)
+def test_many_worker_mean_is_exact_on_dyadic_inputs(K, mode):
+    """Small dyadic rows: every partial sum is exact in fp32 in any order, so the only roundings left are 1/K and
+    the final product (none at all when K is a power of two)."""
+    rng = np.random.default_rng(K)
+    P = 11
+    X = (rng.integers(-64, 65, (K, P)) / 16).astype(np.float32)
+    eng = mean_of(mode, X)
+    want = np.array([float(c) for c in exact_weighted_mean(X)])
+    if K & (K - 1) == 0:
+        np.testing.assert_array_equal(eng.mean.astype(np.float64), want)
+    else:
+        bound = 2.0 ** -23 * np.abs(want) if mode != "f64" else 2.0 ** -52 * np.abs(want)
+        assert np.all(np.abs(eng.mean.astype(np.float64) - want) <= bound)
+    # line 6 with zero drift then hands exactly that mean to every worker
+    eng.comm_end()
+    for i in range(K):
+        np.testing.assert_array_equal(eng.x[i], eng.mean)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("K", MANY_K)
+def test_many_worker_mean_counts_every_worker_exactly_once(K, mode):
+    """Worker i is the only one with a non-zero entry in column i: a dropped, doubled or misplaced row (or whole
+    block of rows) changes that column from 2^j / K to 0 or to a multiple of it."""
+    X = np.zeros((K, K), np.float32)
+    vals = 2.0 ** (np.arange(K) % 7 - 3)
+    X[np.arange(K), np.arange(K)] = vals
+    eng = mean_of(mode, X)
+    want = vals / K
+    np.testing.assert_allclose(eng.mean.astype(np.float64), want, rtol=2.0 ** -22, atol=0)
+    # unequal batch sizes that are powers of two with a power-of-two total keep the weights dyadic: exact
+    if K == 16:
+        M = np.array([8] + [1] * 8 + [2] * 4 + [4] * 2 + [32], float)          # sums to 64
+        eng = mean_of(mode, X, M)
+        np.testing.assert_array_equal(eng.mean.astype(np.float64), vals * M / 64.0)
+
+
+@pytest.mark.parametrize("weighted", [False, True])
+@pytest.mark.parametrize("K", MANY_K)
+def test_many_worker_mean_within_its_rounding_bound_on_gaussian_inputs(K, weighted):
+    """fp32 mirror against exact arithmetic on workload-shaped values: the tree-of-8 order performs at most
+    3 + K/8 dependent additions per column, plus one rounding of each weight and of each product (weighted) or of
+    1/K and the final product (equal sizes).  The fp64-evaluated modes must sit within one fp32 rounding."""
+    rng = np.random.default_rng(100 + K)
+    P = 64
+    X = (rng.standard_normal((K, P)) * 0.01).astype(np.float32)
+    M = rng.integers(1, 9, K).astype(float) if weighted else None
+    exact = exact_weighted_mean(X, M)
+    want = np.array([float(c) for c in exact])
+    w = np.full(K, 1.0 / K) if M is None else M / M.sum()
+    mass = np.abs(w[:, None] * X.astype(np.float64)).sum(axis=0)              # sum_i |w_i x_i| per column
+    mir = mean_of("mirror", X, M).mean.astype(np.float64)
+    assert np.all(np.abs(mir - want) <= (5 + K / 8) * 2.0 ** -24 * mass)
+    ref = mean_of("ref", X, M).mean.astype(np.float64)
+    assert np.all(np.abs(ref - want) <= 2.0 ** -24 * np.abs(want) + 1e-16 * mass)
+    f64 = mean_of("f64", X.astype(np.float64), M).mean
+    assert np.all(np.abs(f64 - want) <= 1e-15 * mass)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("K", [9, 17, 64])
+def test_sequential_schemes_with_many_workers(K, mode):
+    """Local-SGD's averaging and S-SGD's gradient averaging use the same mean: at worker counts that span
+    several blocks they must give every worker the exact weighted mean (dyadic inputs, to the rounding of 1/K)."""
+    rng = np.random.default_rng(K + 7)
+    P = 13
+    X = (rng.integers(-32, 33, (K, P)) / 8).astype(np.float32)
+    want = np.array([float(c) for c in exact_weighted_mean(X)])
+    tol_k = 0.0 if K & (K - 1) == 0 else 2.0 ** -23
+    a = OracleEngine(K, P, 0.5, 0.0, 0.0, mode=mode)
+    a.set_params_all(X)
+    a.local_sgd_average()
+    for i in range(K):
+        assert np.all(np.abs(a.x[i].astype(np.float64) - want) <= tol_k * np.abs(want))
+    # S-SGD from x = 0 with lr = 1/2, mu = wd = 0: x = -mean(g) / 2 on every worker
+    b = OracleEngine(K, P, 0.5, 0.0, 0.0, mode=mode)
+    b.ssgd_step(X)
+    for i in range(K):
+        assert np.all(np.abs(b.x[i].astype(np.float64) + want / 2) <= tol_k * np.abs(want) / 2)
