@@ -49,7 +49,7 @@ enum {
 
 /* Options for cocod_set_option. */
 enum {
-    /* How Step I "stores x_t^i".  COPY: a copy kernel writes the stored copies (8 B per
+    /* How Step I keeps its copy of x_t^i.  COPY: a copy kernel writes the stored copies (8 B per
      * worker-parameter per round).  FLIP (default): the buffer holding x becomes the stored
      * copy and the first local step of the round writes x into the spare buffer (0 B); the
      * values are identical. */
@@ -93,7 +93,7 @@ int cocod_local_step(cocod_handle *h, const float *grads);
 int cocod_local_step_host(cocod_handle *h, const float *host_grads);
 
 /* Algorithm 1, Step I: store x_t^i and start computing the weighted mean of the stored copies
- * x_hat_t = sum_i (M_i / sum_j M_j) x_t^i, "in parallel" with Step II: the mean kernel runs on
+ * x_hat_t = sum_i (M_i / sum_j M_j) x_t^i, concurrently with Step II: the mean kernel runs on
  * `side`, ordered after the compute stream's work so far.  side == compute stream is allowed
  * (then it simply runs in order).  Errors: STATE if a communication is already in flight. */
 int cocod_comm_begin(cocod_handle *h, cocod_stream_t side);
@@ -126,7 +126,7 @@ int cocod_ssgd_step(cocod_handle *h, const float *grads);
  * in flight (STATE). */
 int cocod_set_stream(cocod_handle *h, cocod_stream_t compute);
 
-/* "Initialize: x_i^0 = x_hat_0": broadcast P values to all K workers.  on_host selects what
+/* Algorithm 1, Initialize (x_i^0 = x_hat_0 for every worker): broadcast P values to all K workers.  on_host selects what
  * kind of pointer x0 is.  Stream-ordered on the compute stream (host sources are copied
  * synchronously first).  Not while a communication is in flight (STATE). */
 int cocod_set_params(cocod_handle *h, const float *x0, int on_host);
@@ -148,7 +148,7 @@ int cocod_get_bf16_shadow(cocod_handle *h, void **out);
 /* The paper changes gamma during a run (warm-up, decay at epoch 81; Section 5.1). */
 int cocod_set_lr(cocod_handle *h, float lr);
 
-/* Mini-batch sizes M_1..M_K of Algorithm 1 ("proportionally sampling", Section 3.2): the mean
+/* Mini-batch sizes M_1..M_K of Algorithm 1 (sampling in proportion to the workers' data, Section 3.2): the mean
  * uses weights M_i / sum_j M_j.  M: host, K positive finite values; NULL = all equal. */
 int cocod_set_batch_sizes(cocod_handle *h, const double *M);
 

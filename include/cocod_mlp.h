@@ -2,8 +2,9 @@
  * cocod_mlp.h -- per-worker mini-batch stochastic gradients for the end-to-end configuration
  * (part of libcocod.so).
  *
- * Algorithm 1 of arxiv 1906.12043, Step II: "compute a mini-batch stochastic gradient
- * G_tau^i = (1/M_i) sum_j grad f_i(x_tau^i, xi_tau^{i,j})".  Here f is the softmax cross-entropy
+ * Algorithm 1 of arxiv 1906.12043, Step II: every worker i forms the stochastic gradient G_tau^i of
+ * its current model as the mean of the per-sample gradients over its mini-batch of M_i samples.
+ * Here f is the softmax cross-entropy
  * of a 3-layer ReLU MLP (d_in -> d_hidden -> d_hidden -> d_out) and all K workers' gradients are
  * computed in one batched pass: the contractions run on the sm_100a tensor cores (tcgen05.mma,
  * bf16 operands, fp32 accumulation in TMEM, TMA-staged operands), everything else in small fused
@@ -62,8 +63,10 @@ int cocod_mlp_grad(cocod_mlp_handle *h, const void *params_bf16, const void *x, 
  * update of one iteration in one call).  `engine` must have been created with
  * K = the handle's K and P = cocod_mlp_param_count, with COCOD_OPT_BF16_SHADOW on (STATE otherwise):
  * the gradients are computed from its bf16 copy of x.  For the two weight matrices W1 and W2
- * (99.4 % of the parameters) the weight-gradient GEMMs apply the update d = g + wd x; v = mu v + d;
- * x = x - lr v in their epilogue: the gradient tile never leaves the SM, x, v and the bf16 copy are
+ * (99.4 % of the parameters) one persistent, warp-specialised kernel walks over the 128 x 128 tiles of
+ * W2 and then of W1: it forms a tile's weight gradient on the tensor cores (two accumulators in tensor
+ * memory, so the next tile's product forms meanwhile) and applies d = g + wd x; v = mu v + d;
+ * x = x - lr v to that tile at once: the gradient tile never leaves the SM, x, v and the bf16 copy are
  * read and written once.  The remaining tensors (biases, W3) take the same update inside the kernels
  * that produce their gradients, so no gradient is ever written to memory.  Results are bit-identical
  * to cocod_mlp_grad followed by cocod_local_step.  Runs on the engine's compute stream; counts as

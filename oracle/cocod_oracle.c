@@ -94,7 +94,7 @@ void oracle_local_step_mirror(int K, int64_t P, float *x, float *v, const float 
 }
 
 /* ------------------------------------------------------------------ Step I: store x_t^i
- * Algorithm 1, Step I: "store x_t^i in the memory". */
+ * Algorithm 1, Step I: every worker keeps a copy of its model x_t^i as it is at iteration t. */
 void oracle_snapshot_f32(int K, int64_t P, const float *x, float *snap)
 {
     memcpy(snap, x, (size_t)K * (size_t)P * sizeof(float));

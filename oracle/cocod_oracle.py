@@ -80,7 +80,7 @@ class OracleEngine:
 
     The call sequence is the algorithm's: ``comm_begin`` is Step I (store x_t^i, form the
     weighted mean of the stored copies), ``local_step`` is one iteration of Step II,
-    ``comm_end`` is line 6.  Running Step I "in parallel" with Step II changes no value (the
+    ``comm_end`` is line 6.  Running Step I concurrently with Step II changes no value (the
     mean reads only the stored copies), so this oracle simply does Step I at once.
 
     ``batch_sizes`` are the M_i of Algorithm 1 (None = all equal).  Hyper-parameters are taken

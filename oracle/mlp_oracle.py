@@ -2,8 +2,9 @@
 TEST INFRASTRUCTURE ONLY (same rules as cocod_oracle.py: only tests, the smoke check and the
 benchmark's CPU legs may import it; it imports nothing of the CUDA path).
 
-Algorithm 1, Step II: "compute a mini-batch stochastic gradient G = (1/M) sum_j grad f(x, xi_j)"
-for f = softmax cross-entropy of a 3-layer ReLU MLP.  This is a textbook definition, so the
+Algorithm 1, Step II: each worker's stochastic gradient is the mean, over the M samples of its
+mini-batch, of the per-sample gradients of f at its current model; here f = softmax cross-entropy
+of a 3-layer ReLU MLP.  This is a textbook definition, so the
 oracle is that definition written out in numpy fp64.  The workload stores weights in bfloat16
 (fp32 master copy) and runs the contractions on tensor cores, so with ``emulate_bf16=True`` the
 oracle rounds at exactly the points where the device path stores bfloat16:

@@ -11,11 +11,11 @@
 //   * one elected thread issues tcgen05.mma (kind::f16, bf16 inputs, fp32 accumulation) on
 //     shared-memory descriptors; the 128 x 128 fp32 accumulator lives in TMEM (128 columns);
 //   * all four warps read the accumulator back with tcgen05.ld (32 lanes x 32 columns at a time)
-//     and run a fused epilogue: bias + ReLU or ReLU-mask with packed bf16 stores, an fp32 store
-//     that goes through swizzled shared memory and TMA bulk stores (full 128-byte lines), or -- for
-//     weight gradients -- the momentum-SGD update itself: the matching x and v tiles are fetched by
-//     TMA while the MMAs run, updated in shared memory with the accumulator as the gradient, and
-//     stored back together with the bf16 copy of x, so the gradient never touches HBM.
+//     and run a fused epilogue: bias + ReLU or ReLU-mask (optionally with the column sums of the
+//     tile, written out or applied to a bias vector as its local step) leaving as bf16 through
+//     staged TMA bulk stores, or an fp32 store that goes through swizzled shared memory and TMA
+//     bulk stores (full 128-byte lines).  (The weight-gradient GEMM that applies the momentum
+//     update to its own tile is a kernel of its own: cocod_gemm_update_sm100.cuh.)
 // Out-of-range rows / reduction columns are zero-filled by TMA, so M, N, K need not be
 // multiples of the tile; stores are predicated.
 //

@@ -460,7 +460,7 @@ local_step_shared_grad_scalar(const float *x_in, float *x_out, float *v, const f
     if (shadow != nullptr) shadow[e] = __float2bfloat16_rn(xn);
 }
 
-// Broadcast P values to K rows ("Initialize: x_i^0 = x_hat_0").
+// Broadcast P values to K rows (Algorithm 1, Initialize: x_i^0 = x_hat_0 for every worker).
 static __global__ void __launch_bounds__(kThreads)
 broadcast_rows(const float *__restrict__ x0, float *__restrict__ x, int K, int64_t P)
 {

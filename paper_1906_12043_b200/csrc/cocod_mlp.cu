@@ -1,5 +1,5 @@
-// Per-worker mini-batch gradients of the 3-layer ReLU MLP (Algorithm 1, Step II: "compute a
-// mini-batch stochastic gradient"), batched over the K workers.  Declared in include/cocod_mlp.h.
+// Per-worker mini-batch gradients of the 3-layer ReLU MLP (the stochastic gradient of Algorithm 1,
+// Step II), batched over the K workers.  Declared in include/cocod_mlp.h.
 //
 // Data flow of one call (every matrix exists once per worker; no matrix is ever transposed in
 // memory: the tensor cores read an operand either with the reduction index contiguous or with the
@@ -88,6 +88,16 @@ bool map_out(CUtensorMap *m, float *base, uint64_t cols, uint64_t rows, uint64_t
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Facts that belong to a device (function attributes set, SM count, scratch of the stand-alone GEMM call) are
+// cached per device, indexed by the current device: one process may drive engines on several GPUs.
+constexpr int MAX_DEVICES = 64;
+inline int current_device()
+{
+    int d = 0;
+    if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= MAX_DEVICES) return -1;
+    return d;
+}
+
 // Launch with the programmatic-serialization attribute: the kernel may become resident (and run the
 // part of its prologue that precedes pdl_wait()) while the previous kernel in the stream drains.
 template <typename... KArgs, typename... Args>
@@ -110,13 +120,15 @@ cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtens
 {
     constexpr int NT = 128;
     const int need = smem_bytes(p.stages);
-    static int configured = 0;
-    if (configured < need) {
+    static int configured[MAX_DEVICES] = {};      // per instantiation and per device
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (configured[dev] < need) {
         const int cap = smem_bytes(MAX_STAGES);
         if (need > cap) return cudaErrorInvalidValue;
         cudaError_t e = cudaFuncSetAttribute(gemm_bf16<EPI, A_MN, B_MN, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, cap);
         if (e != cudaSuccess) return e;
-        configured = cap;
+        configured[dev] = cap;
     }
     const dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, workers);
     return launch_dependent(pdl, gemm_bf16<EPI, A_MN, B_MN, NT>, grid, dim3(NT), (size_t)need, s, a, b, c, p);
@@ -125,17 +137,19 @@ cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtens
 // The persistent gradient + update kernel over the tiles of up to two weight matrices.
 cudaError_t launch_update(const UpdateProblem &p0, const UpdateProblem &p1, const UpdateParams &q, cudaStream_t s, bool pdl)
 {
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    static int sm_count[MAX_DEVICES] = {};        // 0 = this device has not been set up yet
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (sm_count[dev] == 0) {
+        int sms = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_update_persistent, cudaFuncAttributeMaxDynamicSharedMemorySize, UPD_SMEM);
-        if (e != cudaSuccess) { sms = 0; return e; }
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = sms;
     }
     const int total = p0.tiles + p1.tiles;
     if (total <= 0) return cudaSuccess;
-    return launch_dependent(pdl, gemm_update_persistent, dim3(std::min(total, sms)), dim3(UPD_THREADS), (size_t)UPD_SMEM, s,
+    return launch_dependent(pdl, gemm_update_persistent, dim3(std::min(total, sm_count[dev])), dim3(UPD_THREADS), (size_t)UPD_SMEM, s,
                             p0, p1, q);
 }
 
@@ -472,8 +486,9 @@ int64_t cocod_mlp_launch_count(const cocod_mlp_handle *h) { return h ? h->launch
 namespace {
 
 // The whole gradient pass.  With fused == nullptr the weight gradients dW1, dW2 are written to `grads`;
-// otherwise their GEMMs apply the engine's local step in their epilogue (x, v and the bf16 copy of x
-// are updated in place, nothing is written to `grads` for W1 and W2).
+// otherwise one persistent kernel (gemm_update_persistent: the tiles of W2, then of W1, two accumulators in
+// tensor memory) forms them and applies the engine's local step tile by tile (x, v and the bf16 copy of x are
+// updated in place, nothing is written to `grads`).
 int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labels, float *grads, float *loss,
              cudaStream_t s, const cocod_step_plan *fused)
 {
@@ -598,6 +613,25 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     return COCOD_OK;
 }
 
+// Device scratch of one self-test call: allocated on the current device, released (after the device has gone
+// idle: the destructor runs only after the call has synchronised its stream or failed) when the call returns.
+struct SelftestScratch {
+    void *ptrs[4] = {nullptr, nullptr, nullptr, nullptr};
+    int n = 0;
+    void *alloc(size_t bytes)
+    {
+        void *p = nullptr;
+        if (n >= 4 || cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        ptrs[n++] = p;
+        return p;
+    }
+    ~SelftestScratch()
+    {
+        if (n > 0) cudaDeviceSynchronize();
+        for (int i = 0; i < n; ++i) cudaFree(ptrs[i]);
+    }
+};
+
 }  // namespace
 
 extern "C" {
@@ -654,11 +688,15 @@ int cocod_gemm_bf16(const void *A, const void *B, float *C, int M, int N, int Kd
     if (!make_map(&ma, A, a_cols, a_rows, batch_count, lda, sa, a_rows_contiguous ? 64 : 128) ||
         !make_map(&mb, B, b_cols, b_rows, batch_count, ldb, sb, b_rows_contiguous ? 64 : 128))
         return COCOD_ERR_CUDA;
-    static int *flag = nullptr;
-    if (!flag) {
-        if (cudaMalloc((void **)&flag, sizeof(int)) != cudaSuccess) return COCOD_ERR_OOM;
-        cudaMemset(flag, 0, sizeof(int));
+    // the kernel's timeout flag: 4 bytes per device that ever makes this call, kept until the process exits
+    static int *flags[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return COCOD_ERR_CUDA;
+    if (!flags[dev]) {
+        if (cudaMalloc((void **)&flags[dev], sizeof(int)) != cudaSuccess) { cudaGetLastError(); return COCOD_ERR_OOM; }
+        cudaMemset(flags[dev], 0, sizeof(int));
     }
+    int *flag = flags[dev];
     Params p{};
     p.M = M; p.N = N; p.K = Kd; p.stages = stages_for(Kd);
     p.c = C; p.c_worker_stride = (long long)sc; p.ldc = (int)ldc;
@@ -686,15 +724,15 @@ int cocod_gemm_bf16(const void *A, const void *B, float *C, int M, int N, int Kd
 int cocod_gemm_wait_selftest(int wait_ms, cocod_stream_t stream)
 {
     if (wait_ms < 1 || wait_ms > 2000) return COCOD_ERR_INVALID;
-    static bf16 *buf = nullptr;
-    static int *flag = nullptr;
-    if (!buf) {
-        if (cudaMalloc((void **)&buf, 128 * 64 * sizeof(bf16)) != cudaSuccess) return COCOD_ERR_OOM;
-        if (cudaMalloc((void **)&flag, sizeof(int)) != cudaSuccess) return COCOD_ERR_OOM;
-        cudaMemset(buf, 0, 128 * 64 * sizeof(bf16));
-    }
+    // scratch of this call only (on the current device), freed before returning
+    SelftestScratch sc;
+    bf16 *buf = static_cast<bf16 *>(sc.alloc(128 * 64 * sizeof(bf16)));
+    int *flag = static_cast<int *>(sc.alloc(sizeof(int)));
+    if (!buf || !flag) return COCOD_ERR_OOM;
     cudaStream_t s = (cudaStream_t)stream;
-    if (cudaMemsetAsync(flag, 0, sizeof(int), s) != cudaSuccess) return COCOD_ERR_CUDA;
+    if (cudaMemsetAsync(buf, 0, 128 * 64 * sizeof(bf16), s) != cudaSuccess ||
+        cudaMemsetAsync(flag, 0, sizeof(int), s) != cudaSuccess)
+        return COCOD_ERR_CUDA;
     CUtensorMap m, none{};
     if (!map_k(&m, buf, 64, 128, 1, 64, 128 * 64)) return COCOD_ERR_CUDA;
     Params p{};
@@ -714,14 +752,11 @@ int cocod_gemm_wait_selftest(int wait_ms, cocod_stream_t stream)
 int cocod_gemm_update_wait_selftest(int wait_ms, cocod_stream_t stream)
 {
     if (wait_ms < 1 || wait_ms > 2000) return COCOD_ERR_INVALID;
-    static bf16 *ops = nullptr;
-    static float *state = nullptr;
-    static int *flag = nullptr;
-    if (!ops) {
-        if (cudaMalloc((void **)&ops, 128 * 128 * sizeof(bf16)) != cudaSuccess) return COCOD_ERR_OOM;
-        if (cudaMalloc((void **)&state, 128 * 128 * sizeof(float)) != cudaSuccess) return COCOD_ERR_OOM;
-        if (cudaMalloc((void **)&flag, sizeof(int)) != cudaSuccess) return COCOD_ERR_OOM;
-    }
+    SelftestScratch sc;                       // scratch of this call only, freed before returning
+    bf16 *ops = static_cast<bf16 *>(sc.alloc(128 * 128 * sizeof(bf16)));
+    float *state = static_cast<float *>(sc.alloc(128 * 128 * sizeof(float)));
+    int *flag = static_cast<int *>(sc.alloc(sizeof(int)));
+    if (!ops || !state || !flag) return COCOD_ERR_OOM;
     cudaStream_t s = (cudaStream_t)stream;
     if (cudaMemsetAsync(flag, 0, sizeof(int), s) != cudaSuccess) return COCOD_ERR_CUDA;
     // three tiles for one CTA: nothing is ever copied, so the maps only have to exist

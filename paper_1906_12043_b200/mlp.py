@@ -77,8 +77,8 @@ class MLPGrad:
             raise _E.CocodError(rc, "cocod_mlp_grad")
 
     def grad_step(self, engine, x, labels, loss):
-        """Gradients and the engine's local step in one call (the update of W1 and W2 happens in the
-        epilogue of the weight-gradient GEMMs).  ``engine``: an Engine with K x P matching and the
+        """Gradients and the engine's local step in one call (a persistent kernel forms the weight
+        gradients of W1 and W2 tile by tile and updates each tile at once).  ``engine``: an Engine with K x P matching and the
         bf16 shadow switched on.  Bit-identical to grad(...) followed by engine.local_step(grads)."""
         import torch
         K, B, d_in = self.K, self.batch, self.dims[0]

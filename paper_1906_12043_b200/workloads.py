@@ -54,6 +54,6 @@ def bytes_merge(K: int) -> float:
 
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per worker-parameter measured by one
-# `ncu --set full` capture on a small case (K=16, P=4,194,304); pure streaming, so it scales with
-# K*P.  Source: the ncu summary of these three kernels committed under profiles/.
+# `ncu --set full` capture of these three kernels on a small case (K=16, P=4,194,304); pure
+# streaming, so it scales with K*P.
 NCU_DRAM_BYTES_PER_WORKER_PARAM = {"local_step": 19.25, "mean": 4.12, "merge": 11.81}
