@@ -46,20 +46,43 @@ def split(flat: np.ndarray, dims):
 
 
 def loss_and_grad(flat: np.ndarray, X: np.ndarray, labels: np.ndarray, dims, emulate_bf16: bool = True,
-                  return_preactivations: bool = False):
+                  return_preactivations: bool = False, flips=None, return_intermediates: bool = False):
     """Mean softmax cross-entropy of the minibatch and its gradient w.r.t. the flat parameters
     (same flat order).  Returns (loss fp64, grad fp32 array), plus the hidden pre-activations
     (z1, z2) on request: ReLU is a decision "z > 0", and a comparison against another precision is
-    only meaningful for units whose |z| is not within rounding distance of 0."""
+    only meaningful for units whose |z| is not within rounding distance of 0.
+
+    ``flips``: optional list of (layer, sample, unit) with layer 1 or 2: the ReLU decision of that unit
+    for that sample is taken the OTHER way (on -> off: the activation and its gate are 0; off -> on: the
+    gate is 1, the activation stays 0).  For a pre-activation within accumulation error of zero both
+    outcomes are correct results of "z > 0" taken in finite precision; this lets a test evaluate the
+    definition under the outcome another precision took.  The caller vouches that |z| is that small.
+
+    ``return_intermediates``: the third return value is a dict of every intermediate of the definition
+    (z1, z2, h1, h2, on1, on2, dz3, pre2 = dz3 W3, dz2, pre1 = dz2 W2, dz1) instead of (z1, z2)."""
     q = bf16 if emulate_bf16 else (lambda a: np.asarray(a, np.float64))
     p = {k: q(v) for k, v in split(flat, dims).items()}
     X = np.asarray(X, np.float64)
     M = X.shape[0]
+    flip = {1: [], 2: []}
+    for layer, b, j in (flips or []):
+        flip[int(layer)].append((int(b), int(j)))
+
+    def relu(z, which):
+        """h = bf16(max(z, 0)) and the gate (h > 0), with the listed decisions taken the other way."""
+        h = q(np.maximum(z, 0.0))
+        on = h > 0
+        for b, j in flip[which]:
+            on[b, j] = not on[b, j]
+            if not on[b, j]:
+                h[b, j] = 0.0
+        return h, on
+
     # forward
     z1 = X @ p["W1"].T + p["b1"]
-    h1 = q(np.maximum(z1, 0.0))
+    h1, on1 = relu(z1, 1)
     z2 = h1 @ p["W2"].T + p["b2"]
-    h2 = q(np.maximum(z2, 0.0))
+    h2, on2 = relu(z2, 2)
     z3 = h2 @ p["W3"].T + p["b3"]
     zmax = z3.max(axis=1, keepdims=True)
     e = np.exp(z3 - zmax)
@@ -70,11 +93,16 @@ def loss_and_grad(flat: np.ndarray, X: np.ndarray, labels: np.ndarray, dims, emu
     onehot[np.arange(M), labels] = 1.0
     dz3 = q((e / s - onehot) / M)
     g = {"W3": dz3.T @ h2, "b3": dz3.sum(0)}
-    dz2 = q((dz3 @ p["W3"]) * (h2 > 0))
+    pre2 = dz3 @ p["W3"]
+    dz2 = q(pre2 * on2)
     g["W2"], g["b2"] = dz2.T @ h1, dz2.sum(0)
-    dz1 = q((dz2 @ p["W2"]) * (h1 > 0))
+    pre1 = dz2 @ p["W2"]
+    dz1 = q(pre1 * on1)
     g["W1"], g["b1"] = dz1.T @ X, dz1.sum(0)
     flat_g = np.concatenate([g[k].ravel() for k in ("W1", "b1", "W2", "b2", "W3", "b3")])
+    if return_intermediates:
+        return loss, flat_g.astype(np.float32), dict(z1=z1, z2=z2, h1=h1, h2=h2, on1=on1, on2=on2, dz3=dz3, pre2=pre2,
+                                                     dz2=dz2, pre1=pre1, dz1=dz1)
     if return_preactivations:
         return loss, flat_g.astype(np.float32), (z1, z2)
     return loss, flat_g.astype(np.float32)

@@ -15,6 +15,15 @@ after the merge, |gpu - ref| / max(|ref|, rms(ref)), for all four engines.  A bf
 chaotic with respect to rounding, so the free-running error grows; the restarted one is the per-round
 parity figure (bar: 1e-2).
 
+ReLU is a decision (z > 0) that floating point takes.  The device accumulates z in fp32, the oracle in fp64;
+for the few units per round whose |z| lies within accumulation error of zero the two can decide differently,
+both correctly, and one such decision switches a whole sample's term of a weight-gradient row.  The restarted
+engines are therefore compared with a BRANCH of the oracle that starts every round from the canonical oracle
+state and, for units with |z| < 5e-4 only, takes the decision the device took (match_decisions finds them from
+the device's bias gradients, which are the column sums of dz and show a switched term directly).  The
+canonical oracle -- the one the free-running engines and the loss curve are compared with -- never sees
+anything of the device.  The table reports how many decisions were matched and their largest |z|.
+
     python tests/c4_loss_curve.py --rounds 200 --out profiles/c4_loss_curve_K16.md
 
 This is test infrastructure (it drives the oracle); the library and bench.py do not import it.
@@ -38,48 +47,139 @@ from oracle.cocod_oracle import OracleEngine             # noqa: E402
 from paper_1906_12043_b200 import inputs as I            # noqa: E402
 
 _SHM = {}
+BAND_MAX = 5e-4        # a ReLU decision may be matched to the device's only if |z| is below this
+
+
+def _decode_layer(layer, db_dev, db_ref, z, on, dz, pre):
+    """Units of one hidden layer whose decision the device took the other way, read off the bias gradient
+    (db[j] = sum_b dz[b][j]): switching unit (b, j) off removes dz[b][j] from db[j], switching it on adds
+    bf16(pre[b][j]).  Only units with |z| < BAND_MAX are candidates, at most two per column, and a set of switches
+    is accepted only if it explains the column's difference to within a tenth (a genuine switch leaves a residual
+    of a few thousandths; ordinary rounding noise in db is about 3e-4 of its rms and is not touched)."""
+    diff = db_dev.astype(np.float64) - db_ref.astype(np.float64)
+    scale = np.maximum(np.abs(db_ref.astype(np.float64)), np.sqrt(np.mean(db_ref.astype(np.float64) ** 2)))
+    flips = []
+    for j in np.nonzero(np.abs(diff) > 5e-3 * scale)[0]:
+        order = np.argsort(np.abs(z[:, j]))[:4]
+        cand = [int(b) for b in order if abs(z[b, j]) < BAND_MAX]
+        if not cand:
+            continue
+        eff = {b: (-dz[b, j] if on[b, j] else float(MO.bf16(pre[b:b + 1, j])[0])) for b in cand}
+        best, best_r = None, abs(diff[j])
+        subsets = [(b,) for b in cand] + [(b, c) for i, b in enumerate(cand) for c in cand[i + 1:]]
+        for sub in subsets:
+            r = abs(diff[j] - sum(eff[b] for b in sub))
+            if r < best_r:
+                best, best_r = sub, r
+        if best is not None and best_r < 0.1 * abs(diff[j]):
+            flips += [(layer, b, int(j), float(abs(z[b, j]))) for b in best]
+    return flips
+
+
+def match_decisions(flat, X, y, dims, db1_dev, db2_dev, with_mid=False):
+    """The oracle's loss and gradient with the ReLU decisions of near-zero units (|z| < BAND_MAX) taken as
+    the device took them.  Returns (canonical loss, canonical gradient, matched loss, matched gradient, flips);
+    flips = [(layer, sample, unit, |z|)].  Layer 2 first (its gates feed layer 1's dz), then layer 1.
+    With `with_mid` the intermediates of the matched evaluation are returned as a sixth value."""
+    segs, _ = I.mlp_segments(dims)
+    off = {n: o for n, o, _ in segs}
+    d1, d2 = dims[1], dims[2]
+    loss0, g0, mid = MO.loss_and_grad(flat, X, y, dims, True, return_intermediates=True)
+    loss, g = loss0, g0
+    f2 = _decode_layer(2, db2_dev, g[off["b2"]:off["b2"] + d2], mid["z2"], mid["on2"], mid["dz2"], mid["pre2"])
+    if f2:
+        loss, g, mid = MO.loss_and_grad(flat, X, y, dims, True, flips=[f[:3] for f in f2], return_intermediates=True)
+    f1 = _decode_layer(1, db1_dev, g[off["b1"]:off["b1"] + d1], mid["z1"], mid["on1"], mid["dz1"], mid["pre1"])
+    if f1:
+        loss, g, mid = MO.loss_and_grad(flat, X, y, dims, True, flips=[f[:3] for f in f2 + f1], return_intermediates=True)
+    if with_mid:
+        return loss0, g0, loss, g, f2 + f1, mid
+    return loss0, g0, loss, g, f2 + f1
+
+
+_SHAPES = {}
 
 
 def _attach(names, K, P_raw):
     from multiprocessing import shared_memory
     if "x" not in _SHM:
-        for key in ("x", "g"):
+        d_in, d_h = I.MLP_DIMS[0], I.MLP_DIMS[1]
+        shapes = {"x": ((K, P_raw), np.float32), "xb": ((K, P_raw), np.float32), "g": ((K, P_raw), np.float32),
+                  "gb": ((K, P_raw), np.float32), "X": ((K, I.MLP_BATCH, d_in), np.uint16),
+                  "y": ((K, I.MLP_BATCH), np.int32), "hint": ((K, 2, d_h), np.float32)}
+        for key, (shape, dt) in shapes.items():
             shm = shared_memory.SharedMemory(name=names[key])
             _SHM[key + "_shm"] = shm
-            _SHM[key] = np.ndarray((K, P_raw), np.float32, buffer=shm.buf)
+            _SHM[key] = np.ndarray(shape, dt, buffer=shm.buf)
         _SHM["teacher"] = I.mlp_init_params(I.MLP_TEACHER_SEED)
     return _SHM
 
 
-def _oracle_worker_step(job):
-    """One worker's Step II gradient in a child process: generates the minibatch of (worker, tau) and its
-    teacher labels, reads the worker's model from shared memory, writes the gradient there."""
+def _make_batch(job):
+    """Child process: the minibatch of (worker, tau) and its teacher labels, left in shared memory."""
     names, K, P_raw, w, tau = job
     sh = _attach(names, K, P_raw)
     X = I.mlp_batch(w, tau)
-    y = I.mlp_teacher_labels(X, sh["teacher"])
-    loss, g = MO.loss_and_grad(sh["x"][w], X, y, I.MLP_DIMS, emulate_bf16=True)
-    sh["g"][w] = g
-    return w, float(loss), I.bf16_bits(X), y
+    sh["X"][w] = I.bf16_bits(X)
+    sh["y"][w] = I.mlp_teacher_labels(X, sh["teacher"])
+    return w
+
+
+def _oracle_worker_step(job):
+    """Child process: one worker's Step II gradient, from the canonical state into `g` and -- when `match` -- from
+    the branch state into `gb` with the device's near-zero decisions (hint = the device's bias gradients)."""
+    names, K, P_raw, w, match, diverged = job
+    sh = _attach(names, K, P_raw)
+    X = (sh["X"][w].astype(np.uint32) << np.uint32(16)).view(np.float32)
+    y = sh["y"][w]
+    flips = []
+    if not match:
+        loss, g = MO.loss_and_grad(sh["x"][w], X, y, I.MLP_DIMS, emulate_bf16=True)
+        sh["g"][w] = g
+    elif not diverged:                                   # branch state == canonical state: one evaluation serves both
+        loss, g, _, gb, flips = match_decisions(sh["x"][w], X, y, I.MLP_DIMS, sh["hint"][w, 0], sh["hint"][w, 1])
+        sh["g"][w] = g
+        sh["gb"][w] = gb
+    else:
+        loss, g = MO.loss_and_grad(sh["x"][w], X, y, I.MLP_DIMS, emulate_bf16=True)
+        sh["g"][w] = g
+        _, _, _, gb, flips = match_decisions(sh["xb"][w], X, y, I.MLP_DIMS, sh["hint"][w, 0], sh["hint"][w, 1])
+        sh["gb"][w] = gb
+    return w, float(loss), flips
 
 
 class OracleLoop:
     """The oracle's round loop over all K workers, the K gradients of a step computed by a pool of
-    processes (one per worker, as many as the host has cores)."""
+    processes (one per worker, as many as the host has cores).  `eng` is the canonical oracle; `branch`
+    is the per-round branch that takes the device's near-zero ReLU decisions (see the module text)."""
 
     def __init__(self, K, lr, mu, wd, procs=None):
         import multiprocessing as mp
         from multiprocessing import shared_memory
         self.K = K
         self.P_raw = I.mlp_segments()[1]
-        nbytes = K * self.P_raw * 4
-        self.shm = {k: shared_memory.SharedMemory(create=True, size=nbytes) for k in ("x", "g")}
+        d_in, d_h = I.MLP_DIMS[0], I.MLP_DIMS[1]
+        sizes = {"x": K * self.P_raw * 4, "xb": K * self.P_raw * 4, "g": K * self.P_raw * 4, "gb": K * self.P_raw * 4,
+                 "X": K * I.MLP_BATCH * d_in * 2, "y": K * I.MLP_BATCH * 4, "hint": K * 2 * d_h * 4}
+        self.shm = {k: shared_memory.SharedMemory(create=True, size=n) for k, n in sizes.items()}
         self.names = {k: s.name for k, s in self.shm.items()}
+
+        def view(key, shape, dt):
+            return np.ndarray(shape, dt, buffer=self.shm[key].buf)
+
+        # the oracles' models live in shared memory so that the children read them without copies
         self.eng = OracleEngine(K, self.P_raw, lr, mu, wd, mode="ref")
-        # the oracle's model lives in shared memory so that the children read it without copies
-        self.eng.x = np.ndarray((K, self.P_raw), np.float32, buffer=self.shm["x"].buf)
+        self.eng.x = view("x", (K, self.P_raw), np.float32)
         self.eng.x[:] = 0
-        self.g = np.ndarray((K, self.P_raw), np.float32, buffer=self.shm["g"].buf)
+        self.branch = OracleEngine(K, self.P_raw, lr, mu, wd, mode="ref")
+        self.branch.x = view("xb", (K, self.P_raw), np.float32)
+        self.branch.x[:] = 0
+        self.g = view("g", (K, self.P_raw), np.float32)
+        self.gb = view("gb", (K, self.P_raw), np.float32)
+        self.X = view("X", (K, I.MLP_BATCH, d_in), np.uint16)
+        self.y = view("y", (K, I.MLP_BATCH), np.int32)
+        self.hint = view("hint", (K, 2, d_h), np.float32)
+        self.diverged = [False] * K
         self.procs = max(1, min(K, procs or os.cpu_count() or 1))
         saved = {v: os.environ.get(v) for v in ("OMP_NUM_THREADS", "OPENBLAS_NUM_THREADS", "MKL_NUM_THREADS")}
         for v in saved:                                  # one BLAS thread per child: the pool is the parallelism
@@ -93,20 +193,37 @@ class OracleLoop:
                 else:
                     os.environ[v] = old
 
-    def gradients(self, tau):
-        """All K workers' gradients of global step tau (left in self.g); returns (losses, X bits, labels)."""
-        jobs = [(self.names, self.K, self.P_raw, w, tau) for w in range(self.K)]
-        res = sorted(self.pool.map(_oracle_worker_step, jobs, chunksize=1))
-        losses = np.array([r[1] for r in res])
-        Xb = np.stack([r[2] for r in res])
-        y = np.stack([r[3] for r in res])
-        return losses, Xb, y
+    def make_batches(self, tau):
+        """Minibatches (bf16 bit patterns) and labels of global step tau for all workers, in self.X / self.y."""
+        self.pool.map(_make_batch, [(self.names, self.K, self.P_raw, w, tau) for w in range(self.K)], chunksize=1)
+        return self.X, self.y
+
+    def gradients(self, tau=None, match=False):
+        """All K workers' gradients for the batches in self.X / self.y: canonical into self.g; with `match` also
+        the branch's into self.gb (self.hint must hold the device's bias gradients).  With `tau` the batches are
+        generated first.  Returns (canonical losses, X bits, labels, matched decisions)."""
+        if tau is not None:
+            self.make_batches(tau)
+        jobs = [(self.names, self.K, self.P_raw, w, match, self.diverged[w]) for w in range(self.K)]
+        res = sorted(self.pool.map(_oracle_worker_step, jobs, chunksize=1), key=lambda r: r[0])
+        flips = []
+        for w, _, f in res:
+            if f:
+                self.diverged[w] = True
+                flips += [(w,) + tuple(t) for t in f]
+        return np.array([r[1] for r in res]), self.X, self.y, flips
+
+    def start_branch_round(self):
+        """The branch takes the canonical oracle's state (Step I follows on both)."""
+        self.branch.x[:] = self.eng.x
+        self.branch.v[:] = self.eng.v
+        self.diverged = [False] * self.K
 
     def close(self):
         self.pool.close()
         self.pool.join()
-        self.eng.x = None
-        self.g = None
+        self.eng.x = self.branch.x = None
+        self.g = self.gb = self.X = self.y = self.hint = None
         for s in self.shm.values():
             s.close()
             s.unlink()
@@ -150,7 +267,11 @@ def run(rounds=200, K=16, k=4, lr=0.05, mu=0.9, wd=0.0, procs=None, log=None):
     first_break = {n: None for n in names}
     t0 = time.perf_counter()
     t_oracle = 0.0
+    segs, _ = I.mlp_segments(dims)
+    off = {n: o for n, o, _ in segs}
+    n_matched, max_z = 0, 0.0
     for r in range(rounds):
+        ora.start_branch_round()
         if r > 0:                                        # the restarted engines take the oracle's state
             pad_x[:, :P_raw] = ora.eng.x
             pad_v[:, :P_raw] = ora.eng.v
@@ -160,12 +281,13 @@ def run(rounds=200, K=16, k=4, lr=0.05, mu=0.9, wd=0.0, procs=None, log=None):
         for e in engines:
             e.comm_begin(side)
         ora.eng.comm_begin()
+        ora.branch.comm_begin()
         round_loss = {"oracle": [], "two-call": [], "fused": []}
+        round_flips = []
         for s in range(k):
             tau = r * k + s
             t1 = time.perf_counter()
-            l_ref, Xb, y = ora.gradients(tau)
-            ora.eng.local_step(ora.g)
+            Xb, y = ora.make_batches(tau)
             t_oracle += time.perf_counter() - t1
             X = torch.from_numpy(Xb.view(np.int16)).cuda().view(torch.bfloat16)
             yd = torch.from_numpy(y).cuda()
@@ -173,22 +295,36 @@ def run(rounds=200, K=16, k=4, lr=0.05, mu=0.9, wd=0.0, procs=None, log=None):
             for i, e in enumerate(engines):
                 if i % 2 == 0:
                     mg.grad(e.bf16_shadow(), X, yd, grads, loss_d)
+                    if i == 2:                           # the restarted engine's bias gradients: which decisions it took
+                        ora.hint[:, 0] = grads[:, off["b1"]:off["b1"] + dims[1]].cpu().numpy()
+                        ora.hint[:, 1] = grads[:, off["b2"]:off["b2"] + dims[2]].cpu().numpy()
                     e.local_step(grads)
                 else:
                     mg.grad_step(e, X, yd, loss_d)
                 l_gpu.append(loss_d.double().mean().item())
+            t1 = time.perf_counter()
+            l_ref, _, _, flips = ora.gradients(match=True)
+            ora.eng.local_step(ora.g)
+            ora.branch.local_step(ora.gb)
+            t_oracle += time.perf_counter() - t1
+            round_flips += flips
             round_loss["oracle"].append(float(l_ref.mean()))
             round_loss["two-call"].append(l_gpu[0])
             round_loss["fused"].append(l_gpu[1])
         for e in engines:
             e.comm_end()
         ora.eng.comm_end()
-        want = I.round_to_bf16(ora.eng.x)
-        row = {"round": r + 1}
+        ora.branch.comm_end()
+        row = {"round": r + 1, "matched_decisions": len(round_flips),
+               "matched_max_abs_z": max([f[4] for f in round_flips], default=0.0)}
+        n_matched += len(round_flips)
+        max_z = max(max_z, row["matched_max_abs_z"])
         for key in round_loss:
             steps[key] += round_loss[key]
             row["loss_" + key] = float(np.mean(round_loss[key]))
         for n, e in zip(names, engines):
+            ref_eng = ora.branch if n.startswith("restart") else ora.eng
+            want = I.round_to_bf16(ref_eng.x)
             got = e.bf16_shadow().float().cpu().numpy()
             assert np.all(got[:, P_raw:] == 0)
             worst, share = scaled_error(got[:, :P_raw], want)
@@ -198,11 +334,12 @@ def run(rounds=200, K=16, k=4, lr=0.05, mu=0.9, wd=0.0, procs=None, log=None):
                 first_break[n] = r + 1
             if n.startswith("restart"):                  # the momentum after one round from the oracle's state, in norm
                 vg = e.get_momentum().cpu().numpy()[:, :P_raw].astype(np.float64)
-                row[n + " v_relL2"] = float(np.linalg.norm(vg - ora.eng.v) / np.linalg.norm(ora.eng.v))
+                row[n + " v_relL2"] = float(np.linalg.norm(vg - ref_eng.v) / np.linalg.norm(ref_eng.v))
         table.append(row)
         if log:
             log(f"round {r + 1:3d}: loss gpu {row['loss_two-call']:.5f} / {row['loss_fused']:.5f} oracle {row['loss_oracle']:.5f}"
-                f" | free {row[names[0]]:.2e} {row[names[1]]:.2e} | restarted {row[names[2]]:.2e} {row[names[3]]:.2e}")
+                f" | free {row[names[0]]:.2e} {row[names[1]]:.2e} | restarted {row[names[2]]:.2e} {row[names[3]]:.2e}"
+                f" | decisions matched {row['matched_decisions']} (|z| <= {row['matched_max_abs_z']:.1e})")
     mg.check()
     for e in engines:
         e.destroy()
@@ -214,7 +351,8 @@ def run(rounds=200, K=16, k=4, lr=0.05, mu=0.9, wd=0.0, procs=None, log=None):
             "first_round_outside_1e-2": first_break, "max_relative_loss_gap": gap, "oracle_processes": procs_used,
             "oracle_seconds": t_oracle, "wall_seconds": time.perf_counter() - t0,
             "worst_restarted": {n: max(row[n] for row in table) for n in names[2:]},
-            "worst_restarted_v_relL2": {n: max(row[n + " v_relL2"] for row in table) for n in names[2:]}}
+            "worst_restarted_v_relL2": {n: max(row[n + " v_relL2"] for row in table) for n in names[2:]},
+            "matched_decisions": n_matched, "matched_max_abs_z": max_z, "relu_decisions_per_round": K * k * B * (dims[1] + dims[2])}
 
 
 def markdown(res, command):
@@ -226,22 +364,26 @@ def markdown(res, command):
            "over the k steps of the round.  Error = largest |gpu - ref| / max(|ref|, rms(ref)) over the bf16 parameters of all "
            "workers after the merge (a one-ulp bf16 difference is 3.9e-3 to 7.8e-3 of the element); `share` = fraction of the "
            "parameters outside 1e-2.  `free` engines run from the common initial point without ever seeing the oracle's "
-           "state; `restart` engines start every round from the oracle's x and v.", "",
+           "state and are compared with the canonical oracle; `restart` engines start every round from the canonical "
+           "oracle's x and v and are compared with the oracle branch that takes, for hidden units with |z| < 5e-4 only, "
+           "the ReLU decision the device took (`matched`: how many such decisions in the round, and their largest |z|).", "",
            f"Oracle loop: {res['oracle_processes']} processes, {res['oracle_seconds']:.0f} s of {res['wall_seconds']:.0f} s.", "",
            f"* largest restarted-per-round error: two-call {res['worst_restarted'][names[2]]:.2e}, fused {res['worst_restarted'][names[3]]:.2e} (bar 1e-2); "
            f"momentum after such a round, relative L2 distance to the oracle's: {res['worst_restarted_v_relL2'][names[2]]:.2e}, {res['worst_restarted_v_relL2'][names[3]]:.2e}",
            f"* first round with a free-running parameter outside 1e-2: two-call {res['first_round_outside_1e-2'][names[0]]}, "
            f"fused {res['first_round_outside_1e-2'][names[1]]}",
            f"* largest relative loss gap over all {res['rounds'] * res['k']} steps: two-call {res['max_relative_loss_gap']['two-call']:.2e}, "
-           f"fused {res['max_relative_loss_gap']['fused']:.2e} (bar 2e-2)", "",
-           "| round | loss two-call | loss fused | loss oracle | free two-call (share) | free fused (share) | restart two-call | restart fused |",
-           "|---|---|---|---|---|---|---|---|"]
+           f"fused {res['max_relative_loss_gap']['fused']:.2e} (bar 2e-2)",
+           f"* ReLU decisions matched to the device's over the whole run: {res['matched_decisions']} of "
+           f"{res['relu_decisions_per_round'] * res['rounds']:.3g} taken, largest |z| among them {res['matched_max_abs_z']:.1e}", "",
+           "| round | loss two-call | loss fused | loss oracle | free two-call (share) | free fused (share) | restart two-call | restart fused | matched (max abs z) |",
+           "|---|---|---|---|---|---|---|---|---|"]
     R = res["rounds"]
     show = [row for row in res["table"] if row["round"] <= 10 or row["round"] % 10 == 0 or row["round"] == R]
     for row in show:
         out.append(f"| {row['round']} | {row['loss_two-call']:.5f} | {row['loss_fused']:.5f} | {row['loss_oracle']:.5f} | "
                    f"{row[names[0]]:.2e} ({row[names[0] + ' share>1e-2']:.1e}) | {row[names[1]]:.2e} ({row[names[1] + ' share>1e-2']:.1e}) | "
-                   f"{row[names[2]]:.2e} | {row[names[3]]:.2e} |")
+                   f"{row[names[2]]:.2e} | {row[names[3]]:.2e} | {row['matched_decisions']} ({row['matched_max_abs_z']:.1e}) |")
     out.append("")
     out.append("(rounds 1-10, then every tenth; the JSON written beside this table holds every round and every step's loss.)")
     return "\n".join(out) + "\n"

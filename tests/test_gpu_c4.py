@@ -15,11 +15,16 @@ def test_first_rounds_of_the_stated_run_match_the_oracle_loop():
     res = C.run(rounds=rounds, K=16, k=4, log=print)
     names = ["free/two-call", "free/fused", "restart/two-call", "restart/fused"]
     for row in res["table"]:
-        # per-round parity: one whole round (Step I, 4 x Step II, line 6) from the oracle's state, bf16 parameters
+        # per-round parity: one whole round (Step I, 4 x Step II, line 6) from the oracle's state, bf16 parameters,
+        # against the oracle with the near-zero ReLU decisions taken as the device took them
         assert row[names[2]] <= 1e-2 and row[names[3]] <= 1e-2, row
-        assert row[names[2] + " v_relL2"] <= 6e-2 and row[names[3] + " v_relL2"] <= 6e-2, row
+        assert row[names[2] + " v_relL2"] <= 1e-2 and row[names[3] + " v_relL2"] <= 1e-2, row
         # the two device paths take identical steps, so their free-running states stay identical
         assert row[names[0]] == row[names[1]] and row["loss_two-call"] == row["loss_fused"]
+    # about 300 of the 16.8 M ReLU decisions of a round are matched: from the second step of a round on, the two
+    # sides' bf16 copies of a few hundred weights per worker differ by one step (their fp32 masters differ in the last
+    # bits and straddle a rounding boundary), which moves the pre-activations of those units by about 1e-4
+    assert res["matched_max_abs_z"] < C.BAND_MAX and res["matched_decisions"] <= 5e-5 * res["relu_decisions_per_round"] * rounds
     assert res["max_relative_loss_gap"]["two-call"] <= 2e-2 and res["max_relative_loss_gap"]["fused"] <= 2e-2
     steps = res["loss_per_step"]
     assert len(steps["oracle"]) == rounds * 4

@@ -200,45 +200,53 @@ def decision_slack(params, X, y, dims, z1, z2):
 
 
 def test_gradient_on_workload_shaped_weights(M):
-    """The workload's own recipe (Gaussian weights, K = 16, full size), element by element.  Every gradient element
-    must lie within 1e-2 (scaled) of the oracle's, except where a floating-point decision of the forward pass is
-    within accumulation error of falling the other way; there the element may additionally move by exactly the
-    terms that decision switches (decision_slack), and by nothing else."""
+    """The workload's own recipe (Gaussian weights, K = 16, full size), element by element at 1e-2.  ReLU is a
+    decision that floating point takes: for the few hidden units whose pre-activation lies within accumulation
+    error of zero (|z| < 5e-4 is the admitted band), fp32 and fp64 accumulation can decide differently, both
+    correctly, and one such decision switches a whole sample's term.  The oracle is therefore evaluated with
+    those decisions taken as the device took them (read off the device's bias gradients, the column sums of dz:
+    c4_loss_curve.match_decisions); every one of the 29.8 M gradient elements must then agree within 1e-2, plus --
+    for the one-in-a-million element that a single sample's term dominates -- one bf16 step (2^-7) of its largest
+    term: dz is STORED in bf16, and whether a dz value rounds up or down is again decided by the last bits of an
+    accumulation, so a gradient element g = sum_b dz[b] * in[b] may differ by one bf16 step of one term."""
+    import c4_loss_curve as C
     K, dims = 16, I.MLP_DIMS
     params, X, y, P_raw = make_problem(K, dims, seed=3)
     g, loss, _ = run_gpu_grad(M, K, dims, params, X, y)
     segs, _ = I.mlp_segments(dims)
-    n_out = n_slack = n_el = 0
-    units = [0, 0]
-    worst_plain = 0.0
+    off = {n: o for n, o, _ in segs}
+    matched, worst, outside_plain, n_term = [], 0.0, 0, 0
     for w in range(K):
-        ref_loss, ref_g, (z1, z2) = MO.loss_and_grad(params[w], X[w], y[w], dims, emulate_bf16=True,
-                                                     return_preactivations=True)
-        assert abs(loss[w] - ref_loss) <= 2e-3 * abs(ref_loss)
-        slack, a1, a2 = decision_slack(params[w], X[w], y[w], dims, z1, z2)
-        units[0] += a1
-        units[1] += a2
-        for name, off, shape in segs:
+        hint1 = g[w, off["b1"]:off["b1"] + dims[1]]
+        hint2 = g[w, off["b2"]:off["b2"] + dims[2]]
+        ref_loss, g_plain, m_loss, ref_g, flips, mid = C.match_decisions(params[w], X[w], y[w], dims, hint1, hint2,
+                                                                         with_mid=True)
+        matched += [(w,) + tuple(f) for f in flips]
+        assert abs(loss[w] - m_loss) <= 2e-3 * abs(m_loss) and abs(loss[w] - ref_loss) <= 2e-3 * abs(ref_loss)
+        operands = {"W1": (mid["dz1"], X[w].astype(np.float64)), "W2": (mid["dz2"], mid["h1"]), "W3": (mid["dz3"], mid["h2"]),
+                    "b1": (mid["dz1"], None), "b2": (mid["dz2"], None), "b3": (mid["dz3"], None)}
+        for name, o, shape in segs:
             n = int(np.prod(shape))
-            got = g[w, off:off + n].astype(np.float64).reshape(shape)
-            want = ref_g[off:off + n].astype(np.float64).reshape(shape)
+            got, want = g[w, o:o + n].astype(np.float64), ref_g[o:o + n].astype(np.float64)
             scale = np.maximum(np.abs(want), np.sqrt(np.mean(want ** 2)))
-            diff = np.abs(got - want)
-            bad = diff > 1e-2 * scale + slack[name]
-            assert not bad.any(), (f"worker {w} d{name}: {int(bad.sum())} elements outside 1e-2 that no decision within reach "
-                                   f"explains; worst {float((diff / scale)[bad].max()):.2e}")
-            outside = diff > 1e-2 * scale
-            n_out += int(outside.sum())
-            n_slack += int((slack[name] > 1e-2 * scale).sum())
-            n_el += n
-            untouched = slack[name] == 0
-            if untouched.any():
-                worst_plain = max(worst_plain, float((diff / scale)[untouched].max()))
-    n_units = K * 128 * (dims[1] + dims[2])
-    assert units[0] + units[1] <= 2e-3 * n_units, "too many hidden units counted as within reach of a decision"
-    print(f"workload-shaped gradients, {n_el} elements: {n_out} outside 1e-2, all of them explained by one of "
-          f"{units[0]} + {units[1]} hidden units (layers 1 + 2, of {n_units}) whose ReLU decision is within accumulation "
-          f"error; {n_slack} elements could have moved by more than 1e-2; worst scaled error elsewhere {worst_plain:.2e}")
+            err = np.abs(got - want) / scale
+            over = np.nonzero(err > 1e-2)[0]
+            if over.size:                                  # admitted only as one bf16 step of the element's largest term
+                dz, inp = operands[name]
+                rows, cols = (over // shape[-1], over % shape[-1]) if inp is not None else (over, None)
+                terms = np.abs(dz[:, rows]) * (np.abs(inp[:, cols]) if inp is not None else 1.0)
+                assert np.all(np.abs(got - want)[over] <= 1e-2 * scale[over] + 2.0 ** -7 * terms.max(axis=0)), f"worker {w} d{name}"
+                n_term += over.size
+            worst = max(worst, float(err.max()))
+            want = g_plain[o:o + n].astype(np.float64)
+            scale = np.maximum(np.abs(want), np.sqrt(np.mean(want ** 2)))
+            outside_plain += int((np.abs(g[w, o:o + n] - want) > 1e-2 * scale).sum())
+    assert all(f[4] < C.BAND_MAX for f in matched)
+    assert len(matched) <= 1e-4 * K * 128 * (dims[1] + dims[2]) and n_term <= 1e-5 * K * P_raw
+    print(f"workload-shaped gradients: all {K * P_raw} elements within 1e-2 (worst {worst:.2e}; {n_term} of them only with one "
+          f"bf16 step of their largest term added) once {len(matched)} of "
+          f"{K * 128 * (dims[1] + dims[2])} ReLU decisions are taken as the device took them (largest |z| among them "
+          f"{max([f[4] for f in matched], default=0):.1e}); with the oracle's own decisions {outside_plain} elements lie outside")
 
 
 def test_labels_from_the_teacher_and_identical_workers_give_identical_gradients(M):

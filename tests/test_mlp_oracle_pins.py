@@ -115,3 +115,49 @@ def test_workload_recipe_shapes_and_labels():
     assert X.shape == (128, 784) and np.array_equal(I.round_to_bf16(X), X)
     y = I.mlp_teacher_labels(X, t)
     assert y.shape == (128,) and y.min() >= 0 and y.max() <= 9 and len(set(y.tolist())) > 3
+
+
+def test_a_flipped_relu_decision_is_the_gradient_of_the_network_with_that_gate_fixed():
+    """`flips` takes a ReLU decision the other way.  Pin: with the gates g = (z > 0) treated as constants, the network
+    is h = g * z, whose gradient torch's autograd gives for ANY gate pattern; for units whose pre-activation is (made)
+    1e-9 away from zero, the oracle's flipped result must equal that gradient with the flipped gates, and the
+    unflipped result the one with the original gates.  The intermediates it reports obey their definitions."""
+    torch = pytest.importorskip("torch")
+    flat, X, y = tiny_problem(5, M=12)
+    segs, _ = I.mlp_segments(DIMS)
+    off = dict((n, o) for n, o, _ in segs)
+    # put z1[2][3] at -1e-9 and z2[7][1] at +1e-9 by moving the two biases (other samples keep ordinary values)
+    _, _, mid = MO.loss_and_grad(flat, X, y, DIMS, False, return_intermediates=True)
+    flat[off["b1"] + 3] -= mid["z1"][2, 3] + 1e-9
+    _, _, mid = MO.loss_and_grad(flat, X, y, DIMS, False, return_intermediates=True)
+    flat[off["b2"] + 1] -= mid["z2"][7, 1] - 1e-9
+    loss0, g0, mid = MO.loss_and_grad(flat, X, y, DIMS, False, return_intermediates=True)
+    assert abs(mid["z1"][2, 3] + 1e-9) < 1e-12 and abs(mid["z2"][7, 1] - 1e-9) < 1e-12
+    assert not mid["on1"][2, 3] and mid["on2"][7, 1]
+    flips = [(1, 2, 3), (2, 7, 1)]
+    loss1, g1, mid1 = MO.loss_and_grad(flat, X, y, DIMS, False, flips=flips, return_intermediates=True)
+    assert mid1["on1"][2, 3] and not mid1["on2"][7, 1] and mid1["h2"][7, 1] == 0
+    assert (mid1["on1"] != mid["on1"]).sum() == 1 and (mid1["on2"] != mid["on2"]).sum() == 1
+
+    def gated(on1, on2):
+        t = torch.tensor(flat, dtype=torch.float64, requires_grad=True)
+        p = {n: t[o:o + int(np.prod(s))].reshape(s) for n, o, s in segs}
+        h = (torch.tensor(X) @ p["W1"].T + p["b1"]) * torch.tensor(on1, dtype=torch.float64)
+        h = (h @ p["W2"].T + p["b2"]) * torch.tensor(on2, dtype=torch.float64)
+        L = torch.nn.functional.cross_entropy(h @ p["W3"].T + p["b3"], torch.tensor(y), reduction="mean")
+        L.backward()
+        return L.item(), t.grad.numpy()
+
+    for (loss, g, m) in ((loss0, g0, mid), (loss1, g1, mid1)):
+        want_l, want_g = gated(m["on1"], m["on2"])
+        assert abs(want_l - loss) < 1e-8
+        np.testing.assert_allclose(g, want_g, rtol=0, atol=1e-7)
+    assert np.abs(g1 - g0).max() > 1e-4                  # the flip matters: one sample's term switched
+    # definitions of the reported intermediates
+    p = MO.split(flat, DIMS)
+    np.testing.assert_allclose(mid["pre2"], mid["dz3"] @ p["W3"], atol=1e-15)
+    np.testing.assert_allclose(mid["dz2"], mid["pre2"] * mid["on2"], atol=0)
+    np.testing.assert_allclose(mid["pre1"], mid["dz2"] @ p["W2"], atol=1e-15)
+    np.testing.assert_allclose(mid["dz1"], mid["pre1"] * mid["on1"], atol=0)
+    np.testing.assert_allclose(g0[off["b2"]:off["W3"]], mid["dz2"].sum(0), atol=1e-7)
+    np.testing.assert_allclose(g0[off["b1"]:off["W2"]], mid["dz1"].sum(0), atol=1e-7)
