@@ -53,6 +53,10 @@ def parse():
                          "over peer addresses")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--repeats", type=int, default=5, help="how many times the timed block of --steps rounds is repeated "
+                                                           "(the line reports the median block, and min and max)")
+    ap.add_argument("--no-other-workloads", action="store_true",
+                    help="default run only: skip the VGG16-sized and MLP digests added under other_workloads")
     ap.add_argument("--cpu-sample-cols", type=int, default=1 << 20)
     ap.add_argument("--sweep-K", default="2,8,16,32,64")
     ap.add_argument("--sweep-logP", default="20,24,26,28")
@@ -188,37 +192,28 @@ def overlap_fraction(by):
     return cov / tot if tot > 0 else None
 
 
-def run_ours(args, wl):
+def median(xs):
+    xs = sorted(xs)
+    n = len(xs)
+    return xs[n // 2] if n % 2 else 0.5 * (xs[n // 2 - 1] + xs[n // 2])
+
+
+def load_peaks():
+    try:
+        return json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        return {}
+
+
+def measure_param_workload(args, wl, ctx, *, ring_n, do_e2e, cpu_seconds, do_graph, do_schemes, sampler=None):
+    """One parameter-path workload on this rank: the timed blocks, the per-kernel passes, and the optional legs.
+    ctx: dict(rank, world, barrier, dist).  Returns the pieces of the JSON line."""
     import torch
-    import torch.distributed as dist
-    from paper_1906_12043_b200 import build, engine as E, inputs as I, workloads as W
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the engine has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    if rank == 0:
-        build.build()
-    if world > 1:
-        dist.barrier()
-    E.load()
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
+    from paper_1906_12043_b200 import engine as E, inputs as I, workloads as W
+    rank, world, barrier, dist = ctx["rank"], ctx["world"], ctx["barrier"], ctx["dist"]
     K, P, k = wl.K, wl.P, wl.k
     p0 = rank * P                                       # this rank's columns of the global vector
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except OSError:
-        pass
+    peaks = load_peaks()
     hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
     peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
 
@@ -228,7 +223,7 @@ def run_ours(args, wl):
     I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, p0, wl.sigma_x0)
     eng.set_params(x0)
     ring = []
-    for t in range(max(1, args.ring)):
+    for t in range(max(1, ring_n)):
         g = torch.empty((K, P), dtype=torch.float32, device="cuda")
         I.device_gradients_into(g, t, wl.sigma_g, p0=p0)
         ring.append(g)
@@ -243,11 +238,14 @@ def run_ours(args, wl):
             step_no[0] += 1
         eng.comm_end()
 
-    # ---- device-resident timed region
-    for _ in range(max(3, args.warmup)):
+    # ---- device-resident timed region: `repeats` blocks of exactly `steps` rounds, each bracketed by a barrier and a
+    #      synchronize on both sides; no per-kernel events inside (those are taken in passes of their own below)
+    warm = max(3, args.warmup)
+    for _ in range(warm):
         one_round(side)
     graph = None
-    if args.graph:
+    steps = args.steps
+    if args.graph and do_graph:
         # two rounds = one full cycle of the buffer flip; the side-stream mean is captured with them
         cap = torch.cuda.Stream()
         eng.sync()
@@ -266,39 +264,34 @@ def run_ours(args, wl):
         for _ in range(3):
             graph.replay()
         torch.cuda.synchronize()
-    else:
-        eng.set_option(E.OPT_PROFILE, 1)
-        eng.profile_reset()
-    barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    launches0 = eng.launch_count
+        steps = max(2, steps // 2 * 2)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(compute)
+    block_ms, launches = [], 0
+    for rep in range(max(1, args.repeats)):
+        barrier()
+        launches0 = eng.launch_count
+        ev0.record(compute)
+        if graph is not None:
+            for _ in range(steps // 2):
+                graph.replay()
+        else:
+            for _ in range(steps):
+                one_round(side)
+        ev1.record(compute)
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        block_ms.append(ms)
+        launches = launches_per_replay * (steps // 2) if graph is not None else eng.launch_count - launches0
     if graph is not None:
-        args.steps = max(2, args.steps // 2 * 2)
-        for _ in range(args.steps // 2):
-            graph.replay()
-    else:
-        for _ in range(args.steps):
-            one_round(side)
-    ev1.record(compute)
-    barrier()
-    clocks = sampler.stop() if sampler else None
-    ms = ev0.elapsed_time(ev1)
-    if graph is not None:
-        launches = launches_per_replay * (args.steps // 2)
-        by = {}
         eng.sync()
         eng.set_stream(compute)
-    else:
-        launches = eng.launch_count - launches0
-        by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
-        eng.set_option(E.OPT_PROFILE, 0)
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * K * P * k * args.steps / (ms * 1e-3)
+    ms = median(block_ms)
+    value = world * K * P * k * steps / (ms * 1e-3)
+    clocks = sampler.stop() if sampler else None
 
     alg_bytes = {"local_step": W.BYTES_LOCAL_STEP * K * P, "snapshot": W.BYTES_SNAPSHOT * K * P,
                  "mean": W.bytes_mean(K) * K * P, "merge": W.bytes_merge(K) * K * P}
@@ -312,14 +305,26 @@ def run_ours(args, wl):
                          "frac_of_peak": round(gbs / hbm_peak, 4)}
         return out
 
-    in_loop = kernel_table(by)
-    overlap = overlap_fraction(by)
-
-    # ---- the same rounds with the mean on the compute stream: isolated kernel times, serial round time
+    # ---- the same rounds with per-kernel CUDA events and the kernels' own time stamps (overlapped, then serial)
+    n_prof = min(steps, 50)
     eng.set_option(E.OPT_PROFILE, 1)
     eng.profile_reset()
     torch.cuda.synchronize()
-    n_ser = min(args.steps, 50)
+    ev0.record(compute)
+    for _ in range(n_prof):
+        one_round(side)
+    ev1.record(compute)
+    torch.cuda.synchronize()
+    ms_profiled = ev0.elapsed_time(ev1) / n_prof
+    by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+    by_dev = summarize_profile(eng.profile_device_records(), E.KERNEL_NAMES)
+    in_loop = kernel_table(by)
+    in_loop_dev = kernel_table(by_dev)
+    overlap = overlap_fraction(by)
+    overlap_dev = overlap_fraction(by_dev)
+    eng.profile_reset()
+    torch.cuda.synchronize()
+    n_ser = min(steps, 50)
     ev0.record(compute)
     for _ in range(n_ser):
         one_round(compute)
@@ -328,6 +333,16 @@ def run_ours(args, wl):
     ms_serial = ev0.elapsed_time(ev1) / n_ser
     isolated = kernel_table(summarize_profile(eng.profile_records(), E.KERNEL_NAMES))
     eng.set_option(E.OPT_PROFILE, 0)
+    # serial round WITHOUT the event brackets: the figure that compares with the headline block
+    for _ in range(2):
+        one_round(compute)
+    torch.cuda.synchronize()
+    ev0.record(compute)
+    for _ in range(n_ser):
+        one_round(compute)
+    ev1.record(compute)
+    torch.cuda.synchronize()
+    ms_serial_plain = ev0.elapsed_time(ev1) / n_ser
 
     # ---- the paper's sequential counterparts on the same kernels: k local steps + blocking averaging
     #      (Local-SGD) and k steps of gradient averaging (S-SGD); for context next to the decoupled round
@@ -353,12 +368,14 @@ def run_ours(args, wl):
             eng.ssgd_step(ring[step_no[0] % len(ring)])
             step_no[0] += 1
 
-    n_cmp = min(args.steps, 30)
-    schemes = {"cocod": ms / args.steps, "local_sgd": timed(local_sgd_round, n_cmp), "ssgd": timed(ssgd_round, n_cmp)}
+    schemes = None
+    if do_schemes:
+        n_cmp = min(steps, 30)
+        schemes = {"cocod": ms / steps, "local_sgd": timed(local_sgd_round, n_cmp), "ssgd": timed(ssgd_round, n_cmp)}
 
     # ---- the same rounds replayed from a CUDA graph (extra figure; the contract value stays the eager one)
     graph_extra = None
-    if graph is None and world == 1:
+    if graph is None and world == 1 and do_graph:
         cap = torch.cuda.Stream()
         eng.sync()
         eng.set_stream(cap)
@@ -373,7 +390,7 @@ def run_ours(args, wl):
         for _ in range(3):
             g2.replay()
         torch.cuda.synchronize()
-        n_rep = max(1, min(args.steps, 200) // 2)
+        n_rep = max(1, min(steps, 200) // 2)
         ev0.record(compute)
         for _ in range(n_rep):
             g2.replay()
@@ -388,15 +405,16 @@ def run_ours(args, wl):
     dom = "local_step"
     traffic = W.NCU_DRAM_BYTES_PER_WORKER_PARAM.get(dom)
     traffic = traffic * K * P if traffic is not None else None
-    dom_tab = in_loop.get(dom) or isolated.get(dom, {})      # graph replays carry no per-kernel events
+    dom_tab = in_loop.get(dom) or isolated.get(dom, {})
     roofline = {"bound": "hbm", "kernel": dom, "achieved": dom_tab.get("gbs"), "peak": hbm_peak,
                 "unit": "GB/s", "frac": dom_tab.get("frac_of_peak"), "traffic": traffic,
                 "peak_kind": peak_kind, "algorithmic_bytes_per_launch": alg_bytes[dom],
-                "avg_launch_ms": dom_tab.get("avg_ms"), "isolated": isolated.get(dom)}
+                "avg_launch_ms": dom_tab.get("avg_ms"), "isolated": isolated.get(dom),
+                "measured_in": "a pass of its own with per-kernel CUDA events, mean kernel overlapping on the side stream"}
 
     # ---- end to end through the host-buffer entry point
     e2e = None
-    if not args.no_e2e:
+    if do_e2e:
         host_ring = []
         for t in range(2):
             hbuf = torch.empty((K, P), dtype=torch.float32, pin_memory=True)
@@ -413,7 +431,7 @@ def run_ours(args, wl):
             eng.comm_end()
             eng.get_mean(mean_out)                      # device -> host read of the round's result
 
-        n_e2e = max(1, min(args.steps, 20))
+        n_e2e = max(1, min(steps, 20))
         for _ in range(2):
             one_round_host()
         barrier()
@@ -432,39 +450,114 @@ def run_ours(args, wl):
         e2e = {"value": world * K * P * k * n_e2e / (ms_e2e * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": k * K * P * 4, "d2h_bytes_per_step": P * 4,
                "rounds": n_e2e, "ms_per_step": ms_e2e / n_e2e, "wall_ms_per_step": wall * 1e3 / n_e2e}
+        del host_ring, mean_out
+
+    eng.destroy()
+    del ring, x0
+    torch.cuda.empty_cache()
 
     # ---- CPU oracle beside it (rank 0, N = 1 only)
     cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and cpu_seconds > 0:
         cols = min(args.cpu_sample_cols, P)
-        target_s = 12.0
         probe, s_per_round, cores = time_oracle(wl, cols, 2, 1)
-        n_rounds = max(2, min(200, int(target_s / max(s_per_round, 1e-6))))
+        n_rounds = max(2, min(200, int(cpu_seconds / max(s_per_round, 1e-6))))
         v, s_per_round, cores = time_oracle(wl, cols, n_rounds, 1)
         cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"{K} workers x first {cols} of {P} columns, {n_rounds} rounds of k={k} "
                                   f"(ref-mode oracle, OpenMP over columns, gradients pre-generated)"}
 
+    return {
+        "value": value, "steps": steps, "ms_per_step": ms / steps,
+        "timed_blocks": {"repeats": len(block_ms), "rounds_per_block": steps,
+                         "ms_per_step": [b / steps for b in block_ms], "ms_per_step_median": ms / steps,
+                         "ms_per_step_min": min(block_ms) / steps, "ms_per_step_max": max(block_ms) / steps,
+                         "reported": "median block"},
+        "config": {"workload": wl.name, "K": K, "P": P, "k": k, "lr": wl.lr, "mu": wl.mu, "wd": wl.wd,
+                   "snapshot": args.snapshot, "gradient_ring": max(1, ring_n),
+                   "cuda_graph": bool(graph is not None),
+                   "l2": "inputs larger than L2 (each K x P buffer is %.0f MB, L2 is 126 MB)" % (K * P * 4 / 1e6)
+                         if K * P * 4 > 126e6 else "L2-resident workload: not an HBM number",
+                   "sharding": "columns, no exchange" if world > 1 else "single GPU"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "kernels_in_loop": in_loop, "kernels_in_loop_device_stamps": in_loop_dev, "kernels_isolated": isolated,
+        "overlap_fraction": overlap, "overlap_fraction_device_stamps": overlap_dev,
+        "ms_per_round_overlapped": ms / steps, "ms_per_round_serial": ms_serial_plain,
+        "ms_per_round_profiled": {"overlapped": ms_profiled, "serial": ms_serial},
+        "cuda_graph_replay": graph_extra, "ms_per_round_by_scheme": schemes,
+        "hbm_gbs_whole_round": wl.bytes_per_round(args.snapshot == "copy") / (ms / steps * 1e-3) / 1e9,
+    }
+
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_1906_12043_b200 import build, engine as E
+    from paper_1906_12043_b200.workloads import WORKLOADS
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the engine has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    E.load()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    ctx = {"rank": rank, "world": world, "barrier": barrier, "dist": dist}
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    res = measure_param_workload(args, wl, ctx, ring_n=args.ring, do_e2e=not args.no_e2e,
+                                 cpu_seconds=0 if args.no_cpu_baseline else 12.0, do_graph=True, do_schemes=True,
+                                 sampler=sampler)
+    # ---- digests of the other stated workloads, so that one default run shows all of them (N = 1 only; their
+    #      end-to-end legs are left to `--workload vgg16` / `--workload mlp`)
+    other = None
+    default_run = (wl.name == "resnet18" and world == 1 and not args.graph and not args.no_other_workloads)
+    if default_run:
+        other = {}
+        saved = (args.steps, args.repeats)
+        try:
+            args.steps = max(2, min(saved[0], 10))
+            v = measure_param_workload(args, WORKLOADS["vgg16"], ctx, ring_n=2, do_e2e=False,
+                                       cpu_seconds=0 if args.no_cpu_baseline else 6.0, do_graph=False, do_schemes=False,
+                                       sampler=ClockSampler(local_rank))
+            other["vgg16"] = {key: v[key] for key in ("value", "steps", "ms_per_step", "timed_blocks", "config", "clocks",
+                                                      "gpu_launches", "roofline", "cpu_baseline", "kernels_in_loop",
+                                                      "kernels_isolated", "overlap_fraction", "overlap_fraction_device_stamps",
+                                                      "ms_per_round_serial", "hbm_gbs_whole_round")}
+            other["vgg16"].update(metric=METRIC, unit=UNIT)
+        except Exception as e:                              # e.g. a smaller GPU: say so instead of losing the headline
+            other["vgg16"] = {"unavailable": f"{type(e).__name__}: {e}"}
+        finally:
+            args.steps, args.repeats = saved
+        try:
+            args.steps = max(2, min(saved[0], 20))
+            other["mlp"] = measure_mlp(args, digest=True)
+        except Exception as e:
+            other["mlp"] = {"unavailable": f"{type(e).__name__}: {e}"}
+        finally:
+            args.steps, args.repeats = saved
+
     if rank == 0:
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": world, "steps": res["steps"],
+            "warmup": max(3, args.warmup), "ms_per_step": res["ms_per_step"], "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "K": K, "P": P, "k": k, "lr": wl.lr, "mu": wl.mu, "wd": wl.wd,
-                       "snapshot": args.snapshot, "gradient_ring": len(ring), "cuda_graph": bool(args.graph),
-                       "l2": "inputs larger than L2 (each K x P buffer is %.0f MB, L2 is 126 MB)" % (K * P * 4 / 1e6)
-                             if K * P * 4 > 126e6 else "L2-resident workload: not an HBM number",
-                       "sharding": "columns, no exchange" if world > 1 else "single GPU"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "kernels_in_loop": in_loop, "kernels_isolated": isolated,
-            "overlap_fraction": overlap, "ms_per_round_overlapped": ms / args.steps,
-            "ms_per_round_serial": ms_serial, "cuda_graph_replay": graph_extra,
-            "ms_per_round_by_scheme": schemes,
-            "hbm_gbs_whole_round": wl.bytes_per_round(args.snapshot == "copy") / (ms / args.steps * 1e-3) / 1e9,
         }
+        line.update({key: res[key] for key in res if key not in ("value", "steps", "ms_per_step")})
+        if other is not None:
+            line["other_workloads"] = other
         print(json.dumps(line))
-    eng.destroy()
     if world > 1:
         dist.destroy_process_group()
 
@@ -486,7 +579,8 @@ def run_reference_mlp(args):
     P_raw = x0.size
     oe = OracleEngine(nw, P_raw, lr, mu, wd, mode="ref")
     oe.set_params(x0)
-    ring = max(k, 8)
+    args.steps = min(args.steps, 10)                      # every (worker, step) has its own minibatch: keep the run bounded
+    ring = (args.warmup + args.steps) * k
     Xo = [[I.mlp_batch(w, t) for w in range(nw)] for t in range(ring)]
     yo = [[I.mlp_teacher_labels(Xo[t][w], teacher) for w in range(nw)] for t in range(ring)]
     tau = [0]
@@ -521,216 +615,350 @@ def run_reference_mlp(args):
     }))
 
 
-def run_mlp(args):
-    """End-to-end synthetic training: K = 16 workers each train the 784-1024-1024-10 ReLU MLP
-    (bf16 weights, fp32 master copy and momentum) on minibatches of 128; gradients come from the
-    tensor-core path, the parameter path is the same engine with its bf16 shadow switched on.
-    A step (round) = comm_begin, k = 4 x (batched gradients + local step), comm_end."""
+def _mlp_oracle_job(job):
+    """Child process of the MLP CPU-baseline leg: one worker's oracle gradient (numpy fp64, bf16 rounding points)."""
+    import numpy as np
+    from oracle import mlp_oracle as MO
+    from paper_1906_12043_b200 import inputs as I
+    flat, xbits, y = job
+    X = (xbits.astype(np.uint32) << np.uint32(16)).view(np.float32)
+    loss, g = MO.loss_and_grad(flat, X, y, I.MLP_DIMS, emulate_bf16=True)
+    return float(loss), g
+
+
+def time_mlp_oracle(K, k, rounds, lr, mu, wd, x0_raw, X_bits, y, procs):
+    """The oracle as it stands on the host cores for the first `rounds` rounds of the MLP workload, all K workers:
+    Step I, k x (numpy fp64 gradient of every worker, one process per worker, + reference-mode update), line 6.
+    X_bits: [rounds * k][K][batch][d_in] uint16 (bf16 patterns), y: [rounds * k][K][batch] int32 -- the bytes the
+    device consumed.  Returns (seconds, per-step mean losses, bf16-rounded parameters after every round)."""
+    import multiprocessing as mp
+    import numpy as np
+    from oracle.cocod_oracle import OracleEngine
+    from paper_1906_12043_b200 import inputs as I
+    P_raw = x0_raw.size
+    oe = OracleEngine(K, P_raw, lr, mu, wd, mode="ref")
+    oe.set_params(x0_raw)
+    saved = {v: os.environ.get(v) for v in ("OMP_NUM_THREADS", "OPENBLAS_NUM_THREADS", "MKL_NUM_THREADS")}
+    for v in saved:                                      # one BLAS thread per process: the pool is the parallelism
+        os.environ[v] = "1"
+    try:
+        pool = mp.get_context("spawn").Pool(procs)
+    finally:
+        for v, old in saved.items():
+            if old is None:
+                os.environ.pop(v, None)
+            else:
+                os.environ[v] = old
+    pool.map(_mlp_oracle_job, [(oe.x[w], X_bits[0][w], y[0][w]) for w in range(min(K, procs))])      # start-up, untimed
+    losses, params = [], []
+    t0 = time.perf_counter()
+    for r in range(rounds):
+        oe.comm_begin()
+        for s_ in range(k):
+            t = r * k + s_
+            res = pool.map(_mlp_oracle_job, [(oe.x[w], X_bits[t][w], y[t][w]) for w in range(K)], chunksize=1)
+            oe.local_step(np.stack([g for _, g in res]))
+            losses.append(float(np.mean([l for l, _ in res])))
+        oe.comm_end()
+        params.append(I.round_to_bf16(oe.x))
+    dt = time.perf_counter() - t0
+    pool.close()
+    pool.join()
+    return dt, losses, params
+
+
+def measure_mlp(args, digest=False):
+    """End-to-end synthetic training: K = 16 workers each train the 784-1024-1024-10 ReLU MLP (bf16 weights, fp32
+    master copy and momentum) on minibatches of 128; gradients come from the tensor-core path, the parameter path is
+    the same engine with its bf16 shadow switched on.  A step (round) = comm_begin, k = 4 x (batched gradients +
+    local step), comm_end.  Every (worker, global step) has its own seeded minibatch (a pool of up to 2048 steps,
+    generated on the device, labels from the teacher in fp64; a longer run goes through the pool again, like epochs
+    over a data set).  Three variants are timed, each from the common initial point: the two calls, the fused
+    gradient + update call, and the fused call replayed from a CUDA graph of two rounds."""
     import numpy as np
     import torch
     from paper_1906_12043_b200 import build, engine as E, inputs as I, mlp as M
     build.build()
-    torch.cuda.set_device(0)
     M.load()
-    K, k, lr, mu, wd = args.K or 16, args.k or 4, 0.05, 0.9, 0.0
+    K, k, lr, mu, wd = (16 if digest else (args.K or 16)), (4 if digest else (args.k or 4)), 0.05, 0.9, 0.0
     dims, B = I.MLP_DIMS, I.MLP_BATCH
     mg = M.MLPGrad(K, B, dims[0], dims[1], dims[3])
     P, P_raw = mg.P, mg.P_raw
     x0 = np.zeros(P, np.float32)
     x0[:P_raw] = I.mlp_init_params(I.MLP_STUDENT_SEED)
     teacher = I.mlp_init_params(I.MLP_TEACHER_SEED)
-    eng = E.Engine(K, P, lr, mu, wd)
-    eng.set_option(E.OPT_BF16_SHADOW, 1)
-    eng.set_params(x0)
-    shadow = eng.bf16_shadow()
-    ring_n = max(k, 8)
-    xs_h, ys_h = [], []
-    for t in range(ring_n):
-        X = np.stack([I.mlp_batch(w, t) for w in range(K)])
-        ys_h.append(torch.from_numpy(np.stack([I.mlp_teacher_labels(X[w], teacher) for w in range(K)])).pin_memory())
-        xs_h.append(torch.from_numpy(X).to(torch.bfloat16).pin_memory())
-    xs_d = [x.cuda() for x in xs_h]
-    ys_d = [y.cuda() for y in ys_h]
-    grads = torch.empty((K, P), dtype=torch.float32, device="cuda")
-    loss = torch.empty(K, dtype=torch.float32, device="cuda")
+    peaks = load_peaks()
+    hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
+    peak_kind = "measured" if "hbm_gbs" in peaks else "fallback"
+    steps, repeats = max(2, args.steps // 2 * 2), max(1, args.repeats)
+    n_cpu_rounds = 0 if args.no_cpu_baseline else 6
+    warm = max(3, args.warmup, n_cpu_rounds)
+    warm += warm % 2
+    need = (warm + repeats * steps) * k
+    pool_n = min(need, 2048) // (2 * k) * (2 * k)
+    pool_x = torch.empty((pool_n, K, B, dims[0]), dtype=torch.bfloat16, device="cuda")
+    I.device_mlp_batches_into(pool_x, 0)
+    pool_y = I.device_mlp_teacher_labels(pool_x, teacher)
     side = torch.cuda.Stream(priority=-1)
     compute = torch.cuda.current_stream()
-    step_no = [0]
-    losses = []
-
-    def one_round(record=False):
-        eng.comm_begin(side)
-        for _ in range(k):
-            i = step_no[0] % ring_n
-            if args.fused:
-                mg.grad_step(eng, xs_d[i], ys_d[i], loss)
-            else:
-                mg.grad(shadow, xs_d[i], ys_d[i], grads, loss)
-                eng.local_step(grads)
-            step_no[0] += 1
-            if record:
-                losses.append(loss.clone())
-        eng.comm_end()
-
-    for r in range(max(3, args.warmup)):
-        one_round(record=True)
-    torch.cuda.synchronize()
-    graph = None
-    if args.graph:
-        cap = torch.cuda.Stream()
-        eng.set_stream(cap)
-        with torch.cuda.stream(cap):
-            one_round()
-            one_round()
-        torch.cuda.synchronize()
-        step_no[0] = 0
-        lb = eng.launch_count + mg.launch_count
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=cap):
-            one_round()
-            one_round()
-        per_replay = eng.launch_count + mg.launch_count - lb
-        for _ in range(3):
-            graph.replay()
-        torch.cuda.synchronize()
-        args.steps = max(2, args.steps // 2 * 2)
-    sampler = ClockSampler(0)
-    l0 = eng.launch_count + mg.launch_count
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record(compute)
-    if graph is not None:
-        for _ in range(args.steps // 2):
-            graph.replay()
-    else:
-        for _ in range(args.steps):
-            one_round()
-    ev1.record(compute)
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    mg.check()
-    ms = ev0.elapsed_time(ev1)
-    launches = per_replay * (args.steps // 2) if graph is not None else eng.launch_count + mg.launch_count - l0
-    if graph is not None:
-        eng.sync()
-        eng.set_stream(compute)
-    final_loss = float(loss.mean().item())
-
-    # end to end: minibatches and labels start in pinned host memory, the loss comes back every step.  The upload
-    # of step t + 1 (copy stream, two device buffers) runs under the kernels of step t.
-    copy_stream = torch.cuda.Stream()
-    x_buf = [torch.empty_like(xs_d[0]) for _ in range(2)]
-    y_buf = [torch.empty_like(ys_d[0]) for _ in range(2)]
-    ev_up = [torch.cuda.Event() for _ in range(2)]
-    ev_used = [torch.cuda.Event() for _ in range(2)]
-    loss_h = torch.empty(K, dtype=torch.float32, pin_memory=True)
-    n_e2e = max(1, min(args.steps, 50))
-    up_no = [0]
-
-    def upload():
-        slot, i = up_no[0] % 2, up_no[0] % ring_n
-        with torch.cuda.stream(copy_stream):
-            if up_no[0] >= 2:
-                copy_stream.wait_event(ev_used[slot])          # the kernels that read this buffer are done
-            x_buf[slot].copy_(xs_h[i], non_blocking=True)
-            y_buf[slot].copy_(ys_h[i], non_blocking=True)
-            ev_up[slot].record(copy_stream)
-        up_no[0] += 1
-
-    torch.cuda.synchronize()
-    upload()
-    host_step = [0]
-
-    def one_round_host():
-        eng.comm_begin(side)
-        for _ in range(k):
-            slot = host_step[0] % 2
-            upload()                                           # next step's inputs
-            compute.wait_event(ev_up[slot])
-            if args.fused:
-                mg.grad_step(eng, x_buf[slot], y_buf[slot], loss)
-            else:
-                mg.grad(shadow, x_buf[slot], y_buf[slot], grads, loss)
-                eng.local_step(grads)
-            ev_used[slot].record(compute)
-            loss_h.copy_(loss, non_blocking=True)
-            host_step[0] += 1
-        eng.comm_end()
-
-    for _ in range(2):
-        one_round_host()
-    torch.cuda.synchronize()
-    ev0.record(compute)
-    for _ in range(n_e2e):
-        one_round_host()
-    ev1.record(compute)
-    torch.cuda.synchronize()
-    ms_e2e = ev0.elapsed_time(ev1)
-    peaks = {}
-    try:
-        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
-    except OSError:
-        pass
+    grads = torch.empty((K, P), dtype=torch.float32, device="cuda")
     flops_step = K * 2 * B * (2 * dims[0] * dims[1] + 3 * dims[1] * dims[2] + 3 * dims[2] * dims[3])
-    # roofline of the dominant kernel (the HBM-bound local step with bf16 shadow: 22 B per worker-parameter);
-    # this workload is launch-latency-bound, so the per-kernel events are taken in a short pass of their own
-    roofline = None
-    by = {}
-    if not args.fused:
-        eng.set_option(E.OPT_PROFILE, 1)
-        eng.profile_reset()
-        for _ in range(min(args.steps, 50)):
-            one_round()
-        by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
-        eng.set_option(E.OPT_PROFILE, 0)
-    if by.get("local_step"):
-        iv = by["local_step"]
-        avg_ms = sum(b - a for a, b in iv) / len(iv)
-        hbm_peak = float(peaks.get("hbm_gbs", 6650.0))
-        gbs = 22.0 * K * P / (avg_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "local_step (with bf16 shadow)", "achieved": round(gbs, 1), "peak": hbm_peak,
-                    "unit": "GB/s", "frac": round(gbs / hbm_peak, 4), "traffic": None,
-                    "peak_kind": "measured" if "hbm_gbs" in peaks else "fallback",
-                    "algorithmic_bytes_per_launch": 22 * K * P, "avg_launch_ms": round(avg_ms, 5),
-                    "measured_in": "separate pass with per-kernel events"}
-    # the oracle beside it: one local step of two workers (numpy fp64 gradient + C update)
-    cpu_baseline = None
-    if not args.no_cpu_baseline:
-        from oracle import mlp_oracle as MO
-        from oracle.cocod_oracle import OracleEngine
-        nw = 2
-        oe = OracleEngine(nw, P_raw, lr, mu, wd, mode="ref")
-        oe.set_params(x0[:P_raw])
-        Xo = [I.mlp_batch(w, 0) for w in range(nw)]
-        yo = [I.mlp_teacher_labels(Xo[w], teacher) for w in range(nw)]
-        t0 = time.perf_counter()
-        n_cpu = 0
-        while time.perf_counter() - t0 < 10.0:
-            g = np.stack([MO.loss_and_grad(oe.x[w], Xo[w], yo[w], dims, emulate_bf16=True)[1] for w in range(nw)])
-            oe.local_step(g)
-            n_cpu += 1
-        dt = time.perf_counter() - t0
-        cpu_baseline = {"value": nw * P_raw * n_cpu / dt, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
-                        "sample": f"{n_cpu} local steps of {nw} workers (numpy fp64 gradient with bf16 rounding points + "
-                                  f"reference-mode update), no averaging rounds"}
-    print(json.dumps({
-        "metric": METRIC, "value": K * P_raw * k * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
-        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 contractions / f32 state",
-        "data": "synthetic",
+    n_w12 = dims[1] * dims[0] + dims[2] * dims[1]                 # parameters the persistent kernel updates
+
+    def run_variant(name):
+        fused, graphed = name != "two-call", name == "fused+graph"
+        eng = E.Engine(K, P, lr, mu, wd)
+        eng.set_option(E.OPT_BF16_SHADOW, 1)
+        eng.set_params(x0)
+        shadow = eng.bf16_shadow()
+        n_rec = (warm + repeats * steps) * k
+        loss_all = torch.zeros((n_rec, K), dtype=torch.float32, device="cuda")
+        step_no = [0]
+        snaps = []
+
+        def one_round(xs, ys, first, record_at=None):
+            eng.comm_begin(side)
+            for j in range(k):
+                out = loss_all[record_at + j] if (record_at is not None and record_at + k <= n_rec) else loss_all[0]
+                if fused:
+                    mg.grad_step(eng, xs[first + j], ys[first + j], out)
+                else:
+                    mg.grad(shadow, xs[first + j], ys[first + j], grads, out)
+                    eng.local_step(grads)
+            eng.comm_end()
+
+        def eager_round():
+            i = step_no[0]
+            one_round(pool_x, pool_y, i % pool_n, record_at=i)
+            step_no[0] += k
+
+        for r in range(warm):
+            eager_round()
+            if name == "two-call" and r < n_cpu_rounds:
+                snaps.append(shadow.clone())
+        torch.cuda.synchronize()
+        graph = None
+        if graphed:
+            # the captured rounds read their minibatches from a fixed staging area that is refilled (two device
+            # copies, inside the timed region) before every replay
+            stage_x = torch.empty((2 * k,) + tuple(pool_x.shape[1:]), dtype=pool_x.dtype, device="cuda")
+            stage_y = torch.empty((2 * k,) + tuple(pool_y.shape[1:]), dtype=pool_y.dtype, device="cuda")
+            cap = torch.cuda.Stream()
+            eng.sync()
+            eng.set_stream(cap)
+            lb = eng.launch_count + mg.launch_count
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=cap):
+                one_round(stage_x, stage_y, 0)
+                one_round(stage_x, stage_y, k)
+            per_replay = eng.launch_count + mg.launch_count - lb
+
+            def replay():
+                i = step_no[0] % pool_n
+                stage_x.copy_(pool_x[i:i + 2 * k], non_blocking=True)
+                stage_y.copy_(pool_y[i:i + 2 * k], non_blocking=True)
+                graph.replay()
+                step_no[0] += 2 * k
+
+            for _ in range(2):
+                replay()
+            torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        block_ms, launches = [], 0
+        for rep in range(repeats):
+            torch.cuda.synchronize()
+            l0 = eng.launch_count + mg.launch_count
+            ev0.record(compute)
+            if graph is not None:
+                for _ in range(steps // 2):
+                    replay()
+            else:
+                for _ in range(steps):
+                    eager_round()
+            ev1.record(compute)
+            torch.cuda.synchronize()
+            block_ms.append(ev0.elapsed_time(ev1))
+            launches = per_replay * (steps // 2) if graph is not None else eng.launch_count + mg.launch_count - l0
+        mg.check()
+        if graph is not None:
+            eng.sync()
+            eng.set_stream(compute)
+        ms = median(block_ms)
+        out = {"value": K * P_raw * k * steps / (ms * 1e-3), "ms_per_step": ms / steps, "ms_per_local_step": ms / (k * steps),
+               "local_steps_per_s": k * steps / (ms * 1e-3), "gpu_launches": launches,
+               "timed_blocks": {"repeats": repeats, "rounds_per_block": steps, "ms_per_step": [b_ / steps for b_ in block_ms],
+                                "ms_per_step_min": min(block_ms) / steps, "ms_per_step_max": max(block_ms) / steps,
+                                "reported": "median block"},
+               "tensor_tflops": flops_step * k * steps / (ms * 1e-3) / 1e12}
+        # ---- per-kernel pass of its own (events break the programmatic launch edges, so never inside the timed blocks)
+        if not graphed:
+            n_prof = min(steps, 25)
+            mg.set_profile(True)
+            eng.set_option(E.OPT_PROFILE, 1)
+            eng.profile_reset()
+            for _ in range(n_prof):
+                eager_round()
+            calls, pass_ms, upd_ms = mg.profile()
+            by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+            eng.set_option(E.OPT_PROFILE, 0)
+            mg.set_profile(False)
+            if fused:
+                alg = 18 * K * n_w12
+                gbs = alg / (upd_ms * 1e-3) / 1e9 if upd_ms > 0 else None
+                out["roofline"] = {"bound": "hbm", "kernel": "gemm_update_persistent (weight gradients of W1, W2 + their momentum update)",
+                                   "achieved": round(gbs, 1) if gbs else None, "peak": hbm_peak, "unit": "GB/s",
+                                   "frac": round(gbs / hbm_peak, 4) if gbs else None, "traffic": None, "peak_kind": peak_kind,
+                                   "algorithmic_bytes_per_launch": alg, "avg_launch_ms": round(upd_ms, 5),
+                                   "bytes_per_parameter": 18,
+                                   "measured_in": "a pass of its own with CUDA events around the kernel"}
+                out["gradient_pass_ms"] = {"whole_call": round(pass_ms, 5), "update_kernel": round(upd_ms, 5),
+                                           "everything_else": round(pass_ms - upd_ms, 5), "calls": calls}
+            else:
+                iv = by.get("local_step", [])
+                avg_ms = sum(b_ - a_ for a_, b_ in iv) / max(1, len(iv))
+                gbs = 22.0 * K * P / (avg_ms * 1e-3) / 1e9 if iv else None
+                out["roofline"] = {"bound": "hbm", "kernel": "local_step (with bf16 shadow)", "achieved": round(gbs, 1) if gbs else None,
+                                   "peak": hbm_peak, "unit": "GB/s", "frac": round(gbs / hbm_peak, 4) if gbs else None,
+                                   "traffic": None, "peak_kind": peak_kind, "algorithmic_bytes_per_launch": 22 * K * P,
+                                   "avg_launch_ms": round(avg_ms, 5), "bytes_per_parameter": 22,
+                                   "measured_in": "a pass of its own with per-kernel CUDA events"}
+                out["gradient_pass_ms"] = {"whole_call": round(pass_ms, 5), "calls": calls}
+        torch.cuda.synchronize()
+        n_done = min(step_no[0], n_rec) if not graphed else warm * k
+        curve = loss_all[:n_done].double().mean(dim=1).cpu().numpy()
+        out["loss_first_steps"] = [round(float(v), 5) for v in curve[:4 * k]]
+        out["loss_last"] = round(float(curve[-1]), 5) if not graphed else None
+        return out, eng, curve, snaps
+
+    variants = {}
+    curve2, snaps2 = None, None
+    sampler = ClockSampler(0)
+    names = ["two-call", "fused", "fused+graph"]
+    engines = {}
+    for name in names:
+        variants[name], engines[name], curve, snaps = run_variant(name)
+        if name == "two-call":
+            curve2, snaps2 = curve, snaps
+        if name != "fused" or digest:
+            engines.pop(name).destroy()
+    clocks = sampler.stop()
+
+    # ---- end to end (stand-alone run only): minibatches and labels start in pinned host memory, the loss comes back every
+    #      step; the upload of step t + 1 (copy stream, two device buffers) runs under the kernels of step t
+    e2e = None
+    if not digest and not args.no_e2e:
+        eng = engines.pop("fused")
+        ring_n = min(pool_n, 256)
+        xs_h = pool_x[:ring_n].cpu().pin_memory()
+        ys_h = pool_y[:ring_n].cpu().pin_memory()
+        copy_stream = torch.cuda.Stream()
+        x_buf = [torch.empty_like(pool_x[0]) for _ in range(2)]
+        y_buf = [torch.empty_like(pool_y[0]) for _ in range(2)]
+        ev_up = [torch.cuda.Event() for _ in range(2)]
+        ev_used = [torch.cuda.Event() for _ in range(2)]
+        loss = torch.empty(K, dtype=torch.float32, device="cuda")
+        loss_h = torch.empty(K, dtype=torch.float32, pin_memory=True)
+        n_e2e = max(1, min(steps, 50))
+        up_no, host_step = [0], [0]
+
+        def upload():
+            slot, i = up_no[0] % 2, up_no[0] % ring_n
+            with torch.cuda.stream(copy_stream):
+                if up_no[0] >= 2:
+                    copy_stream.wait_event(ev_used[slot])          # the kernels that read this buffer are done
+                x_buf[slot].copy_(xs_h[i], non_blocking=True)
+                y_buf[slot].copy_(ys_h[i], non_blocking=True)
+                ev_up[slot].record(copy_stream)
+            up_no[0] += 1
+
+        def one_round_host():
+            eng.comm_begin(side)
+            for _ in range(k):
+                slot = host_step[0] % 2
+                upload()                                           # next step's inputs
+                compute.wait_event(ev_up[slot])
+                mg.grad_step(eng, x_buf[slot], y_buf[slot], loss)
+                ev_used[slot].record(compute)
+                loss_h.copy_(loss, non_blocking=True)
+                host_step[0] += 1
+            eng.comm_end()
+
+        torch.cuda.synchronize()
+        upload()
+        for _ in range(2):
+            one_round_host()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(compute)
+        for _ in range(n_e2e):
+            one_round_host()
+        ev1.record(compute)
+        torch.cuda.synchronize()
+        ms_e2e = ev0.elapsed_time(ev1)
+        e2e = {"value": K * P_raw * k * n_e2e / (ms_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": k * (xs_h[0].numel() * 2 + ys_h[0].numel() * 4), "d2h_bytes_per_step": k * K * 4,
+               "rounds": n_e2e, "ms_per_step": ms_e2e / n_e2e, "path": "fused gradient + update call"}
+        eng.destroy()
+    for e_ in engines.values():
+        e_.destroy()
+
+    # ---- the oracle beside it: the first rounds of the SAME run (same minibatch and label bytes), all K workers, one
+    #      process per worker on the host's cores; gives the paired loss curve and the per-round parameter distance
+    cpu_baseline, paired = None, None
+    if n_cpu_rounds > 0:
+        procs = max(1, min(K, os.cpu_count() or 1))
+        nst = n_cpu_rounds * k
+        Xb = pool_x[:nst].view(torch.int16).cpu().numpy().view(np.uint16)
+        yb = pool_y[:nst].cpu().numpy()
+        dt, o_losses, o_params = time_mlp_oracle(K, k, n_cpu_rounds, lr, mu, wd, x0[:P_raw], Xb, yb, procs)
+        cpu_baseline = {"value": K * P_raw * k * n_cpu_rounds / dt, "unit": UNIT, "cores": procs, "kind": "oracle",
+                        "sample": f"the first {n_cpu_rounds} rounds (k={k}) of the same run, all {K} workers: numpy fp64 gradient "
+                                  f"with the bf16 rounding points (one process per worker) + reference-mode parameter path"}
+        worst, first_break = [], None
+        for r in range(n_cpu_rounds):
+            got = snaps2[r].float().cpu().numpy()[:, :P_raw]
+            want = o_params[r]
+            scale = np.maximum(np.abs(want), np.sqrt(np.mean(want.astype(np.float64) ** 2)))
+            e_ = float((np.abs(got - want) / scale).max())
+            worst.append(round(e_, 5))
+            if e_ > 1e-2 and first_break is None:
+                first_break = r + 1
+        paired = {"steps": nst, "gpu": [round(float(v), 5) for v in curve2[:nst]], "oracle": [round(v, 5) for v in o_losses],
+                  "max_relative_gap": float(max(abs(a_ - b_) / abs(b_) for a_, b_ in zip(curve2[:nst], o_losses))),
+                  "bf16_parameters_max_scaled_error_per_round_free_running": worst,
+                  "first_round_outside_1e-2": first_break,
+                  "note": "free-running device run against the canonical oracle; the per-round parity run with the "
+                          "restarted engines over all 200 rounds is tests/c4_loss_curve.py"}
+    head = "fused+graph" if (args.fused and args.graph) else "fused" if args.fused else "fused+graph" if args.graph else "two-call"
+    if digest:
+        head = "fused"
+    hv = variants[head]
+    res = {
+        "metric": METRIC, "value": hv["value"], "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warm,
+        "ms_per_step": hv["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 contractions / f32 state", "data": "synthetic",
         "config": {"workload": "mlp", "K": K, "P": P_raw, "P_padded": P, "k": k, "lr": lr, "mu": mu, "wd": wd,
-                   "mlp": list(dims), "batch": B, "minibatch_ring": ring_n, "cuda_graph": bool(args.graph),
-                   "fused_update": bool(args.fused)},
-        "clocks": clocks, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_baseline,
-        "local_steps_per_s": k * args.steps / (ms * 1e-3), "ms_per_local_step": ms / (k * args.steps),
-        "tensor_tflops": flops_step * k * args.steps / (ms * 1e-3) / 1e12,
-        "tensor_peak_tflops": peaks.get("bf16_tflops"),
-        "e2e": {"value": K * P_raw * k * n_e2e / (ms_e2e * 1e-3), "unit": UNIT,
-                "h2d_bytes_per_step": k * (xs_h[0].numel() * 2 + ys_h[0].numel() * 4), "d2h_bytes_per_step": k * K * 4,
-                "rounds": n_e2e, "ms_per_step": ms_e2e / n_e2e},
-        "loss_first_steps": [round(float(l.mean().item()), 4) for l in losses[:8]], "loss_last": round(final_loss, 4),
-    }))
-    eng.destroy()
+                   "mlp": list(dims), "batch": B, "minibatch_pool_steps": pool_n,
+                   "minibatches": "one per (worker, global step), seeded; the pool repeats after minibatch_pool_steps steps",
+                   "headline_variant": head,
+                   "l2": "the K x P state is 119 MB fp32 + 119 MB momentum + 60 MB bf16 copy: larger than the 126 MB L2"},
+        "clocks": clocks, "gpu_launches": hv["gpu_launches"], "roofline": hv.get("roofline") or variants["fused"].get("roofline"),
+        "cpu_baseline": cpu_baseline, "variants": variants, "loss_curve_vs_oracle": paired,
+        "local_steps_per_s": hv["local_steps_per_s"], "ms_per_local_step": hv["ms_per_local_step"],
+        "tensor_peak_tflops": peaks.get("bf16_tflops"), "e2e": e2e,
+    }
     mg.destroy()
+    del pool_x, pool_y, grads
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_mlp(args):
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the engine has no CPU fallback")
+    torch.cuda.set_device(0)
+    print(json.dumps(measure_mlp(args, digest=False)))
 
 
 # ---------------------------------------------------------------------------------------------- workers over GPUs

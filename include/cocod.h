@@ -54,7 +54,8 @@ enum {
      * copy and the first local step of the round writes x into the spare buffer (0 B); the
      * values are identical. */
     COCOD_OPT_SNAPSHOT = 1,
-    /* Record CUDA events around every kernel (cocod_profile_*). 0 = off (default). */
+    /* Record CUDA events around every kernel and let the kernels stamp their own start and end on the GPU's
+     * clock (cocod_profile_*). 0 = off (default).  Switching it on the first time allocates 256 KB on the device. */
     COCOD_OPT_PROFILE = 2,
     /* Keep a bfloat16 copy of x (K x P, same layout) current: the local-step and merge kernels
      * write bf16(x) next to x (22 B and 14 B + 4/K per worker-parameter instead of 20 and
@@ -178,6 +179,14 @@ const char *cocod_strerror(int code);
 int cocod_profile_reset(cocod_handle *h);
 int cocod_profile_count(cocod_handle *h);
 int cocod_profile_get(cocod_handle *h, int i, int *kind, float *start_ms, float *end_ms);
+
+/* The same record's lifetime as the kernel itself saw it: the earliest start and the latest end of its
+ * thread blocks in nanoseconds of the GPU's own clock (one clock for all streams, so the lifetimes of the
+ * mean kernel on the side stream and of the local steps on the compute stream can be intersected exactly:
+ * the overlap Algorithm 1 asks for between Step I and Step II).  Valid after cocod_profile_count (STATE
+ * before it).  Both are 0 for a record whose kernel takes no stamps (the scalar fall-back kernels, the
+ * stored-copy kernel, the gather kernel). */
+int cocod_profile_get_device_ns(cocod_handle *h, int i, uint64_t *start_ns, uint64_t *end_ns);
 
 /* Number of kernels this handle has launched since creation (all kinds). */
 int64_t cocod_launch_count(const cocod_handle *h);

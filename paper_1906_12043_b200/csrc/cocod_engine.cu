@@ -38,6 +38,10 @@ struct ProfileRec {
     cudaEvent_t a, b;
 };
 
+// Where the kernel launched inside the current profiling bracket leaves its device-side time stamps
+// (nullptr outside a bracket, for the stateless entry points, and while profiling is off).
+thread_local unsigned long long *g_stamp = nullptr;
+
 }  // namespace
 
 struct cocod_engine {
@@ -78,6 +82,8 @@ struct cocod_engine {
     int cuda_error = 0;
     bool profile = false;
     std::vector<ProfileRec> prof;
+    unsigned long long *stamps = nullptr;       // device: kMaxProfile x {earliest start, latest end} in ns of the GPU's clock
+    std::vector<unsigned long long> stamps_host; // copy taken by cocod_profile_count
 };
 
 namespace {
@@ -113,11 +119,11 @@ cudaError_t launch_local_step(const float *x_in, float *x_out, float *v, const f
         if (shadow != nullptr)
             local_step_vec4<THREADS, UNROLL, true><<<grid, THREADS, 0, s>>>(
                 reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
-                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, shadow);
+                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, shadow, g_stamp);
         else
             local_step_vec4<THREADS, UNROLL, false><<<grid, THREADS, 0, s>>>(
                 reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
-                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, nullptr);
+                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, nullptr, g_stamp);
         done = nvec * 4;
         if (n_launch) ++*n_launch;
     }
@@ -159,12 +165,12 @@ cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, flo
     using namespace cocod;
     if (K <= 4 && (P % 8) == 0 && aligned32(snap) && aligned32(mean)) {
         const unsigned grid = grid_for(P / 8, kThreads);
-        if (K <= 2) mean_vec8<2><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
-        else mean_vec8<4><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
+        if (K <= 2) mean_vec8<2><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k, g_stamp);
+        else mean_vec8<4><<<grid, kThreads, 0, s>>>(snap, K, P, w, mean, inv_k, g_stamp);
     } else if ((P % 4) == 0 && aligned16(snap) && aligned16(mean)) {
         const int64_t pvec = P / 4;
         mean_vec4<<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
-            reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k);
+            reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k, g_stamp);
     } else {
         mean_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
     }
@@ -204,16 +210,16 @@ cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, 
         (shadow == nullptr || aligned16(shadow))) {
         // rows per thread: as many as K allows up to 8 (registers scale with it)
         const unsigned gx = grid_for(P / 8, kThreads);
-        if (K >= 8) merge_vec8<8><<<dim3(gx, (unsigned)((K + 7) / 8)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
-        else if (K >= 4) merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
-        else if (K >= 2) merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
-        else merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
+        if (K >= 8) merge_vec8<8><<<dim3(gx, (unsigned)((K + 7) / 8)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
+        else if (K >= 4) merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
+        else if (K >= 2) merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
+        else merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
     } else if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean) &&
                (shadow == nullptr || (reinterpret_cast<uintptr_t>(shadow) & 7u) == 0)) {
         const int64_t pvec = P / 4;
         merge_vec4<4><<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
             reinterpret_cast<float4 *>(x), reinterpret_cast<const float4 *>(snap),
-            reinterpret_cast<const float4 *>(mean), K, pvec, shadow);
+            reinterpret_cast<const float4 *>(mean), K, pvec, shadow, g_stamp);
     } else {
         merge_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(x, snap, mean, K, P, shadow);
     }
@@ -234,15 +240,26 @@ struct Bracket {
         if (cudaEventCreate(&a) != cudaSuccess) { a = nullptr; return; }
         if (cudaEventCreate(&b) != cudaSuccess) { cudaEventDestroy(a); a = b = nullptr; return; }
         on = true;
+        if (h->stamps) g_stamp = h->stamps + 2 * h->prof.size();      // this record's slot
         cudaEventRecord(a, s);
     }
     ~Bracket()
     {
+        g_stamp = nullptr;
         if (!on) return;
         cudaEventRecord(b, s);
         h->prof.push_back({kind, a, b});
     }
 };
+
+// start = all ones (atomicMin), end = 0 (atomicMax); the engine is idle when this is called
+cudaError_t stamps_reset(cocod_engine *h)
+{
+    if (!h->stamps) return cudaSuccess;
+    std::vector<unsigned long long> init(2 * (size_t)kMaxProfile);
+    for (size_t i = 0; i < init.size(); i += 2) { init[i] = ~0ull; init[i + 1] = 0ull; }
+    return cudaMemcpy(h->stamps, init.data(), init.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice);
+}
 
 void profile_clear(cocod_engine *h)
 {
@@ -251,6 +268,8 @@ void profile_clear(cocod_engine *h)
         cudaEventDestroy(r.b);
     }
     h->prof.clear();
+    h->stamps_host.clear();
+    stamps_reset(h);
 }
 
 int check_live(const cocod_engine *h)
@@ -287,6 +306,7 @@ void detach_peers(cocod_engine *h)
 void free_all(cocod_engine *h)
 {
     profile_clear(h);
+    if (h->stamps) { cudaFree(h->stamps); h->stamps = nullptr; }
     detach_peers(h);
     if (h->wg) cudaFree(h->wg);
     for (int i = 0; i < 2; ++i) if (h->buf[i]) cudaFree(h->buf[i]);
@@ -727,6 +747,15 @@ int cocod_set_option(cocod_handle *h, int option, int value)
         h->snapshot_mode = value;
         return COCOD_OK;
     case COCOD_OPT_PROFILE:
+        if (value && !h->stamps) {      // device-side time stamps: 256 KB, kept until the handle is destroyed
+            if (cudaMalloc((void **)&h->stamps, 2 * (size_t)kMaxProfile * sizeof(unsigned long long)) != cudaSuccess) {
+                cudaGetLastError();
+                h->stamps = nullptr;
+                return COCOD_ERR_OOM;
+            }
+            CK(h, cudaDeviceSynchronize());
+            CK(h, stamps_reset(h));
+        }
         h->profile = value != 0;
         return COCOD_OK;
     case COCOD_OPT_BF16_SHADOW:
@@ -814,7 +843,24 @@ int cocod_profile_count(cocod_handle *h)
 {
     if (int rc = check_live(h)) return rc;
     if (int rc = cocod_sync(h)) return rc;
+    if (h->stamps && !h->prof.empty()) {
+        h->stamps_host.resize(2 * h->prof.size());
+        CK(h, cudaMemcpy(h->stamps_host.data(), h->stamps, h->stamps_host.size() * sizeof(unsigned long long),
+                         cudaMemcpyDeviceToHost));
+    }
     return (int)h->prof.size();
+}
+
+int cocod_profile_get_device_ns(cocod_handle *h, int i, uint64_t *start_ns, uint64_t *end_ns)
+{
+    if (int rc = check_live(h)) return rc;
+    if (i < 0 || i >= (int)h->prof.size() || !start_ns || !end_ns) return COCOD_ERR_INVALID;
+    if (2 * (size_t)i + 1 >= h->stamps_host.size()) return COCOD_ERR_STATE;      // cocod_profile_count first
+    const unsigned long long a = h->stamps_host[2 * i], b = h->stamps_host[2 * i + 1];
+    const bool have = (a != ~0ull) && (b != 0ull);
+    *start_ns = have ? (uint64_t)a : 0;
+    *end_ns = have ? (uint64_t)b : 0;
+    return COCOD_OK;
 }
 
 int cocod_profile_get(cocod_handle *h, int i, int *kind, float *start_ms, float *end_ms)

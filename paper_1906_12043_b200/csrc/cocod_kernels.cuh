@@ -78,6 +78,32 @@ __device__ __forceinline__ void sgd_update(float4 &x, float4 &v, const float4 &g
     d = __fmaf_rn(wd, x.w, g.w); v.w = __fmaf_rn(mu, v.w, d); x.w = __fmaf_rn(-lr, v.w, x.w);
 }
 
+// ------------------------------------------------------------------------------------------ device-side time stamps
+// Profiling only (stamp == nullptr otherwise): stamp[0] = earliest start, stamp[1] = latest end of the kernel's CTAs
+// on the GPU's own nanosecond clock, which all streams share -- so the lifetimes of kernels on different streams can
+// be intersected.  Only the first and the last 2048 CTAs of a grid take part (they contain the first CTA to start
+// and the last to finish), which keeps the same-address atomics to a few thousand per launch.
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void stamp_begin(unsigned long long *stamp)
+{
+    if (stamp != nullptr && threadIdx.x == 0) {
+        const unsigned long long lin = (unsigned long long)blockIdx.y * gridDim.x + blockIdx.x;
+        if (lin < 2048ull) atomicMin(stamp, global_ns());
+    }
+}
+__device__ __forceinline__ void stamp_end(unsigned long long *stamp)
+{
+    if (stamp != nullptr && threadIdx.x == 0) {
+        const unsigned long long lin = (unsigned long long)blockIdx.y * gridDim.x + blockIdx.x;
+        if (lin + 2048ull >= (unsigned long long)gridDim.x * gridDim.y) atomicMax(stamp + 1, global_ns());
+    }
+}
+
 // ------------------------------------------------------------------------------------------ local step (Step II)
 // One CTA owns a contiguous tile of THREADS * UNROLL float4 of the flat K*P vector: all
 // 3 * UNROLL loads of a thread are issued before the first use.  x_in may equal x_out.
@@ -88,8 +114,10 @@ __device__ __forceinline__ void sgd_update(float4 &x, float4 &v, const float4 &g
 template <int THREADS, int UNROLL, bool SHADOW>
 __global__ void __launch_bounds__(THREADS)
 local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__restrict__ g,
-                int64_t nvec, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow)
+                int64_t nvec, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow,
+                unsigned long long *stamp)
 {
+    stamp_begin(stamp);
     const int64_t base = (int64_t)blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
     float4 xr[UNROLL], vr[UNROLL], gr[UNROLL];
     if (base + (int64_t)(UNROLL - 1) * THREADS < nvec) {       // full tile: no predicates
@@ -121,6 +149,7 @@ local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__re
             }
         }
     }
+    stamp_end(stamp);
 }
 
 // Scalar path: misaligned pointers and the n mod 4 tail.  Elements [first, first + count).
@@ -236,8 +265,9 @@ __device__ __forceinline__ void mean_rows(float (&s)[NV], int K, const float *__
 // One thread owns one float4 of columns.  Needs P mod 4 == 0 and 16-byte aligned bases.
 static __global__ void __launch_bounds__(kThreads)
 mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__restrict__ w,
-          float4 *__restrict__ mean, float inv_k)
+          float4 *__restrict__ mean, float inv_k, unsigned long long *stamp)
 {
+    stamp_begin(stamp);
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (c >= pvec) return;
     const float4 *col = snap + c;
@@ -247,6 +277,7 @@ mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__r
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
     });
     mean[c] = make_float4(s[0], s[1], s[2], s[3]);
+    stamp_end(stamp);
 }
 
 // Few workers (K <= CAP <= 4): a float4 per row would leave too few bytes in flight per thread, so
@@ -254,8 +285,9 @@ mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__r
 template <int CAP>
 __global__ void __launch_bounds__(kThreads)
 mean_vec8(const float *__restrict__ snap, int K, int64_t P, const float *__restrict__ w,
-          float *__restrict__ mean, float inv_k)
+          float *__restrict__ mean, float inv_k, unsigned long long *stamp)
 {
+    stamp_begin(stamp);
     const int64_t c = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 8;
     if (c >= P) return;
     float s[8];
@@ -268,6 +300,7 @@ mean_vec8(const float *__restrict__ snap, int K, int64_t P, const float *__restr
 #pragma unroll
     for (int q = 0; q < 8; ++q) o.a[q] = s[q];
     st256(mean + c, o);
+    stamp_end(stamp);
 }
 
 // Any P / alignment: one thread per column.
@@ -349,8 +382,9 @@ mean_gather_scalar(const float *const *__restrict__ rows, int K, int64_t p_lo, i
 template <int RC>
 __global__ void __launch_bounds__(kThreads)
 merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K, int64_t pvec,
-           __nv_bfloat16 *__restrict__ shadow)
+           __nv_bfloat16 *__restrict__ shadow, unsigned long long *stamp)
 {
+    stamp_begin(stamp);
     const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
     if (c >= pvec) return;
     const float4 m = mean[c];
@@ -376,6 +410,7 @@ merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K
                 if (shadow != nullptr) st_shadow4(shadow + 4 * e, o);
             }
     }
+    stamp_end(stamp);
 }
 
 // Widest path (P mod 8 == 0, 32-byte aligned bases): one thread owns 8 columns (256-bit accesses,
@@ -385,8 +420,9 @@ merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K
 template <int RC>
 __global__ void __launch_bounds__(kThreads)
 merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P,
-           __nv_bfloat16 *__restrict__ shadow)
+           __nv_bfloat16 *__restrict__ shadow, unsigned long long *stamp)
 {
+    stamp_begin(stamp);
     const int64_t c = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 8;
     if (c >= P) return;
     const f32x8 m = ld256(mean + c);
@@ -412,6 +448,7 @@ merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, i
                     make_uint4(pack_bf16x2(o.a[0], o.a[1]), pack_bf16x2(o.a[2], o.a[3]),
                                pack_bf16x2(o.a[4], o.a[5]), pack_bf16x2(o.a[6], o.a[7]));
         }
+    stamp_end(stamp);
 }
 
 static __global__ void __launch_bounds__(kThreads)

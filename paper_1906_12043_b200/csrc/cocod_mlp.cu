@@ -21,6 +21,8 @@
 #include <algorithm>
 #include <cstdio>
 #include <new>
+#include <utility>
+#include <vector>
 
 namespace {
 
@@ -396,12 +398,39 @@ struct cocod_mlp {
     // joined to the caller's stream by events
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    // COCOD_MLP_OPT_PROFILE: CUDA events around every gradient pass and around its gradient + update kernel
+    bool profile = false;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_pass, prof_update;
 };
 
 namespace {
 
+void mlp_profile_clear(cocod_mlp *h)
+{
+    for (auto *list : {&h->prof_pass, &h->prof_update}) {
+        for (auto &pr : *list) {
+            cudaEventDestroy(pr.first);
+            cudaEventDestroy(pr.second);
+        }
+        list->clear();
+    }
+}
+
+// An event pair whose first event is recorded now; the caller records the second one.
+bool mlp_profile_open(cocod_mlp *h, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> &list, cudaStream_t s)
+{
+    if (!h->profile || list.size() >= 4096) return false;
+    cudaEvent_t a = nullptr, b = nullptr;
+    if (cudaEventCreate(&a) != cudaSuccess) { cudaGetLastError(); return false; }
+    if (cudaEventCreate(&b) != cudaSuccess) { cudaGetLastError(); cudaEventDestroy(a); return false; }
+    cudaEventRecord(a, s);
+    list.emplace_back(a, b);
+    return true;
+}
+
 void mlp_free(cocod_mlp *h)
 {
+    mlp_profile_clear(h);
     void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
@@ -524,6 +553,8 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     if (cudaStreamIsCapturing(s, &capturing) != cudaSuccess) return COCOD_ERR_CUDA;
     const bool pdl = (capturing == cudaStreamCaptureStatusNone);
     const bool pdl_fwd = true;
+    // profiling (never while capturing): events around the whole pass and around the gradient + update kernel
+    const bool prof_pass = (capturing == cudaStreamCaptureStatusNone) && mlp_profile_open(h, h->prof_pass, s);
     // fused call: the small tensors (biases, W3, padding) take their local step inside the kernels that produce
     // their gradients; otherwise those kernels write the gradients out
     StepTarget small{};
@@ -586,7 +617,9 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
             u1.tiles = K * u1.tiles_m * u1.tiles_n;
             UpdateParams uq{};
             uq.K = B; uq.lr = fused->lr; uq.mu = fused->mu; uq.wd = fused->wd; uq.error_flag = h->error_flag;
-            GEMM_OK(launch_update(u2, u1, uq, s, pdl));
+            const bool prof_upd = (capturing == cudaStreamCaptureStatusNone) && mlp_profile_open(h, h->prof_update, s);
+            GEMM_OK(launch_update(u2, u1, uq, s, pdl && !prof_upd));
+            if (prof_upd) cudaEventRecord(h->prof_update.back().second, s);
         }
     } else if (fork) {
         // dW2 needs only dz2 and h1: it runs beside dz1 -> dW1.  dz1 is queued first and keeps a ring of three
@@ -610,6 +643,7 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     }
 #undef LAUNCH_OK
 #undef GEMM_OK
+    if (prof_pass) cudaEventRecord(h->prof_pass.back().second, s);
     return COCOD_OK;
 }
 
@@ -659,6 +693,35 @@ int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x
     if (int rc = run_grad(h, plan.shadow, static_cast<const bf16 *>(x), labels, nullptr, loss, plan.compute, &plan))
         return rc;
     return cocod_internal_finish_step(engine, 0);
+}
+
+int cocod_mlp_set_option(cocod_mlp_handle *h, int option, int value)
+{
+    if (!h) return COCOD_ERR_INVALID;
+    if (option != COCOD_MLP_OPT_PROFILE) return COCOD_ERR_INVALID;
+    if (cudaDeviceSynchronize() != cudaSuccess) return COCOD_ERR_CUDA;
+    mlp_profile_clear(h);
+    h->profile = value != 0;
+    return COCOD_OK;
+}
+
+int cocod_mlp_profile_get(cocod_mlp_handle *h, int *calls, float *pass_ms, float *update_ms)
+{
+    if (!h || !calls || !pass_ms || !update_ms) return COCOD_ERR_INVALID;
+    if (cudaDeviceSynchronize() != cudaSuccess) return COCOD_ERR_CUDA;
+    auto average = [](const std::vector<std::pair<cudaEvent_t, cudaEvent_t>> &list, float *out) {
+        double sum = 0.0;
+        for (const auto &pr : list) {
+            float ms = 0.0f;
+            if (cudaEventElapsedTime(&ms, pr.first, pr.second) != cudaSuccess) return false;
+            sum += ms;
+        }
+        *out = list.empty() ? 0.0f : (float)(sum / (double)list.size());
+        return true;
+    };
+    if (!average(h->prof_pass, pass_ms) || !average(h->prof_update, update_ms)) { cudaGetLastError(); return COCOD_ERR_CUDA; }
+    *calls = (int)h->prof_pass.size();
+    return COCOD_OK;
 }
 
 int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream)

@@ -51,6 +51,7 @@ SIGNATURES = {
     "cocod_profile_reset": (_i, [_vp]),
     "cocod_profile_count": (_i, [_vp]),
     "cocod_profile_get": (_i, [_vp, _i, ctypes.POINTER(_i), ctypes.POINTER(_f), ctypes.POINTER(_f)]),
+    "cocod_profile_get_device_ns": (_i, [_vp, _i, ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]),
     "cocod_launch_count": (_i64, [_vp]),
     "cocod_set_shard": (_i, [_vp, _i, _i, ctypes.POINTER(ctypes.c_double)]),
     "cocod_mean_buffer": (_i, [_vp, ctypes.POINTER(_vp)]),
@@ -335,6 +336,27 @@ class Engine:
                      "cocod_profile_get")
             out.append((kind.value, a.value, b.value))
         return out
+
+    def profile_device_records(self):
+        """[(kind, start_ms, end_ms)] of the same records from the kernels' own stamps on the GPU's clock
+        (milliseconds relative to the earliest stamp); records without stamps are left out."""
+        n = self._lib.cocod_profile_count(self._h)
+        if n < 0:
+            self._ck(n, "cocod_profile_count")
+        kind, a, b = _i(), _f(), _f()
+        t0, t1 = ctypes.c_uint64(), ctypes.c_uint64()
+        raw = []
+        for i in range(n):
+            self._ck(self._lib.cocod_profile_get(self._h, i, ctypes.byref(kind), ctypes.byref(a), ctypes.byref(b)),
+                     "cocod_profile_get")
+            self._ck(self._lib.cocod_profile_get_device_ns(self._h, i, ctypes.byref(t0), ctypes.byref(t1)),
+                     "cocod_profile_get_device_ns")
+            if t0.value and t1.value:
+                raw.append((kind.value, t0.value, t1.value))
+        if not raw:
+            return []
+        base = min(r[1] for r in raw)
+        return [(k, (s - base) * 1e-6, (e - base) * 1e-6) for k, s, e in raw]
 
 
 # ---------------------------------------------------------------------------------------------- stateless kernels

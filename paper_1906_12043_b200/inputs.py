@@ -291,3 +291,30 @@ def mlp_teacher_labels(X: np.ndarray, teacher: np.ndarray, dims=MLP_DIMS) -> np.
     h = np.maximum(X.astype(np.float64) @ p["W1"].T + p["b1"], 0.0)
     h = np.maximum(h @ p["W2"].T + p["b2"], 0.0)
     return np.argmax(h @ p["W3"].T + p["b3"], axis=1).astype(np.int32)
+
+
+def device_mlp_batches_into(out, first_step: int, seed: int = MLP_DATA_SEED) -> None:
+    """Fill a CUDA bfloat16 tensor [steps][K][batch][d_in] with the minibatches of global steps
+    first_step .. first_step + steps - 1 (the same bytes as ``mlp_batch`` gives on the host)."""
+    steps, K = out.shape[0], out.shape[1]
+    for t in range(steps):
+        for w in range(K):
+            device_gaussian_into(out[t, w], seed, STREAM_DATA, w, first_step + t, 0, 1.0)
+
+
+def device_mlp_teacher_labels(X, teacher: np.ndarray, dims=MLP_DIMS, rows_per_pass: int = 1 << 16):
+    """Labels of minibatches held on the device: argmax of the teacher MLP's logits in fp64 (torch on the
+    device; the same definition as ``mlp_teacher_labels``).  X: CUDA bfloat16 [..., d_in]; returns int32
+    [...].  Whoever compares two implementations hands BOTH this one array (a near-tie could fall
+    differently under another summation order)."""
+    import torch
+    segs, _ = mlp_segments(dims)
+    p = {name: torch.from_numpy(teacher[off:off + int(np.prod(shape))].astype(np.float64).reshape(shape)).to(X.device)
+         for name, off, shape in segs}
+    flat = X.reshape(-1, X.shape[-1])
+    out = torch.empty(flat.shape[0], dtype=torch.int32, device=X.device)
+    for r0 in range(0, flat.shape[0], rows_per_pass):
+        h = torch.relu(flat[r0:r0 + rows_per_pass].double() @ p["W1"].T + p["b1"])
+        h = torch.relu(h @ p["W2"].T + p["b2"])
+        out[r0:r0 + rows_per_pass] = torch.argmax(h @ p["W3"].T + p["b3"], dim=1).to(torch.int32)
+    return out.reshape(X.shape[:-1])

@@ -19,12 +19,15 @@ SIGNATURES = {
     "cocod_mlp_grad": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "cocod_mlp_grad_step": (_i, [_vp, _vp, _vp, _vp, _vp]),
     "cocod_mlp_check": (_i, [_vp, _vp]),
+    "cocod_mlp_set_option": (_i, [_vp, _i, _i]),
+    "cocod_mlp_profile_get": (_i, [_vp, ctypes.POINTER(_i), ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]),
     "cocod_mlp_launch_count": (_i64, [_vp]),
     "cocod_gemm_wait_selftest": (_i, [_i, _vp]),
     "cocod_gemm_update_wait_selftest": (_i, [_i, _vp]),
     "cocod_gemm_bf16": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i64, _i64, _i64, _vp]),
 }
 
+OPT_PROFILE = 1
 _declared = False
 
 
@@ -94,6 +97,19 @@ class MLPGrad:
         rc = self._lib.cocod_mlp_check(self._h, _cur_stream(stream))
         if rc != _E.OK:
             raise _E.CocodError(rc, "cocod_mlp_check")
+
+    def set_profile(self, on: bool):
+        rc = self._lib.cocod_mlp_set_option(self._h, OPT_PROFILE, int(bool(on)))
+        if rc != _E.OK:
+            raise _E.CocodError(rc, "cocod_mlp_set_option")
+
+    def profile(self):
+        """(recorded calls, average ms of a whole gradient pass, average ms of the gradient + update kernel)."""
+        n, a, b = _i(), ctypes.c_float(), ctypes.c_float()
+        rc = self._lib.cocod_mlp_profile_get(self._h, ctypes.byref(n), ctypes.byref(a), ctypes.byref(b))
+        if rc != _E.OK:
+            raise _E.CocodError(rc, "cocod_mlp_profile_get")
+        return n.value, a.value, b.value
 
     @property
     def launch_count(self) -> int:

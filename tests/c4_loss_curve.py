@@ -19,7 +19,7 @@ ReLU is a decision (z > 0) that floating point takes.  The device accumulates z 
 for the few units per round whose |z| lies within accumulation error of zero the two can decide differently,
 both correctly, and one such decision switches a whole sample's term of a weight-gradient row.  The restarted
 engines are therefore compared with a BRANCH of the oracle that starts every round from the canonical oracle
-state and, for units with |z| < 5e-4 only, takes the decision the device took (match_decisions finds them from
+state and, for units with |z| < 2e-3 only, takes the decision the device took (match_decisions finds them from
 the device's bias gradients, which are the column sums of dz and show a switched term directly).  The
 canonical oracle -- the one the free-running engines and the loss curve are compared with -- never sees
 anything of the device.  The table reports how many decisions were matched and their largest |z|.
@@ -47,7 +47,11 @@ from oracle.cocod_oracle import OracleEngine             # noqa: E402
 from paper_1906_12043_b200 import inputs as I            # noqa: E402
 
 _SHM = {}
-BAND_MAX = 5e-4        # a ReLU decision may be matched to the device's only if |z| is below this
+# A ReLU decision may be matched to the device's only if |z| is below this.  The band is not set by fp32 accumulation
+# error (about 1e-6) but by the bf16 copies of the weights: from the second step of a round on, the two sides' fp32
+# masters differ in their last bits, a few hundred of them per worker straddle a bf16 rounding boundary, and each such
+# weight moves the pre-activations of its unit by one bf16 step of the weight times the input (up to about 7e-4).
+BAND_MAX = 2e-3
 
 
 def _decode_layer(layer, db_dev, db_ref, z, on, dz, pre):
@@ -365,7 +369,7 @@ def markdown(res, command):
            "workers after the merge (a one-ulp bf16 difference is 3.9e-3 to 7.8e-3 of the element); `share` = fraction of the "
            "parameters outside 1e-2.  `free` engines run from the common initial point without ever seeing the oracle's "
            "state and are compared with the canonical oracle; `restart` engines start every round from the canonical "
-           "oracle's x and v and are compared with the oracle branch that takes, for hidden units with |z| < 5e-4 only, "
+           "oracle's x and v and are compared with the oracle branch that takes, for hidden units with |z| < 2e-3 only, "
            "the ReLU decision the device took (`matched`: how many such decisions in the round, and their largest |z|).", "",
            f"Oracle loop: {res['oracle_processes']} processes, {res['oracle_seconds']:.0f} s of {res['wall_seconds']:.0f} s.", "",
            f"* largest restarted-per-round error: two-call {res['worst_restarted'][names[2]]:.2e}, fused {res['worst_restarted'][names[3]]:.2e} (bar 1e-2); "
