@@ -674,7 +674,8 @@ def measure_mlp(args, digest=False):
     local step), comm_end.  Every (worker, global step) has its own seeded minibatch (a pool of up to 2048 steps,
     generated on the device, labels from the teacher in fp64; a longer run goes through the pool again, like epochs
     over a data set).  Three variants are timed, each from the common initial point: the two calls, the fused
-    gradient + update call, and the fused call replayed from a CUDA graph of two rounds."""
+    gradient + update call, and the fused call replayed from CUDA graphs of two rounds each (one graph per pair of
+    rounds of the pool)."""
     import numpy as np
     import torch
     from paper_1906_12043_b200 import build, engine as E, inputs as I, mlp as M
@@ -712,14 +713,14 @@ def measure_mlp(args, digest=False):
         eng.set_params(x0)
         shadow = eng.bf16_shadow()
         n_rec = (warm + repeats * steps) * k
-        loss_all = torch.zeros((n_rec, K), dtype=torch.float32, device="cuda")
+        loss_all = torch.zeros((n_rec + 1, K), dtype=torch.float32, device="cuda")      # last row: calls that are not recorded
         step_no = [0]
         snaps = []
 
         def one_round(xs, ys, first, record_at=None):
             eng.comm_begin(side)
             for j in range(k):
-                out = loss_all[record_at + j] if (record_at is not None and record_at + k <= n_rec) else loss_all[0]
+                out = loss_all[record_at + j] if (record_at is not None and record_at + k <= n_rec) else loss_all[n_rec]
                 if fused:
                     mg.grad_step(eng, xs[first + j], ys[first + j], out)
                 else:
@@ -739,25 +740,30 @@ def measure_mlp(args, digest=False):
         torch.cuda.synchronize()
         graph = None
         if graphed:
-            # the captured rounds read their minibatches from a fixed staging area that is refilled (two device
-            # copies, inside the timed region) before every replay
-            stage_x = torch.empty((2 * k,) + tuple(pool_x.shape[1:]), dtype=pool_x.dtype, device="cuda")
-            stage_y = torch.empty((2 * k,) + tuple(pool_y.shape[1:]), dtype=pool_y.dtype, device="cuda")
+            # One captured graph per pair of rounds of the minibatch pool (two rounds = one full cycle of the buffer
+            # flip), each reading its own 2 k minibatches in place: replaying them in turn walks through the pool with
+            # nothing but graph launches in the timed region.
             cap = torch.cuda.Stream()
             eng.sync()
             eng.set_stream(cap)
-            lb = eng.launch_count + mg.launch_count
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=cap):
-                one_round(stage_x, stage_y, 0)
-                one_round(stage_x, stage_y, k)
-            per_replay = eng.launch_count + mg.launch_count - lb
+            graphs, per_replay = [], 0
+            n_graphs = min(pool_n // (2 * k), (repeats * steps + 4) // 2 + 2)
+            base = step_no[0]
+            for gi in range(n_graphs):
+                first = (base + gi * 2 * k) % pool_n
+                lb = eng.launch_count + mg.launch_count
+                g_ = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g_, stream=cap):
+                    one_round(pool_x, pool_y, first)
+                    one_round(pool_x, pool_y, first + k)
+                per_replay = eng.launch_count + mg.launch_count - lb
+                graphs.append(g_)
+            graph = graphs
+            plays = [0]
 
             def replay():
-                i = step_no[0] % pool_n
-                stage_x.copy_(pool_x[i:i + 2 * k], non_blocking=True)
-                stage_y.copy_(pool_y[i:i + 2 * k], non_blocking=True)
-                graph.replay()
+                graphs[plays[0] % n_graphs].replay()
+                plays[0] += 1
                 step_no[0] += 2 * k
 
             for _ in range(2):
