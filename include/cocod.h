@@ -61,7 +61,11 @@ enum {
      * write bf16(x) next to x (22 B and 14 B + 4/K per worker-parameter instead of 20 and
      * 12 + 4/K).  For workloads that compute gradients from bf16 weights with an fp32 master
      * copy.  1 allocates it, 0 frees it.  Not while a communication is in flight. */
-    COCOD_OPT_BF16_SHADOW = 3
+    COCOD_OPT_BF16_SHADOW = 3,
+    /* 1: consecutive local-step / merge kernels walk the K x P vector in alternating directions (and the mean kernel
+     * against the kernel that last wrote x), so that each starts on what its predecessor left in the L2 cache.
+     * Same values bit for bit.  0 (default): every kernel walks forwards. */
+    COCOD_OPT_SWEEP = 4
 };
 enum { COCOD_SNAPSHOT_COPY = 0, COCOD_SNAPSHOT_FLIP = 1 };
 

@@ -41,6 +41,8 @@ struct ProfileRec {
 // Where the kernel launched inside the current profiling bracket leaves its device-side time stamps
 // (nullptr outside a bracket, for the stateless entry points, and while profiling is off).
 thread_local unsigned long long *g_stamp = nullptr;
+// Experiment: direction in which the next streaming kernel walks its data (see COCOD_OPT_SWEEP).
+thread_local int g_backwards = 0;
 
 }  // namespace
 
@@ -80,6 +82,8 @@ struct cocod_engine {
     // bookkeeping
     int64_t steps = 0, launches = 0;
     int cuda_error = 0;
+    bool sweep = false;                 // COCOD_OPT_SWEEP: consecutive streaming kernels walk in alternating directions
+    int dir = 0;                        // direction of the last kernel on the compute stream
     bool profile = false;
     std::vector<ProfileRec> prof;
     unsigned long long *stamps = nullptr;       // device: kMaxProfile x {earliest start, latest end} in ns of the GPU's clock
@@ -119,11 +123,11 @@ cudaError_t launch_local_step(const float *x_in, float *x_out, float *v, const f
         if (shadow != nullptr)
             local_step_vec4<THREADS, UNROLL, true><<<grid, THREADS, 0, s>>>(
                 reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
-                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, shadow, g_stamp);
+                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, shadow, g_stamp, g_backwards);
         else
             local_step_vec4<THREADS, UNROLL, false><<<grid, THREADS, 0, s>>>(
                 reinterpret_cast<const float4 *>(x_in), reinterpret_cast<float4 *>(x_out),
-                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, nullptr, g_stamp);
+                reinterpret_cast<float4 *>(v), reinterpret_cast<const float4 *>(g), nvec, lr, mu, wd, nullptr, g_stamp, g_backwards);
         done = nvec * 4;
         if (n_launch) ++*n_launch;
     }
@@ -170,7 +174,7 @@ cudaError_t launch_mean(const float *snap, int K, int64_t P, const float *w, flo
     } else if ((P % 4) == 0 && aligned16(snap) && aligned16(mean)) {
         const int64_t pvec = P / 4;
         mean_vec4<<<grid_for(pvec, kThreads), kThreads, 0, s>>>(
-            reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k, g_stamp);
+            reinterpret_cast<const float4 *>(snap), K, pvec, w, reinterpret_cast<float4 *>(mean), inv_k, g_stamp, g_backwards);
     } else {
         mean_scalar<<<grid_for(P, kThreads), kThreads, 0, s>>>(snap, K, P, w, mean, inv_k);
     }
@@ -210,10 +214,10 @@ cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, 
         (shadow == nullptr || aligned16(shadow))) {
         // rows per thread: as many as K allows up to 8 (registers scale with it)
         const unsigned gx = grid_for(P / 8, kThreads);
-        if (K >= 8) merge_vec8<8><<<dim3(gx, (unsigned)((K + 7) / 8)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
-        else if (K >= 4) merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
-        else if (K >= 2) merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
-        else merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp);
+        if (K >= 8) merge_vec8<8><<<dim3(gx, (unsigned)((K + 7) / 8)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp, g_backwards);
+        else if (K >= 4) merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp, g_backwards);
+        else if (K >= 2) merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp, g_backwards);
+        else merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x, snap, mean, K, P, shadow, g_stamp, g_backwards);
     } else if ((P % 4) == 0 && aligned16(x) && aligned16(snap) && aligned16(mean) &&
                (shadow == nullptr || (reinterpret_cast<uintptr_t>(shadow) & 7u) == 0)) {
         const int64_t pvec = P / 4;
@@ -368,8 +372,12 @@ int step_range(cocod_engine *h, const float *g, int64_t off, int64_t len)
     int nl = 0;
     {
         Bracket br(h, h->compute, COCOD_KERNEL_LOCAL_STEP);
-        CK(h, launch_local_step(x_in, x_out, h->v + off, g, len, h->lr, h->mu, h->wd,
-                                h->shadow ? h->shadow + off : nullptr, h->compute, &nl));
+        if (h->sweep && off == 0) h->dir ^= 1;
+        g_backwards = h->sweep ? h->dir : 0;
+        const cudaError_t e = launch_local_step(x_in, x_out, h->v + off, g, len, h->lr, h->mu, h->wd,
+                                                h->shadow ? h->shadow + off : nullptr, h->compute, &nl);
+        g_backwards = 0;
+        CK(h, e);
     }
     h->launches += nl;
     return COCOD_OK;
@@ -523,7 +531,10 @@ int cocod_comm_begin(cocod_handle *h, cocod_stream_t side)
     int nl = 0;
     {
         Bracket br(h, h->side, COCOD_KERNEL_MEAN);
-        CK(h, launch_mean(h->snap, h->K, h->P, mean_weights(h), h->mean, mean_scale(h), h->side, &nl));
+        g_backwards = h->sweep ? (h->dir ^ 1) : 0;       // against the kernel that last wrote x
+        const cudaError_t e = launch_mean(h->snap, h->K, h->P, mean_weights(h), h->mean, mean_scale(h), h->side, &nl);
+        g_backwards = 0;
+        CK(h, e);
     }
     h->launches += nl;
     h->mean_started = true;
@@ -575,7 +586,11 @@ int cocod_comm_end(cocod_handle *h)
     {
         Bracket br(h, h->compute, COCOD_KERNEL_MERGE);
         // with no local step since comm_begin (FLIP) x still aliases the stored copies
-        CK(h, launch_merge(h->buf[h->cur], h->snap, h->mean, h->K, h->P, h->shadow, h->compute, &nl));
+        if (h->sweep) h->dir ^= 1;
+        g_backwards = h->sweep ? h->dir : 0;
+        const cudaError_t e = launch_merge(h->buf[h->cur], h->snap, h->mean, h->K, h->P, h->shadow, h->compute, &nl);
+        g_backwards = 0;
+        CK(h, e);
     }
     h->launches += nl;
     h->pending_flip = false;
@@ -745,6 +760,10 @@ int cocod_set_option(cocod_handle *h, int option, int value)
         if (value != COCOD_SNAPSHOT_COPY && value != COCOD_SNAPSHOT_FLIP) return COCOD_ERR_INVALID;
         if (h->state != IDLE) return COCOD_ERR_STATE;
         h->snapshot_mode = value;
+        return COCOD_OK;
+    case COCOD_OPT_SWEEP:
+        h->sweep = value != 0;
+        h->dir = 0;
         return COCOD_OK;
     case COCOD_OPT_PROFILE:
         if (value && !h->stamps) {      // device-side time stamps: 256 KB, kept until the handle is destroyed

@@ -37,9 +37,11 @@ constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTE
 constexpr int TMEM_COLS = 128;
 constexpr int MAX_STAGES = STAGES;
 // ring (at least two stages: the fp32 epilogue stages a whole 128 x 128 tile = 64 KB there) + alignment
-// slack + a tail holding the barriers (256 B) and the bias tile (512 B)
+// slack + a tail holding the barriers (256 B), the bias tile (512 B)
 __host__ __device__ constexpr int ring_stages(int stages) { return stages < 2 ? 2 : stages; }
-__host__ __device__ constexpr int smem_bytes(int stages) { return ring_stages(stages) * STAGE_BYTES + 1024 + 1024; }
+// ... and, behind them, room for a slice of the output layer's weights (16 classes x 128 columns fp32, 8 KB)
+constexpr int TAIL_BYTES = 1024 + 16 * BN * 4;
+__host__ __device__ constexpr int smem_bytes(int stages) { return ring_stages(stages) * STAGE_BYTES + 1024 + TAIL_BYTES; }
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 enum Epilogue {
@@ -85,6 +87,13 @@ struct Params {
     float *colsum;                     // EPI_MASK, optional: [N] column sums of the bf16 output (needs M <= 128)
     long long colsum_worker_stride;
     StepTarget colsum_step;            // ... or (x_in != nullptr) the local step of that [N] tensor, the sums as gradient
+    // EPI_BIAS_RELU, optional (logit_part != nullptr; needs M <= 128 and 128 threads): this tile's contribution to the
+    // next (narrow) layer, part[w][tile_n][m][c] = sum_{n in tile} o[m][n] * w_next[c][n] for c < next_out <= 16, taken
+    // from the bf16 values o the tile stores; rows of 16 floats.  Summed over tile_n by whoever reads it.
+    float *logit_part;
+    const __nv_bfloat16 *w_next;       // [next_out][N] per worker, row stride N
+    long long w_next_worker_stride;
+    int next_out;
     int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
@@ -251,6 +260,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
     float *sbias = reinterpret_cast<float *>(tail + 256);
+    float *swn = reinterpret_cast<float *>(tail + 1024);       // [16][BN] slice of the next layer's weights
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, wk = blockIdx.z;
@@ -357,6 +367,13 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (EPI == EPI_BIAS_RELU) {
             const __nv_bfloat16 *bias = p.bias + (long long)wk * p.bias_worker_stride;
             for (int i = threadIdx.x - 64; i < BN; i += NT - 64) sbias[i] = (n0 + i < p.N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
+            if (p.logit_part != nullptr) {
+                const __nv_bfloat16 *wn = p.w_next + (long long)wk * p.w_next_worker_stride;
+                for (int i = threadIdx.x - 64; i < 16 * BN; i += NT - 64) {
+                    const int c = i / BN, j = i % BN;
+                    swn[i] = (c < p.next_out && n0 + j < p.N) ? __bfloat162float(wn[(long long)c * p.N + n0 + j]) : 0.0f;
+                }
+            }
         }
     }
     auto load_mask = [&]() {
@@ -427,6 +444,9 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                         if (n0 + (cbase + cc) * 32 + j < p.N) dst[(cbase + cc) * 32 + j] = __uint_as_float(r[cc][j]);
             }
         } else {
+            float nacc[16];                    // EPI_BIAS_RELU with logit_part: this row's partial outputs of the next layer
+#pragma unroll
+            for (int c = 0; c < 16; ++c) nacc[c] = 0.0f;
 #pragma unroll
             for (int cc = 0; cc < NCH; ++cc) {
                 const int c = cbase + cc;
@@ -442,6 +462,23 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     }
                     outv[j] = __float2bfloat16_rn(a);
                 }
+                if (EPI == EPI_BIAS_RELU && NT == 128 && p.logit_part != nullptr) {
+                    // columns in order, classes innermost: a fixed summation order
+                    for (int j4 = 0; j4 < 32; j4 += 4) {
+                        const float h0 = __bfloat162float(outv[j4]), h1 = __bfloat162float(outv[j4 + 1]);
+                        const float h2 = __bfloat162float(outv[j4 + 2]), h3 = __bfloat162float(outv[j4 + 3]);
+#pragma unroll
+                        for (int q = 0; q < 16; ++q) {
+                            if (q < p.next_out) {
+                                const float4 wv = *reinterpret_cast<const float4 *>(swn + q * BN + c * 32 + j4);
+                                nacc[q] = fmaf(h0, wv.x, nacc[q]);
+                                nacc[q] = fmaf(h1, wv.y, nacc[q]);
+                                nacc[q] = fmaf(h2, wv.z, nacc[q]);
+                                nacc[q] = fmaf(h3, wv.w, nacc[q]);
+                            }
+                        }
+                    }
+                }
                 // stage the bf16 row in the (now idle) ring in the TMA swizzle: 64-column boxes of 128-byte rows,
                 // 16-byte piece j of row r at piece j ^ (r & 7)
                 {
@@ -451,6 +488,11 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     for (int j = 0; j < 4; ++j)
                         *reinterpret_cast<uint4 *>(box + ((((c & 1) * 4 + j) ^ (row & 7)) << 4)) = src[j];
                 }
+            }
+            if (EPI == EPI_BIAS_RELU && NT == 128 && p.logit_part != nullptr && m < p.M) {
+                float4 *dst = reinterpret_cast<float4 *>(p.logit_part + (((long long)wk * gridDim.x + blockIdx.x) * BM + row) * 16);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) dst[q] = make_float4(nacc[4 * q], nacc[4 * q + 1], nacc[4 * q + 2], nacc[4 * q + 3]);
             }
             // the tile leaves through two bulk stores (whole 128-byte lines; rows and columns beyond the
             // matrix are clipped by the tensor map)

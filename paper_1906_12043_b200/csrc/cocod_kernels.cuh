@@ -115,10 +115,13 @@ template <int THREADS, int UNROLL, bool SHADOW>
 __global__ void __launch_bounds__(THREADS)
 local_step_vec4(const float4 *x_in, float4 *x_out, float4 *v, const float4 *__restrict__ g,
                 int64_t nvec, float lr, float mu, float wd, __nv_bfloat16 *__restrict__ shadow,
-                unsigned long long *stamp)
+                unsigned long long *stamp, int backwards)
 {
     stamp_begin(stamp);
-    const int64_t base = (int64_t)blockIdx.x * (THREADS * UNROLL) + threadIdx.x;
+    // backwards: the grid walks the vector from its end, so that a kernel that follows one that walked forwards starts
+    // on what that one left in L2
+    const unsigned blk = backwards ? gridDim.x - 1u - blockIdx.x : blockIdx.x;
+    const int64_t base = (int64_t)blk * (THREADS * UNROLL) + threadIdx.x;
     float4 xr[UNROLL], vr[UNROLL], gr[UNROLL];
     if (base + (int64_t)(UNROLL - 1) * THREADS < nvec) {       // full tile: no predicates
 #pragma unroll
@@ -265,10 +268,11 @@ __device__ __forceinline__ void mean_rows(float (&s)[NV], int K, const float *__
 // One thread owns one float4 of columns.  Needs P mod 4 == 0 and 16-byte aligned bases.
 static __global__ void __launch_bounds__(kThreads)
 mean_vec4(const float4 *__restrict__ snap, int K, int64_t pvec, const float *__restrict__ w,
-          float4 *__restrict__ mean, float inv_k, unsigned long long *stamp)
+          float4 *__restrict__ mean, float inv_k, unsigned long long *stamp, int backwards)
 {
     stamp_begin(stamp);
-    const int64_t c = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    const unsigned blk = backwards ? gridDim.x - 1u - blockIdx.x : blockIdx.x;
+    const int64_t c = (int64_t)blk * kThreads + threadIdx.x;
     if (c >= pvec) return;
     const float4 *col = snap + c;
     float s[4];
@@ -420,13 +424,15 @@ merge_vec4(float4 *x, const float4 *snap, const float4 *__restrict__ mean, int K
 template <int RC>
 __global__ void __launch_bounds__(kThreads)
 merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P,
-           __nv_bfloat16 *__restrict__ shadow, unsigned long long *stamp)
+           __nv_bfloat16 *__restrict__ shadow, unsigned long long *stamp, int backwards)
 {
     stamp_begin(stamp);
-    const int64_t c = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * 8;
+    const unsigned bx = backwards ? gridDim.x - 1u - blockIdx.x : blockIdx.x;
+    const unsigned by = backwards ? gridDim.y - 1u - blockIdx.y : blockIdx.y;
+    const int64_t c = ((int64_t)bx * kThreads + threadIdx.x) * 8;
     if (c >= P) return;
     const f32x8 m = ld256(mean + c);
-    const int i0 = blockIdx.y * RC;
+    const int i0 = by * RC;
     f32x8 xr[RC], sr[RC];
 #pragma unroll
     for (int j = 0; j < RC; ++j)

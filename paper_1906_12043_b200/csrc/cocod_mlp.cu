@@ -7,7 +7,8 @@
 //
 //   h1 = bf16(relu(x  W1^T + b1))     GEMM 128 x d_h x d_in   A = x, B = W1            epilogue bias+ReLU
 //   h2 = bf16(relu(h1 W2^T + b2))     GEMM 128 x d_h x d_h    A = h1, B = W2           epilogue bias+ReLU
-//   logits = h2 W3^T + b3 ; loss ; dz3 = bf16((softmax - onehot)/batch)                CUDA cores
+//   logits = h2 W3^T + b3 (per-tile partial sums from the epilogue of the GEMM above) ;
+//   loss ; dz3 = bf16((softmax - onehot)/batch)                                       CUDA cores
 //   dz2 = bf16((dz3 W3) * (h2 > 0)) ; dW3 = dz3^T h2 ; db3, db2 = column sums           CUDA cores
 //   dz1 = bf16((dz2 W2) * (h1 > 0))   GEMM 128 x d_h x d_h    A = dz2, B = W2 read [k][n]  epilogue mask,
 //   db1 = column sums of dz1                                   (same epilogue: the batch is one tile)
@@ -161,103 +162,20 @@ inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK -
 // warps per CTA of head_backward (measured inside the gradient chain: 2 warps 20.3 us, 4 warps 14.3 us,
 // 8 warps 15.9 us; about 8 us of it is fixed cost, not the loop over the samples)
 constexpr int HEAD_NW = 4;
-// Output layer forward and loss.  One CTA = 8 samples of one worker (one per warp); W3 sits in shared
-// memory; every lane loads its slices of the h2 row up front (all loads in flight at once):
-// logits = h2 W3^T + b3 (fp32), row loss = -log softmax[label], dz3 = bf16((softmax - onehot) / batch)
-// kept as fp32 values in dz3[w][b][16].  grid (B / 8, K).
-// DOUT: compile-time bound of the class loops (>= d_out; 10 for the paper-shaped workload, else 16).
-template <int DOUT>
-__global__ void __launch_bounds__(256)
-head_logits(const bf16 *__restrict__ h2, const bf16 *__restrict__ params, long long P, long long oW3, long long ob3,
-            const int *__restrict__ labels, float *__restrict__ dz3, float *__restrict__ rowloss, int B, int d_h,
-            int d_out)
-{
-    extern __shared__ __align__(16) uint8_t head_smem[];
-    bf16 *sW3 = reinterpret_cast<bf16 *>(head_smem);                 // [d_out][d_h]
-    pdl_launch_dependents();
-    pdl_wait();
-    const int w = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.x * 8 + warp;
-    const bf16 *hrow = h2 + ((long long)w * B + b) * d_h;
-    constexpr int MAXV = 4;                                          // 4 x 256 columns per pass
-    uint4 hv[MAXV];
-#pragma unroll
-    for (int q = 0; q < MAXV; ++q) {
-        const int j = lane * 8 + q * 256;
-        hv[q] = (j < d_h) ? *reinterpret_cast<const uint4 *>(hrow + j) : make_uint4(0, 0, 0, 0);
-    }
-    const bf16 *W3 = params + (long long)w * P + oW3;
-    for (int i = threadIdx.x * 8; i < d_out * d_h; i += 256 * 8)
-        *reinterpret_cast<uint4 *>(sW3 + i) = *reinterpret_cast<const uint4 *>(W3 + i);
-    const bf16 *b3 = params + (long long)w * P + ob3;
-    const float bias = (lane < d_out) ? __bfloat162float(b3[lane]) : 0.0f;
-    const int y = labels[(long long)w * B + b];
-    __syncthreads();
-    float acc[DOUT];
-#pragma unroll
-    for (int c = 0; c < DOUT; ++c) acc[c] = 0.0f;
-    for (int j0 = 0; j0 < d_h; j0 += 256 * MAXV) {
-        if (j0 > 0) {
-#pragma unroll
-            for (int q = 0; q < MAXV; ++q) {
-                const int j = j0 + lane * 8 + q * 256;
-                hv[q] = (j < d_h) ? *reinterpret_cast<const uint4 *>(hrow + j) : make_uint4(0, 0, 0, 0);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < MAXV; ++q) {
-            const int j = j0 + lane * 8 + q * 256;
-            if (j < d_h) {
-                const bf16 *hp = reinterpret_cast<const bf16 *>(&hv[q]);
-                float hf[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) hf[e] = __bfloat162float(hp[e]);
-#pragma unroll
-                for (int c = 0; c < DOUT; ++c) {
-                    if (DOUT == 10 || c < d_out) {
-                        const uint4 wv = *reinterpret_cast<const uint4 *>(sW3 + c * d_h + j);
-                        const bf16 *wp = reinterpret_cast<const bf16 *>(&wv);
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) acc[c] = fmaf(hf[e], __bfloat162float(wp[e]), acc[c]);
-                    }
-                }
-            }
-        }
-    }
-#pragma unroll
-    for (int c = 0; c < DOUT; ++c)
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
-    // lane c finishes class c
-    float z = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < DOUT; ++c)
-        if (lane == c && c < d_out) z = acc[c] + bias;
-    float zmax = z;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
-    const float e = (lane < d_out) ? expf(z - zmax) : 0.0f;
-    float ssum = e;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
-    const float pc = e / ssum;
-    if (lane < 16) {
-        const float d = (lane < d_out) ? (pc - (lane == y ? 1.0f : 0.0f)) / (float)B : 0.0f;
-        dz3[((long long)w * B + b) * 16 + lane] = __bfloat162float(__float2bfloat16_rn(d));
-    }
-    const float py = __shfl_sync(0xffffffffu, pc, y);
-    if (lane == 0) rowloss[(long long)w * B + b] = -logf(py);
-}
-
-// Everything downstream of dz3 that runs on CUDA cores, for 32 hidden units j and all 128 samples:
+// The output layer and everything downstream of it that runs on CUDA cores.  The second hidden layer's GEMM leaves, per
+// 128-column tile t, the partial logits part[w][t][b][c] = sum_{j in tile} h2[b][j] W3[c][j]; every CTA here first finishes
+// them for all samples of its worker (thread b: z[c] = b3[c] + sum_t part[t][b][c] in tile order, softmax, row loss
+// -log softmax[label], dz3[b][c] = bf16((softmax - onehot) / batch), kept in shared memory), then, for its 32 hidden
+// units j and all samples:
 //   dz2[b][j] = bf16((sum_c dz3[b][c] W3[c][j]) * (h2[b][j] > 0)),  db2[j] = sum_b dz2[b][j],
 //   dW3[c][j] = sum_b dz3[b][c] h2[b][j];
-// one extra CTA per worker writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b rowloss and the zero padding of
-// the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32 + 1, K).
+// one extra CTA per worker writes db3[c] = sum_b dz3[b][c], loss[w] = mean_b row loss and the zero padding of
+// the gradient.  Fixed summation orders (deterministic).  grid (d_h / 32 + 1, K).  (Recomputing the 128 softmaxes in
+// each of a worker's 33 CTAs costs about a microsecond and saves a kernel of 8.5 us that did nothing else.)
 template <int DOUT, int NW>
 __global__ void __launch_bounds__(32 * NW)
-head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__restrict__ dz3,
-              const float *__restrict__ rowloss, bf16 *__restrict__ dz2, float *__restrict__ grads,
+head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__restrict__ part, int n_tiles,
+              const int *__restrict__ labels, bf16 *__restrict__ dz2, float *__restrict__ grads,
               float *__restrict__ loss, long long P, long long P_raw, long long oW3, long long ob2, long long ob3,
               int B, int d_h, int d_out, const StepTarget step)
 {
@@ -268,17 +186,60 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
     static_assert(NW >= 2, "the scalar CTA uses two warps");
     constexpr int C4 = (DOUT + 3) / 4;
     __shared__ __align__(16) float sdz[128 * 16];
+    __shared__ float srowloss[128];
     __shared__ float red[NW][16][33];
     __shared__ float colsum[NW][33];
     const int w = blockIdx.y, j0 = blockIdx.x * 32, lane = threadIdx.x & 31, wp = threadIdx.x >> 5;
     const int j = j0 + lane;
+    const bool scalar_cta = (blockIdx.x == gridDim.x - 1);
     pdl_launch_dependents();
     pdl_wait();
-    if (blockIdx.x == gridDim.x - 1) {
+    // first batch of this thread's h2 values: in flight while the logits are finished
+    float hreg[16];
+    if (!scalar_cta) {
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+            const int b = wp + NW * q;
+            hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
+        }
+    }
+    // the logits, softmax, row loss and dz3 of sample b (B <= 128)
+    for (int b = threadIdx.x; b < B; b += 32 * NW) {
+        float z[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) z[c] = (c < d_out) ? __bfloat162float(params[(long long)w * P + ob3 + c]) : 0.0f;
+        const float4 *pp = reinterpret_cast<const float4 *>(part + (((long long)w * n_tiles) * 128 + b) * 16);
+        for (int t = 0; t < n_tiles; ++t) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float4 v = __ldcg(pp + (long long)t * (128 * 16 / 4) + q);
+                z[4 * q] += v.x; z[4 * q + 1] += v.y; z[4 * q + 2] += v.z; z[4 * q + 3] += v.w;
+            }
+        }
+        float zmax = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) if (c < d_out) zmax = fmaxf(zmax, z[c]);
+        float e[16], ssum = 0.0f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            e[c] = (c < d_out) ? expf(z[c] - zmax) : 0.0f;
+            ssum += e[c];
+        }
+        const int y = labels[(long long)w * B + b];
+        float py = 0.0f;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            const float pc = e[c] / ssum;
+            if (c == y) py = pc;
+            const float d = (c < d_out) ? (pc - (c == y ? 1.0f : 0.0f)) / (float)B : 0.0f;
+            sdz[b * 16 + c] = __bfloat162float(__float2bfloat16_rn(d));
+        }
+        srowloss[b] = -logf(py);
+    }
+    if (scalar_cta) {
         // The extra CTA of every worker: the per-worker scalars db3[c] = sum_b dz3[b][c], loss = mean_b rowloss and
         // the zero padding of the gradient, each by one warp (lane-strided partial sums, then a fixed shuffle tree).
         // As an epilogue of one of the column CTAs this made that CTA the straggler of the kernel (2.3 us).
-        for (int i = threadIdx.x; i < B * 16; i += 32 * NW) sdz[i] = dz3[(long long)w * B * 16 + i];
         __syncthreads();
         if (wp == 0) {
             for (int c = 0; c < d_out; ++c) {
@@ -295,9 +256,8 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
             float t[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-                if (lane + 32 * i < B) t[i] = rowloss[(long long)w * B + lane + 32 * i];
+                if (lane + 32 * i < B) t[i] = srowloss[lane + 32 * i];
             float s = (t[0] + t[1]) + (t[2] + t[3]);
-            for (int b = lane + 128; b < B; b += 32) s += rowloss[(long long)w * B + b];
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             if (lane == 0) loss[w] = s / (float)B;
@@ -308,14 +268,6 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
         }
         return;
     }
-    // first batch of this thread's h2 values: in flight while dz3 and W3 are fetched
-    float hreg[16];
-#pragma unroll
-    for (int q = 0; q < 16; ++q) {
-        const int b = wp + NW * q;
-        hreg[q] = (b < B) ? __bfloat162float(h2[((long long)w * B + b) * d_h + j]) : 0.0f;
-    }
-    for (int i = threadIdx.x; i < B * 16; i += 32 * NW) sdz[i] = dz3[(long long)w * B * 16 + i];
     float w3[4 * C4], acc3[4 * C4];
 #pragma unroll
     for (int c = 0; c < 4 * C4; ++c) {
@@ -388,7 +340,7 @@ struct cocod_mlp {
     int K, B, d_in, d_h, d_out;
     long long P, P_raw, oW1, ob1, oW2, ob2, oW3, ob3;
     bf16 *h1 = nullptr, *h2 = nullptr, *dz2 = nullptr, *dz1 = nullptr;
-    float *dz3 = nullptr, *rowloss = nullptr;
+    float *logit_part = nullptr;        // [K][d_h / 128][128][16]: per-tile partial logits left by the second layer's GEMM
     int *error_flag = nullptr;
     // maps over scratch (fixed addresses): reduction-contiguous (k) and row-contiguous (mn) views
     CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
@@ -431,7 +383,7 @@ bool mlp_profile_open(cocod_mlp *h, std::vector<std::pair<cudaEvent_t, cudaEvent
 void mlp_free(cocod_mlp *h)
 {
     mlp_profile_clear(h);
-    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->dz3, h->rowloss, h->error_flag};
+    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->logit_part, h->error_flag};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
@@ -467,17 +419,12 @@ int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_h
     alloc((void **)&h->h2, act);
     alloc((void **)&h->dz2, act);
     alloc((void **)&h->dz1, act);
-    alloc((void **)&h->dz3, (size_t)K * batch * 16 * sizeof(float));
-    alloc((void **)&h->rowloss, (size_t)K * batch * sizeof(float));
+    alloc((void **)&h->logit_part, (size_t)K * (d_hidden / 128) * 128 * 16 * sizeof(float));
     alloc((void **)&h->error_flag, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->error_flag, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(head_logits<10>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * d_hidden * (int)sizeof(bf16));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(head_logits<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 16 * d_hidden * (int)sizeof(bf16));
     if (e != cudaSuccess) {
         cudaGetLastError();
         mlp_free(h);
@@ -568,15 +515,13 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
     p.bias = prm + h->ob1; p.bias_worker_stride = P;
     GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, pdl_fwd)));
-    // h2 = relu(h1 W2^T + b2)
+    // h2 = relu(h1 W2^T + b2), and per 128-column tile the partial logits h2 W3^T of that tile
     p.K = d_h; p.stages = stages_for(d_h); p.bias = prm + h->ob2;
+    p.logit_part = h->logit_part; p.w_next = prm + h->oW3; p.w_next_worker_stride = P; p.next_out = d_out;
     GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, pdl_fwd)));
-    // output layer, loss, dz3; then dz2, dW3, db3, db2
-    const size_t w3_bytes = (size_t)d_out * d_h * sizeof(bf16);
-    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_logits<10> : head_logits<16>, dim3(B / 8, K), dim3(256), w3_bytes, s,
-                             h->h2, prm, P, h->oW3, h->ob3, labels, h->dz3, h->rowloss, B, d_h, d_out));
+    // logits, loss, dz3; then dz2, dW3, db3, db2
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
-                             dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->dz3, (const float *)h->rowloss,
+                             dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->logit_part, d_h / 128, labels,
                              h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out, small));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
     Params q{};

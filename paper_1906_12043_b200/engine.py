@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libcocod.so")
 OK, ERR_INVALID, ERR_OOM, ERR_STATE, ERR_CUDA, ERR_TIMEOUT, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
 NOALLOC_MAX_ELEMS = 4 * 1024 * 1024
 IPC_EXPORT_BYTES = 256
-OPT_SNAPSHOT, OPT_PROFILE, OPT_BF16_SHADOW = 1, 2, 3
+OPT_SNAPSHOT, OPT_PROFILE, OPT_BF16_SHADOW, OPT_SWEEP = 1, 2, 3, 4
 SNAPSHOT_COPY, SNAPSHOT_FLIP = 0, 1
 KERNEL_LOCAL_STEP, KERNEL_SNAPSHOT, KERNEL_MEAN, KERNEL_MERGE = 0, 1, 2, 3
 KERNEL_NAMES = {0: "local_step", 1: "snapshot", 2: "mean", 3: "merge"}

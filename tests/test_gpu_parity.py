@@ -157,9 +157,15 @@ def test_config1_full_vector_parity(E, snapshot):
     x = cpu(eng.get_params()).astype(np.float64)
     rel = np.abs(x - ref.x) / np.maximum(np.abs(ref.x.astype(np.float64)), 1e-300)
     ulps = np.abs(cpu(eng.get_params()).view(np.int32).astype(np.int64) - mir.x.view(np.int32).astype(np.int64))
+    # the unfloored figure: plain per-element relative error over all elements that are not vanishingly small
+    # (|ref| > 1e-3 * rms; the scaled bar above puts a floor of rms under |ref|, because an element that happens to lie
+    # near zero after cancellation carries the absolute rounding error of its much larger summands)
+    rms = np.sqrt(np.mean(ref.x.astype(np.float64) ** 2))
+    big = np.abs(ref.x) > 1e-3 * rms
     print(f"config1 after the run: max relative error {rel.max():.3e}, 99.99th percentile {np.quantile(rel, 0.9999):.3e}, "
+          f"max over the {big.mean():.4%} of elements with |ref| > 1e-3 rms {rel[big].max():.3e}, "
           f"max distance to the mirror {int(ulps.max())} ulp")
-    assert ulps.max() == 0 and np.quantile(rel, 0.9999) < 1e-3
+    assert ulps.max() == 0 and np.quantile(rel, 0.9999) < 1e-3 and rel[big].max() < 1e-2
 
 
 # ----------------------------------------------------------------------------- shapes: tiles, ragged tails, misaligned rows
