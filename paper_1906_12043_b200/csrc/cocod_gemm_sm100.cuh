@@ -35,6 +35,7 @@ namespace gemm {
 constexpr int BM = 128, BN = 128, BK = 64, STAGES = 6, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int TMEM_COLS = 128;
+constexpr int NEXT_N = 16;             // width of the optional second contraction (the output layer's classes, padded)
 constexpr int MAX_STAGES = STAGES;
 // ring (at least two stages: the fp32 epilogue stages a whole 128 x 128 tile = 64 KB there) + alignment
 // slack + a tail holding the barriers (256 B), the bias tile (512 B)
@@ -89,10 +90,12 @@ struct Params {
     StepTarget colsum_step;            // ... or (x_in != nullptr) the local step of that [N] tensor, the sums as gradient
     // EPI_BIAS_RELU, optional (logit_part != nullptr; needs M <= 128 and 128 threads): this tile's contribution to the
     // next (narrow) layer, part[w][tile_n][m][c] = sum_{n in tile} o[m][n] * w_next[c][n] for c < next_out <= 16, taken
-    // from the bf16 values o the tile stores; rows of 16 floats.  Summed over tile_n by whoever reads it.
+    // from the bf16 values o the tile stores; rows of 16 floats.  Summed over tile_n by whoever reads it.  It is a second,
+    // small contraction on the tensor cores: A = the staged output tile (it sits in shared memory in exactly the
+    // operand layout), B = the 16 x 128 slice of w_next fetched through map_n, accumulator = 16 more TMEM columns.
     float *logit_part;
-    const __nv_bfloat16 *w_next;       // [next_out][N] per worker, row stride N
-    long long w_next_worker_stride;
+    const __nv_bfloat16 *b_next;       // [next_out] per worker: added by the CTAs of tile_n == 0
+    long long b_next_worker_stride;
     int next_out;
     int stages;                        // shared-memory ring depth, 1 .. MAX_STAGES
     int *error_flag;
@@ -213,6 +216,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
                    "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
                  : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptors (version 1 = sm_100, 128-byte swizzle), for tiles laid out by TMA:
@@ -233,21 +244,23 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, bool mn_major)
     return d;
 }
 // Instruction descriptor: D fp32, A and B bf16, M = 128, N = 128, operand majors as given.
-__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn)
+__host__ __device__ constexpr uint32_t instr_desc(bool a_mn, bool b_mn, int n = BN)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------------ kernel
 // Tensor maps: a K-major operand is {k (contiguous), rows, workers} with box {64, 128, 1}; an
 // MN-major operand is {m or n (contiguous), k, workers} with box {64, 64, 1} (two boxes per tile).
 // map_c (EPI_F32 only): {n (contiguous), m, workers} fp32 with box {32, 128, 1}, 128-byte swizzle.
+// map_n (EPI_BIAS_RELU with logit_part): the next layer's weights {n (contiguous), classes, workers} bf16, box {64, 16, 1}
+// (classes beyond the matrix are zero-filled).
 // NT threads per CTA: 128 (every thread drains one accumulator row; 256 would let two threads share a row).
 template <int EPI, bool A_MN, bool B_MN, int NT>
 __global__ void __launch_bounds__(NT)
 gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-          const __grid_constant__ CUtensorMap map_c, const Params p)
+          const __grid_constant__ CUtensorMap map_c, const __grid_constant__ CUtensorMap map_n, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -260,7 +273,9 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
     float *sbias = reinterpret_cast<float *>(tail + 256);
-    float *swn = reinterpret_cast<float *>(tail + 1024);       // [16][BN] slice of the next layer's weights
+    uint8_t *swn = tail + 1024;                  // the next layer's weight slice: two k-blocks of 16 rows x 128 bytes
+    const uint32_t wn_full = smem_u32(bars + 2 * MAX_STAGES + 1), wn_done = smem_u32(bars + 2 * MAX_STAGES + 2);
+    const bool with_next = (EPI == EPI_BIAS_RELU) && (NT == 128) && (p.logit_part != nullptr);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM, wk = blockIdx.z;
@@ -298,6 +313,8 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             mbar_init(empty0 + 8 * s, 1);
         }
         mbar_init(accum, 1);
+        mbar_init(wn_full, 1);
+        mbar_init(wn_done, 1);
         abort[0] = 0;
         abort[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -306,11 +323,18 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         // the first ring of copies starts now, under the rest of the set-up
         if (!p.debug_no_loads)
             for (; armed < nkb && armed < stages; ++armed) issue_loads(armed, armed);
+        if (with_next && !p.debug_no_loads) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_n) : "memory");
+            mbar_expect_tx(wn_full, 2 * NEXT_N * 128);
+            tma_load_3d(smem_u32(swn), &map_n, wn_full, n0, 0, wk);
+            tma_load_3d(smem_u32(swn) + NEXT_N * 128, &map_n, wn_full, n0 + 64, 0, wk);
+        }
     }
     if (threadIdx.x == 0) COCOD_TRACE(6);
     __syncwarp();
+    const uint32_t tmem_cols = with_next ? 2 * TMEM_COLS : TMEM_COLS;      // (a power of two)
     if (warp == 0) {                  // warp-collective TMEM allocation
-        tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+        tmem_alloc(smem_u32(tmem_slot), tmem_cols);
         tmem_relinquish();
     }
     if (threadIdx.x == 0) COCOD_TRACE(7);
@@ -367,13 +391,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (EPI == EPI_BIAS_RELU) {
             const __nv_bfloat16 *bias = p.bias + (long long)wk * p.bias_worker_stride;
             for (int i = threadIdx.x - 64; i < BN; i += NT - 64) sbias[i] = (n0 + i < p.N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
-            if (p.logit_part != nullptr) {
-                const __nv_bfloat16 *wn = p.w_next + (long long)wk * p.w_next_worker_stride;
-                for (int i = threadIdx.x - 64; i < 16 * BN; i += NT - 64) {
-                    const int c = i / BN, j = i % BN;
-                    swn[i] = (c < p.next_out && n0 + j < p.N) ? __bfloat162float(wn[(long long)c * p.N + n0 + j]) : 0.0f;
-                }
-            }
         }
     }
     auto load_mask = [&]() {
@@ -444,9 +461,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                         if (n0 + (cbase + cc) * 32 + j < p.N) dst[(cbase + cc) * 32 + j] = __uint_as_float(r[cc][j]);
             }
         } else {
-            float nacc[16];                    // EPI_BIAS_RELU with logit_part: this row's partial outputs of the next layer
-#pragma unroll
-            for (int c = 0; c < 16; ++c) nacc[c] = 0.0f;
 #pragma unroll
             for (int cc = 0; cc < NCH; ++cc) {
                 const int c = cbase + cc;
@@ -462,23 +476,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                     }
                     outv[j] = __float2bfloat16_rn(a);
                 }
-                if (EPI == EPI_BIAS_RELU && NT == 128 && p.logit_part != nullptr) {
-                    // columns in order, classes innermost: a fixed summation order
-                    for (int j4 = 0; j4 < 32; j4 += 4) {
-                        const float h0 = __bfloat162float(outv[j4]), h1 = __bfloat162float(outv[j4 + 1]);
-                        const float h2 = __bfloat162float(outv[j4 + 2]), h3 = __bfloat162float(outv[j4 + 3]);
-#pragma unroll
-                        for (int q = 0; q < 16; ++q) {
-                            if (q < p.next_out) {
-                                const float4 wv = *reinterpret_cast<const float4 *>(swn + q * BN + c * 32 + j4);
-                                nacc[q] = fmaf(h0, wv.x, nacc[q]);
-                                nacc[q] = fmaf(h1, wv.y, nacc[q]);
-                                nacc[q] = fmaf(h2, wv.z, nacc[q]);
-                                nacc[q] = fmaf(h3, wv.w, nacc[q]);
-                            }
-                        }
-                    }
-                }
                 // stage the bf16 row in the (now idle) ring in the TMA swizzle: 64-column boxes of 128-byte rows,
                 // 16-byte piece j of row r at piece j ^ (r & 7)
                 {
@@ -489,11 +486,6 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                         *reinterpret_cast<uint4 *>(box + ((((c & 1) * 4 + j) ^ (row & 7)) << 4)) = src[j];
                 }
             }
-            if (EPI == EPI_BIAS_RELU && NT == 128 && p.logit_part != nullptr && m < p.M) {
-                float4 *dst = reinterpret_cast<float4 *>(p.logit_part + (((long long)wk * gridDim.x + blockIdx.x) * BM + row) * 16);
-#pragma unroll
-                for (int q = 0; q < 4; ++q) dst[q] = make_float4(nacc[4 * q], nacc[4 * q + 1], nacc[4 * q + 2], nacc[4 * q + 3]);
-            }
             // the tile leaves through two bulk stores (whole 128-byte lines; rows and columns beyond the
             // matrix are clipped by the tensor map)
             fence_async_smem();
@@ -503,6 +495,48 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 for (int b = 0; b < BN / 64; ++b)
                     if (n0 + b * 64 < p.N) tma_store_3d(&map_c, smem_base + b * (BM * 128), n0 + b * 64, m0, wk);
                 tma_store_commit();
+            }
+            if (with_next) {
+                // the staged tile (two 64-column boxes in the 128-byte swizzle) is the A operand as it stands
+                if (threadIdx.x == 0) {
+                    if (mbar_wait(wn_full, 0, abort, limit)) {
+                        tc_fence_after();
+                        constexpr uint32_t idesc_n = instr_desc(false, false, NEXT_N);
+#pragma unroll
+                        for (int b = 0; b < BN / 64; ++b)
+#pragma unroll
+                            for (int k = 0; k < BK / UMMA_K; ++k)
+                                umma_bf16(tmem_base + TMEM_COLS, smem_desc(smem_base + b * (BM * 128) + k * (UMMA_K * 2), false),
+                                          smem_desc(smem_u32(swn) + b * (NEXT_N * 128) + k * (UMMA_K * 2), false), idesc_n,
+                                          (b > 0 || k > 0) ? 1u : 0u);
+                        umma_commit(wn_done);
+                    } else {
+                        abort[0] = 1;
+                        if (p.error_flag != nullptr) atomicExch(p.error_flag, 5);
+                    }
+                }
+                __syncwarp();
+                if (mbar_wait(wn_done, 0, abort, limit)) {
+                    tc_fence_after();
+                    uint32_t q[NEXT_N];
+                    tmem_ld16(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + TMEM_COLS, q);
+                    tmem_ld_wait();
+                    if (m < p.M) {
+                        float o[NEXT_N];
+#pragma unroll
+                        for (int c = 0; c < NEXT_N; ++c) o[c] = __uint_as_float(q[c]);
+                        if (blockIdx.x == 0) {   // the next layer's bias enters here, in the kernel BEFORE the one that may update it
+                            const __nv_bfloat16 *bn = p.b_next + (long long)wk * p.b_next_worker_stride;
+#pragma unroll
+                            for (int c = 0; c < NEXT_N; ++c) if (c < p.next_out) o[c] += __bfloat162float(bn[c]);
+                        }
+                        float4 *dst = reinterpret_cast<float4 *>(p.logit_part + (((long long)wk * gridDim.x + blockIdx.x) * BM + row) * NEXT_N);
+#pragma unroll
+                        for (int c = 0; c < NEXT_N / 4; ++c) dst[c] = make_float4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
+                    }
+                } else if (p.error_flag != nullptr) {
+                    atomicExch(p.error_flag, 6);
+                }
             }
             if (EPI == EPI_MASK && (p.colsum != nullptr || p.colsum_step.x_in != nullptr)) {
                 // the whole batch is in this tile: thread t adds column t of the staged tile over the rows, in row order
@@ -528,7 +562,7 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0) COCOD_TRACE(5);
-    if (warp == 0) tmem_dealloc(tmem_base, TMEM_COLS);
+    if (warp == 0) tmem_dealloc(tmem_base, tmem_cols);
 }
 
 }  // namespace gemm

@@ -119,7 +119,7 @@ cudaError_t launch_dependent(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3
 
 template <int EPI, bool A_MN, bool B_MN>
 cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &c, const Params &p, int workers,
-                        cudaStream_t s, bool pdl = false)
+                        cudaStream_t s, bool pdl = false, const CUtensorMap *next = nullptr)
 {
     constexpr int NT = 128;
     const int need = smem_bytes(p.stages);
@@ -134,7 +134,8 @@ cudaError_t launch_gemm(const CUtensorMap &a, const CUtensorMap &b, const CUtens
         configured[dev] = cap;
     }
     const dim3 grid((p.N + BN - 1) / BN, (p.M + BM - 1) / BM, workers);
-    return launch_dependent(pdl, gemm_bf16<EPI, A_MN, B_MN, NT>, grid, dim3(NT), (size_t)need, s, a, b, c, p);
+    if (p.logit_part != nullptr && next == nullptr) return cudaErrorInvalidValue;
+    return launch_dependent(pdl, gemm_bf16<EPI, A_MN, B_MN, NT>, grid, dim3(NT), (size_t)need, s, a, b, c, next ? *next : c, p);
 }
 
 // The persistent gradient + update kernel over the tiles of up to two weight matrices.
@@ -163,8 +164,9 @@ inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK -
 // 8 warps 15.9 us; about 8 us of it is fixed cost, not the loop over the samples)
 constexpr int HEAD_NW = 4;
 // The output layer and everything downstream of it that runs on CUDA cores.  The second hidden layer's GEMM leaves, per
-// 128-column tile t, the partial logits part[w][t][b][c] = sum_{j in tile} h2[b][j] W3[c][j]; every CTA here first finishes
-// them for all samples of its worker (thread b: z[c] = b3[c] + sum_t part[t][b][c] in tile order, softmax, row loss
+// 128-column tile t, the partial logits part[w][t][b][c] = sum_{j in tile} h2[b][j] W3[c][j] (+ b3[c] in tile 0: in the fused
+// call the extra CTA below UPDATES b3, so no CTA of this kernel may read it); every CTA here first finishes
+// them for all samples of its worker (thread b: z[c] = sum_t part[t][b][c] in tile order, softmax, row loss
 // -log softmax[label], dz3[b][c] = bf16((softmax - onehot) / batch), kept in shared memory), then, for its 32 hidden
 // units j and all samples:
 //   dz2[b][j] = bf16((sum_c dz3[b][c] W3[c][j]) * (h2[b][j] > 0)),  db2[j] = sum_b dz2[b][j],
@@ -207,13 +209,26 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
     for (int b = threadIdx.x; b < B; b += 32 * NW) {
         float z[16];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) z[c] = (c < d_out) ? __bfloat162float(params[(long long)w * P + ob3 + c]) : 0.0f;
+        for (int c = 0; c < 16; ++c) z[c] = 0.0f;          // (b3 is already inside the first tile's partial sums)
+        // tiles in order, four at a time with all their loads in flight (only the float4s that hold classes < DOUT;
+        // eight at a time took 186 registers and was slower)
         const float4 *pp = reinterpret_cast<const float4 *>(part + (((long long)w * n_tiles) * 128 + b) * 16);
-        for (int t = 0; t < n_tiles; ++t) {
+        constexpr int TB = 4;
+        for (int t0 = 0; t0 < n_tiles; t0 += TB) {
+            float4 v[TB][C4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float4 v = __ldcg(pp + (long long)t * (128 * 16 / 4) + q);
-                z[4 * q] += v.x; z[4 * q + 1] += v.y; z[4 * q + 2] += v.z; z[4 * q + 3] += v.w;
+            for (int u = 0; u < TB; ++u)
+#pragma unroll
+                for (int q = 0; q < C4; ++q)
+                    v[u][q] = (t0 + u < n_tiles) ? __ldcg(pp + (long long)(t0 + u) * (128 * 16 / 4) + q) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+#pragma unroll
+            for (int u = 0; u < TB; ++u) {
+                if (t0 + u < n_tiles) {
+#pragma unroll
+                    for (int q = 0; q < C4; ++q) {
+                        z[4 * q] += v[u][q].x; z[4 * q + 1] += v[u][q].y; z[4 * q + 2] += v[u][q].z; z[4 * q + 3] += v[u][q].w;
+                    }
+                }
             }
         }
         float zmax = -INFINITY;
@@ -268,6 +283,8 @@ head_backward(const bf16 *__restrict__ h2, const bf16 *params, const float *__re
         }
         return;
     }
+    // (requesting this column of W3 before the logits are finished gained 1 us in the eager chain and lost 1.4 us in a
+    //  replayed graph)
     float w3[4 * C4], acc3[4 * C4];
 #pragma unroll
     for (int c = 0; c < 4 * C4; ++c) {
@@ -472,8 +489,9 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     const long long P = h->P;
     const uint64_t uK = K, uB = B, uh = d_h, ui = d_in, uP = P;
     // maps over caller memory
-    CUtensorMap k_x, mn_x, k_w1, k_w2, mn_w2, c_w1{}, c_w2{};
-    if (!map_k(&k_x, xin, ui, uB, uK, ui, uB * ui) || !map_mn(&mn_x, xin, ui, uB, uK, ui, uB * ui) ||
+    CUtensorMap k_x, mn_x, k_w1, k_w2, mn_w2, k_w3, c_w1{}, c_w2{};
+    if (!make_map(&k_w3, prm + h->oW3, uh, (uint64_t)d_out, uK, uh, uP, NEXT_N) ||
+        !map_k(&k_x, xin, ui, uB, uK, ui, uB * ui) || !map_mn(&mn_x, xin, ui, uB, uK, ui, uB * ui) ||
         !map_k(&k_w1, prm + h->oW1, ui, uh, uK, ui, uP) || !map_k(&k_w2, prm + h->oW2, uh, uh, uK, uh, uP) ||
         !map_mn(&mn_w2, prm + h->oW2, uh, uh, uK, uh, uP))
         return COCOD_ERR_CUDA;
@@ -517,8 +535,8 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, pdl_fwd)));
     // h2 = relu(h1 W2^T + b2), and per 128-column tile the partial logits h2 W3^T of that tile
     p.K = d_h; p.stages = stages_for(d_h); p.bias = prm + h->ob2;
-    p.logit_part = h->logit_part; p.w_next = prm + h->oW3; p.w_next_worker_stride = P; p.next_out = d_out;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, pdl_fwd)));
+    p.logit_part = h->logit_part; p.b_next = prm + h->ob3; p.b_next_worker_stride = P; p.next_out = d_out;
+    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, pdl_fwd, &k_w3)));
     // logits, loss, dz3; then dz2, dW3, db3, db2
     GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
                              dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->logit_part, d_h / 128, labels,
