@@ -55,6 +55,8 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--repeats", type=int, default=5, help="how many times the timed block of --steps rounds is repeated "
                                                            "(the line reports the median block, and min and max)")
+    ap.add_argument("--alternate-sweep", action="store_true",
+                    help="experiment: consecutive streaming kernels walk the vector in alternating directions (COCOD_OPT_SWEEP)")
     ap.add_argument("--no-other-workloads", action="store_true",
                     help="default run only: skip the VGG16-sized and MLP digests added under other_workloads")
     ap.add_argument("--cpu-sample-cols", type=int, default=1 << 20)
@@ -219,6 +221,8 @@ def measure_param_workload(args, wl, ctx, *, ring_n, do_e2e, cpu_seconds, do_gra
 
     eng = E.Engine(K, P, wl.lr, wl.mu, wl.wd)
     eng.set_option(E.OPT_SNAPSHOT, E.SNAPSHOT_FLIP if args.snapshot == "flip" else E.SNAPSHOT_COPY)
+    if args.alternate_sweep:
+        eng.set_option(E.OPT_SWEEP, 1)
     x0 = torch.empty(P, dtype=torch.float32, device="cuda")
     I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, p0, wl.sigma_x0)
     eng.set_params(x0)
@@ -474,7 +478,7 @@ def measure_param_workload(args, wl, ctx, *, ring_n, do_e2e, cpu_seconds, do_gra
                          "ms_per_step_min": min(block_ms) / steps, "ms_per_step_max": max(block_ms) / steps,
                          "reported": "median block"},
         "config": {"workload": wl.name, "K": K, "P": P, "k": k, "lr": wl.lr, "mu": wl.mu, "wd": wl.wd,
-                   "snapshot": args.snapshot, "gradient_ring": max(1, ring_n),
+                   "snapshot": args.snapshot, "alternate_sweep": bool(args.alternate_sweep), "gradient_ring": max(1, ring_n),
                    "cuda_graph": bool(graph is not None),
                    "l2": "inputs larger than L2 (each K x P buffer is %.0f MB, L2 is 126 MB)" % (K * P * 4 / 1e6)
                          if K * P * 4 > 126e6 else "L2-resident workload: not an HBM number",

@@ -678,3 +678,49 @@ def test_a_request_beyond_the_device_memory_fails_cleanly(E):
     eng.local_step(torch.ones(2, 1024, device="cuda"))
     assert np.allclose(cpu(eng.get_params()), 0.9)
     eng.destroy()
+
+
+# ----------------------------------------------------------------------------- measurement options change no value
+@pytest.mark.parametrize("K,P,shadow", [(16, 200_000, False), (5, 100_008, True), (3, 1001, False)])
+def test_alternating_sweep_and_device_time_stamps_change_no_value(E, K, P, shadow):
+    """COCOD_OPT_SWEEP lets consecutive kernels walk the vector in alternating directions, COCOD_OPT_PROFILE lets
+    them stamp their start and end on the GPU's clock: the models, momenta, averages (and bf16 copies) must equal
+    the plain run bit for bit, and the stamps must be ordered and cover every recorded kernel that takes them."""
+    k, rounds = 3, 3
+    x0 = I.initial_point(P)
+    side = torch.cuda.Stream(priority=-1)
+    engines = [E.Engine(K, P, 0.1, 0.9, 5e-4) for _ in range(2)]
+    for eng in engines:
+        if shadow:
+            eng.set_option(E.OPT_BF16_SHADOW, 1)
+        eng.set_params(x0)
+    engines[1].set_option(E.OPT_SWEEP, 1)
+    engines[1].set_option(E.OPT_PROFILE, 1)
+    engines[1].profile_reset()
+    for r in range(rounds):
+        for eng in engines:
+            eng.comm_begin(side)
+        for s in range(k):
+            g = torch.from_numpy(I.gradients(K, P, r * k + s)).cuda()
+            for eng in engines:
+                eng.local_step(g)
+        for eng in engines:
+            eng.comm_end()
+    a, b = engines
+    assert_bit_equal(cpu(b.get_params()), cpu(a.get_params()), "x")
+    assert_bit_equal(cpu(b.get_momentum()), cpu(a.get_momentum()), "v")
+    assert_bit_equal(cpu(b.get_mean()), cpu(a.get_mean()), "average")
+    if shadow:
+        assert torch.equal(a.bf16_shadow().view(torch.int16), b.bf16_shadow().view(torch.int16))
+    events = b.profile_records()
+    stamps = b.profile_device_records()
+    assert len(events) == rounds * (k + 2)
+    if P % 4 == 0:                                   # the vectorised kernels take stamps, the scalar fall-backs do not
+        assert len(stamps) == len(events)
+        for kind, t0, t1 in stamps:
+            assert 0.0 <= t0 < t1 < 1e4
+        # stream order on the compute stream: every local step / merge starts after its predecessor started
+        comp = [(t0, t1) for kind, t0, t1 in stamps if E.KERNEL_NAMES[kind] != "mean"]
+        assert all(comp[i][0] <= comp[i + 1][0] for i in range(len(comp) - 1))
+    else:                                            # the flat local step still has a vectorised body; mean and merge do not
+        assert len(stamps) == rounds * k and all(E.KERNEL_NAMES[kind] == "local_step" for kind, _, _ in stamps)
