@@ -18,6 +18,14 @@
 //
 // so that the loads of tile t + 1 run under the update and the store drain of tile t.  All waits are
 // bounded (the kernel reports a timeout through error_flag, lets issued copies land, frees TMEM, returns).
+//
+// Every x / v chunk buffer and its two barriers belong to ONE update group for the whole kernel.  That matters: an
+// mbarrier wait knows only the parity of the phase it waits for, so a waiter that could get two uses ahead of a
+// barrier would pass at once on stale data.  (A variant with the operands in a single stage and a ring of five
+// chunk slots handed from group to group -- one more chunk of x and v in flight per SM -- had exactly that fault
+// until each slot got three "landed" barriers used in turn; it was then correct and 3 us per step SLOWER, because
+// the tensor-core thread had to fetch its two operand blocks one after the other: bytes in flight are not what
+// bounds this kernel.)
 #pragma once
 #include "cocod_gemm_sm100.cuh"
 

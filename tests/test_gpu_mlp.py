@@ -417,6 +417,60 @@ def test_fused_gradient_and_update_is_bit_identical_to_the_two_calls(M, E, K, di
     assert e.value.code == E.ERR_STATE
 
 
+def test_fused_and_two_call_paths_stay_identical_over_long_uninterrupted_runs(M, E):
+    """600 local steps (150 rounds) queued back to back without the host ever waiting, twice through the fused call and
+    once through the two calls, all from the same state on the same minibatches: x, v and the bf16 copy must agree bit
+    for bit after every 50 rounds.  (A step-by-step comparison synchronises after every call and cannot see a hazard
+    that needs kernels of consecutive steps, or the roles inside the persistent kernel, to run far ahead of one
+    another; a hand-shake that is wrong once in a thousand steps shows up here.)"""
+    K, k, rounds, dims = 16, 4, 150, I.MLP_DIMS
+    mg = M.MLPGrad(K, 128, dims[0], dims[1], dims[3])
+    P, P_raw = mg.P, mg.P_raw
+    x0 = np.zeros(P, np.float32)
+    x0[:P_raw] = I.mlp_init_params(I.MLP_STUDENT_SEED)
+    n_pool = 64
+    pool = torch.empty((n_pool, K, 128, dims[0]), dtype=torch.bfloat16, device="cuda")
+    I.device_mlp_batches_into(pool, 0)
+    labels = I.device_mlp_teacher_labels(pool, I.mlp_init_params(I.MLP_TEACHER_SEED))
+    np.testing.assert_array_equal(cpu(pool[3, 5].float()), I.mlp_batch(5, 3))      # device generator == host recipe
+    side = torch.cuda.Stream(priority=-1)
+    grads = torch.empty((K, P), dtype=torch.float32, device="cuda")
+    loss = torch.empty(K, dtype=torch.float32, device="cuda")
+
+    def run(fused):
+        eng = E.Engine(K, P, 0.05, 0.9, 0.0)
+        eng.set_option(E.OPT_BF16_SHADOW, 1)
+        eng.set_params(x0)
+        marks = []
+        for r in range(rounds):
+            eng.comm_begin(side)
+            for s in range(k):
+                t = (r * k + s) % n_pool
+                if fused:
+                    mg.grad_step(eng, pool[t], labels[t], loss)
+                else:
+                    mg.grad(eng.bf16_shadow(), pool[t], labels[t], grads, loss)
+                    eng.local_step(grads)
+            eng.comm_end()
+            if (r + 1) % 50 == 0:                      # stream-ordered copies: the host still does not wait
+                marks.append((eng.get_params().clone(), eng.get_momentum().clone(), eng.bf16_shadow().clone()))
+        torch.cuda.synchronize()
+        mg.check()
+        eng.destroy()
+        return marks
+
+    want = run(False)
+    for trial in range(2):
+        got = run(True)
+        for i, ((xa, va, sa), (xb, vb, sb)) in enumerate(zip(want, got)):
+            what = f"trial {trial}, after {50 * (i + 1)} rounds"
+            assert torch.equal(xa.view(torch.int32), xb.view(torch.int32)), "x, " + what
+            assert torch.equal(va.view(torch.int32), vb.view(torch.int32)), "v, " + what
+            assert torch.equal(sa.view(torch.int16), sb.view(torch.int16)), "bf16 copy, " + what
+    again = run(False)
+    assert all(torch.equal(a[0].view(torch.int32), b[0].view(torch.int32)) for a, b in zip(want, again)), "two calls, rerun"
+
+
 @pytest.mark.parametrize("K,dims,wd", [(3, (200, 256, 256, 7), 5e-4), (16, I.MLP_DIMS, 0.0)])
 def test_fused_gradient_and_update_matches_the_oracle(M, E, K, dims, wd):
     """cocod_mlp_grad_step held to the ORACLE directly (not to the two-call device path): both sides start from the
