@@ -81,10 +81,16 @@ int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x
  * ordinary, not a programmatic, dependent, so that the events bracket it alone).  At most 4096 calls are recorded.
  * Setting the option (to either value) synchronises the device and discards the records.
  * cocod_mlp_profile_get synchronises the device and returns the number of recorded calls and the average
- * milliseconds of the pass and of the update kernel (0 when no call recorded one). */
+ * milliseconds of the pass and of the update kernel (0 when no call recorded one).
+ * COCOD_MLP_OPT_PROFILE = 2: no events and no change to how anything is launched; the update kernel alone stamps the
+ * earliest start (after its wait for the predecessor) and the latest end of its thread blocks on the GPU's own clock,
+ * so that its duration INSIDE the chain, with the programmatic overlap at both ends, can be read
+ * (cocod_mlp_profile_get_device: number of stamped launches and their average milliseconds; also filled with
+ * value 1).  The first non-zero setting allocates 64 KB on the device. */
 enum { COCOD_MLP_OPT_PROFILE = 1 };
 int cocod_mlp_set_option(cocod_mlp_handle *h, int option, int value);
 int cocod_mlp_profile_get(cocod_mlp_handle *h, int *calls, float *pass_ms, float *update_ms);
+int cocod_mlp_profile_get_device(cocod_mlp_handle *h, int *calls, float *update_ms);
 
 /* Synchronise `stream` and report whether any kernel of this handle gave up a wait. */
 int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream);

@@ -47,6 +47,8 @@ struct UpdateParams {
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
     int debug_no_loads;                // self-test: the producer issues nothing, so the waits run out
+    unsigned long long *stamp;         // measurement (nullptr = off): [0] earliest start, [1] latest end of the CTAs, in ns
+                                       // of the GPU's clock, taken after the wait for the predecessor and at the very end
 };
 
 constexpr int UPD_THREADS = 320;       // producer warp, MMA warp, 8 update warps
@@ -112,6 +114,7 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
     const uint32_t tmem_base = *tmem_slot;
     pdl_launch_dependents();
     pdl_wait();
+    if (q.stamp != nullptr && threadIdx.x == 0) atomicMin(q.stamp, now_ns());
 
     // tile t of the whole list -> problem, worker, tile origin
     auto decode = [&](int t, const UpdateProblem *&P, int &wk, int &m0, int &n0) {
@@ -267,6 +270,7 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, 2 * TMEM_COLS);
+    if (q.stamp != nullptr && threadIdx.x == 0) atomicMax(q.stamp + 1, now_ns());
 }
 
 }  // namespace gemm

@@ -368,14 +368,24 @@ struct cocod_mlp {
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // COCOD_MLP_OPT_PROFILE: CUDA events around every gradient pass and around its gradient + update kernel
-    bool profile = false;
+    int profile = 0;                    // 0 off, 1 events (+ stamps), 2 stamps only
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_pass, prof_update;
+    unsigned long long *stamps = nullptr;     // device: kMaxStamps x {earliest start, latest end} of the update kernel's CTAs
+    int n_stamps = 0;
 };
 
 namespace {
 
+constexpr int kMaxStamps = 4096;
+
 void mlp_profile_clear(cocod_mlp *h)
 {
+    h->n_stamps = 0;
+    if (h->stamps) {                   // start = all ones (atomicMin), end = 0 (atomicMax); the device is idle here
+        std::vector<unsigned long long> init(2 * (size_t)kMaxStamps);
+        for (size_t i = 0; i < init.size(); i += 2) { init[i] = ~0ull; init[i + 1] = 0ull; }
+        cudaMemcpy(h->stamps, init.data(), init.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice);
+    }
     for (auto *list : {&h->prof_pass, &h->prof_update}) {
         for (auto &pr : *list) {
             cudaEventDestroy(pr.first);
@@ -388,7 +398,7 @@ void mlp_profile_clear(cocod_mlp *h)
 // An event pair whose first event is recorded now; the caller records the second one.
 bool mlp_profile_open(cocod_mlp *h, std::vector<std::pair<cudaEvent_t, cudaEvent_t>> &list, cudaStream_t s)
 {
-    if (!h->profile || list.size() >= 4096) return false;
+    if (h->profile != 1 || list.size() >= 4096) return false;
     cudaEvent_t a = nullptr, b = nullptr;
     if (cudaEventCreate(&a) != cudaSuccess) { cudaGetLastError(); return false; }
     if (cudaEventCreate(&b) != cudaSuccess) { cudaGetLastError(); cudaEventDestroy(a); return false; }
@@ -400,7 +410,7 @@ bool mlp_profile_open(cocod_mlp *h, std::vector<std::pair<cudaEvent_t, cudaEvent
 void mlp_free(cocod_mlp *h)
 {
     mlp_profile_clear(h);
-    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->logit_part, h->error_flag};
+    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->logit_part, h->error_flag, h->stamps};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (h->ev_fork) cudaEventDestroy(h->ev_fork);
     if (h->ev_join) cudaEventDestroy(h->ev_join);
@@ -581,6 +591,8 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
             UpdateParams uq{};
             uq.K = B; uq.lr = fused->lr; uq.mu = fused->mu; uq.wd = fused->wd; uq.error_flag = h->error_flag;
             const bool prof_upd = (capturing == cudaStreamCaptureStatusNone) && mlp_profile_open(h, h->prof_update, s);
+            if (h->profile != 0 && h->stamps && capturing == cudaStreamCaptureStatusNone && h->n_stamps < kMaxStamps)
+                uq.stamp = h->stamps + 2 * (size_t)(h->n_stamps++);
             GEMM_OK(launch_update(u2, u1, uq, s, pdl && !prof_upd));
             if (prof_upd) cudaEventRecord(h->prof_update.back().second, s);
         }
@@ -662,9 +674,16 @@ int cocod_mlp_set_option(cocod_mlp_handle *h, int option, int value)
 {
     if (!h) return COCOD_ERR_INVALID;
     if (option != COCOD_MLP_OPT_PROFILE) return COCOD_ERR_INVALID;
+    if (value < 0 || value > 2) return COCOD_ERR_INVALID;
     if (cudaDeviceSynchronize() != cudaSuccess) return COCOD_ERR_CUDA;
+    if (value != 0 && !h->stamps &&
+        cudaMalloc((void **)&h->stamps, 2 * (size_t)kMaxStamps * sizeof(unsigned long long)) != cudaSuccess) {
+        cudaGetLastError();
+        h->stamps = nullptr;
+        return COCOD_ERR_OOM;
+    }
     mlp_profile_clear(h);
-    h->profile = value != 0;
+    h->profile = value;
     return COCOD_OK;
 }
 
@@ -684,6 +703,27 @@ int cocod_mlp_profile_get(cocod_mlp_handle *h, int *calls, float *pass_ms, float
     };
     if (!average(h->prof_pass, pass_ms) || !average(h->prof_update, update_ms)) { cudaGetLastError(); return COCOD_ERR_CUDA; }
     *calls = (int)h->prof_pass.size();
+    return COCOD_OK;
+}
+
+int cocod_mlp_profile_get_device(cocod_mlp_handle *h, int *calls, float *update_ms)
+{
+    if (!h || !calls || !update_ms) return COCOD_ERR_INVALID;
+    if (cudaDeviceSynchronize() != cudaSuccess) return COCOD_ERR_CUDA;
+    *calls = 0;
+    *update_ms = 0.0f;
+    if (!h->stamps || h->n_stamps == 0) return COCOD_OK;
+    std::vector<unsigned long long> st(2 * (size_t)h->n_stamps);
+    if (cudaMemcpy(st.data(), h->stamps, st.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return COCOD_ERR_CUDA;
+    }
+    double sum = 0.0;
+    int n = 0;
+    for (int i = 0; i < h->n_stamps; ++i)
+        if (st[2 * i] != ~0ull && st[2 * i + 1] > st[2 * i]) { sum += (double)(st[2 * i + 1] - st[2 * i]); ++n; }
+    *calls = n;
+    *update_ms = n ? (float)(sum / n * 1e-6) : 0.0f;
     return COCOD_OK;
 }
 

@@ -21,6 +21,7 @@ SIGNATURES = {
     "cocod_mlp_check": (_i, [_vp, _vp]),
     "cocod_mlp_set_option": (_i, [_vp, _i, _i]),
     "cocod_mlp_profile_get": (_i, [_vp, ctypes.POINTER(_i), ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]),
+    "cocod_mlp_profile_get_device": (_i, [_vp, ctypes.POINTER(_i), ctypes.POINTER(ctypes.c_float)]),
     "cocod_mlp_launch_count": (_i64, [_vp]),
     "cocod_gemm_wait_selftest": (_i, [_i, _vp]),
     "cocod_gemm_update_wait_selftest": (_i, [_i, _vp]),
@@ -98,8 +99,10 @@ class MLPGrad:
         if rc != _E.OK:
             raise _E.CocodError(rc, "cocod_mlp_check")
 
-    def set_profile(self, on: bool):
-        rc = self._lib.cocod_mlp_set_option(self._h, OPT_PROFILE, int(bool(on)))
+    def set_profile(self, on):
+        """0 / False: off; 1 / True: CUDA events around each pass and the update kernel; 2: the update kernel's own
+        time stamps only (nothing about the launches changes)."""
+        rc = self._lib.cocod_mlp_set_option(self._h, OPT_PROFILE, int(on))
         if rc != _E.OK:
             raise _E.CocodError(rc, "cocod_mlp_set_option")
 
@@ -110,6 +113,14 @@ class MLPGrad:
         if rc != _E.OK:
             raise _E.CocodError(rc, "cocod_mlp_profile_get")
         return n.value, a.value, b.value
+
+    def profile_device(self):
+        """(stamped launches of the gradient + update kernel, their average ms by the kernel's own stamps)."""
+        n, a = _i(), ctypes.c_float()
+        rc = self._lib.cocod_mlp_profile_get_device(self._h, ctypes.byref(n), ctypes.byref(a))
+        if rc != _E.OK:
+            raise _E.CocodError(rc, "cocod_mlp_profile_get_device")
+        return n.value, a.value
 
     @property
     def launch_count(self) -> int:

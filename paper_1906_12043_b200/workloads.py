@@ -57,3 +57,8 @@ def bytes_merge(K: int) -> float:
 # `ncu --set full` capture of these three kernels on a small case (K=16, P=4,194,304); pure
 # streaming, so it scales with K*P.
 NCU_DRAM_BYTES_PER_WORKER_PARAM = {"local_step": 19.25, "mean": 4.12, "merge": 11.81}
+
+# The same for one launch of the persistent gradient + update kernel of the end-to-end MLP workload (K = 16 workers,
+# 784-1024-1024-10): dram__bytes_read.sum + dram__bytes_write.sum of one `ncu --set full` capture, in bytes.  (Below the
+# 533 MB it moves algorithmically because the tail of its output is still in L2 when it ends.)
+NCU_DRAM_BYTES_MLP_UPDATE_KERNEL_K16 = 252.9e6 + 242.0e6
