@@ -77,8 +77,9 @@ int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x
 
 /* Measurement.  COCOD_MLP_OPT_PROFILE = 1: every later call of cocod_mlp_grad / cocod_mlp_grad_step that is not
  * being captured into a CUDA graph records a CUDA-event pair around the whole pass (first kernel to last) and, for
- * cocod_mlp_grad_step, a second pair around its persistent gradient + update kernel (which is then launched as an
- * ordinary, not a programmatic, dependent, so that the events bracket it alone).  At most 4096 calls are recorded.
+ * both calls, a second pair around the persistent kernel that forms the weight gradients of W1 and W2 (and, in
+ * cocod_mlp_grad_step, updates them; it is then launched as an ordinary, not a programmatic, dependent, so that the
+ * events bracket it alone).  At most 4096 calls are recorded.
  * Setting the option (to either value) synchronises the device and discards the records.
  * cocod_mlp_profile_get synchronises the device and returns the number of recorded calls and the average
  * milliseconds of the pass and of the update kernel (0 when no call recorded one).

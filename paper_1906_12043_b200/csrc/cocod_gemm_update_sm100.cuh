@@ -16,7 +16,9 @@
 //   warps 2..9          update: TMEM -> registers, x and v updated in place in shared memory (TMA swizzle),
 //                       bulk stores chunk by chunk (x, v and the staged bf16 copy of x)
 //
-// so that the loads of tile t + 1 run under the update and the store drain of tile t.  All waits are
+// so that the loads of tile t + 1 run under the update and the store drain of tile t.  The same kernel also serves the
+// gradient call that writes the weight gradients out (store_only): the update warps then stage the product itself, in
+// the x / v buffers alternately from tile to tile, and store it through x_out.  All waits are
 // bounded (the kernel reports a timeout through error_flag, lets issued copies land, frees TMEM, returns).
 //
 // Every x / v chunk buffer and its two barriers belong to ONE update group for the whole kernel.  That matters: an
@@ -47,6 +49,8 @@ struct UpdateParams {
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
     int debug_no_loads;                // self-test: the producer issues nothing, so the waits run out
+    int store_only;                    // 1: no update -- the product itself (the weight gradient) is written through x_out;
+                                       //    x_in, v and shadow of the problems are unused, nothing but the operands is loaded
     unsigned long long *stamp;         // measurement (nullptr = off): [0] earliest start, [1] latest end of the CTAs, in ns
                                        // of the GPU's clock, taken after the wait for the predecessor and at the very end
 };
@@ -146,7 +150,7 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
             }
             if (failed) break;
             issued_ops = i + 1;
-            for (int cq = 0; cq < 4; ++cq) {
+            for (int cq = 0; cq < 4 && !q.store_only; ++cq) {
                 const int c = ((cq & 1) << 1) | (cq >> 1);      // 0, 2, 1, 3: each group's first chunk first
                 if (i > 0 && !mbar_wait(xve0 + 8 * c, (i - 1) & 1, abort, limit)) { failed = 1; break; }
                 const uint32_t bar = xvf0 + 8 * c;
@@ -202,6 +206,10 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
             uint2 held[8];            // bf16 copy of the first chunk: staged together with the second one (see below)
+            // store_only: tile i stages in the x buffers, tile i + 1 in the v buffers.  A thread that writes tile i + 1 has
+            // passed the named barriers of tile i, which the leader joined only after the stores of tile i - 1 (the last
+            // user of the same buffers) had read them (its wait at the end of tile i - 1, below).
+            uint8_t *xb = (q.store_only && (i & 1)) ? vs : xs;
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
                 const int c = group * 2 + cc;
@@ -215,9 +223,16 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
                     __syncwarp();
                     if (lane == 0) mbar_arrive(acce0 + 8 * a);
                 }
-                ok = ok && mbar_wait(xvf0 + 8 * c, i & 1, abort, limit);      // this chunk's x and v
-                ok = __all_sync(0xffffffffu, ok);
-                if (ok) {
+                if (!q.store_only) {
+                    ok = ok && mbar_wait(xvf0 + 8 * c, i & 1, abort, limit);      // this chunk's x and v
+                    ok = __all_sync(0xffffffffu, ok);
+                }
+                if (ok && q.store_only) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4 *>(xb + c * (BM * 128) + row * 128 + ((j ^ (row & 7)) << 4)) =
+                            make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                } else if (ok) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int off = c * (BM * 128) + row * 128 + ((j ^ (row & 7)) << 4);
@@ -245,26 +260,31 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
                 asm volatile("bar.sync %0, 128;" ::"r"(group + 1) : "memory");
                 if (leader) {
                     if (ok && n0 + c * 32 < P->N) {
-                        tma_store_3d(&P->x_out, smem_u32(xs) + c * (BM * 128), n0 + c * 32, m0, wk);
-                        tma_store_3d(&P->v, smem_u32(vs) + c * (BM * 128), n0 + c * 32, m0, wk);
+                        tma_store_3d(&P->x_out, smem_u32(xb) + c * (BM * 128), n0 + c * 32, m0, wk);
+                        if (!q.store_only) tma_store_3d(&P->v, smem_u32(vs) + c * (BM * 128), n0 + c * 32, m0, wk);
                     }
                     // the group's 64-column box of the bf16 copy is complete after its second chunk
-                    if (ok && cc == 1 && P->has_shadow && n0 + group * 64 < P->N)
+                    if (ok && cc == 1 && !q.store_only && P->has_shadow && n0 + group * 64 < P->N)
                         tma_store_3d(&P->shadow, smem_u32(ss) + group * (BM * 128), n0 + group * 64, m0, wk);
                     tma_store_commit();
                 }
             }
-            if (leader) {             // a chunk's buffers go back to the producer once its stores have read them
-                tma_store_wait_read<1>();
-                mbar_arrive(xve0 + 8 * (group * 2));
-                tma_store_wait_read<0>();
-                mbar_arrive(xve0 + 8 * (group * 2 + 1));
+            if (leader) {
+                if (q.store_only) {
+                    tma_store_wait_read<0>();
+                } else {              // a chunk's buffers go back to the producer once its stores have read them
+                    tma_store_wait_read<1>();
+                    mbar_arrive(xve0 + 8 * (group * 2));
+                    tma_store_wait_read<0>();
+                    mbar_arrive(xve0 + 8 * (group * 2 + 1));
+                }
             }
             if (!ok && !failed) {
                 failed = 3;
                 abort[0] = 1;
             }
         }
+        if (leader) tma_store_wait_read<0>();      // shared memory must outlive the reads of the last stores
     }
     if (failed && q.error_flag != nullptr) atomicExch(q.error_flag, 10 + failed);
     tc_fence_before();

@@ -12,8 +12,9 @@
 //   dz2 = bf16((dz3 W3) * (h2 > 0)) ; dW3 = dz3^T h2 ; db3, db2 = column sums           CUDA cores
 //   dz1 = bf16((dz2 W2) * (h1 > 0))   GEMM 128 x d_h x d_h    A = dz2, B = W2 read [k][n]  epilogue mask,
 //   db1 = column sums of dz1                                   (same epilogue: the batch is one tile)
-//   dW2 = dz2^T h1                    GEMM d_h x d_h x 128    A = dz2 read [k][m], B = h1 read [k][n]   fp32 out
-//   dW1 = dz1^T x                     GEMM d_h x d_in x 128   A = dz1 read [k][m], B = x  read [k][n]   fp32 out
+//   dW2 = dz2^T h1                    GEMM d_h x d_h x 128    A = dz2 read [k][m], B = h1 read [k][n]   one persistent kernel over
+//   dW1 = dz1^T x                     GEMM d_h x d_in x 128   A = dz1 read [k][m], B = x  read [k][n]   the tiles of both: fp32
+//                                                                                      out, or the local step applied in place
 #include "cocod_mlp.h"
 #include "cocod_gemm_sm100.cuh"
 #include "cocod_gemm_update_sm100.cuh"
@@ -363,10 +364,6 @@ struct cocod_mlp {
     CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
     CUtensorMap st_h2, st_dz1;          // store views (64 columns x 128 rows) of outputs that are not read that way
     long long launches = 0;
-    // second branch of the backward pass (dW2 beside dz1 -> dW1): a stream of the handle's own, forked from and
-    // joined to the caller's stream by events
-    cudaStream_t side = nullptr;
-    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // COCOD_MLP_OPT_PROFILE: CUDA events around every gradient pass and around its gradient + update kernel
     int profile = 0;                    // 0 off, 1 events (+ stamps), 2 stamps only
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_pass, prof_update;
@@ -412,9 +409,6 @@ void mlp_free(cocod_mlp *h)
     mlp_profile_clear(h);
     void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->logit_part, h->error_flag, h->stamps};
     for (void *p : ptrs) if (p) cudaFree(p);
-    if (h->ev_fork) cudaEventDestroy(h->ev_fork);
-    if (h->ev_join) cudaEventDestroy(h->ev_join);
-    if (h->side) cudaStreamDestroy(h->side);
     delete h;
 }
 
@@ -449,9 +443,6 @@ int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_h
     alloc((void **)&h->logit_part, (size_t)K * (d_hidden / 128) * 128 * 16 * sizeof(float));
     alloc((void **)&h->error_flag, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->error_flag, 0, sizeof(int));
-    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming);
     if (e != cudaSuccess) {
         cudaGetLastError();
         mlp_free(h);
@@ -488,10 +479,10 @@ int64_t cocod_mlp_launch_count(const cocod_mlp_handle *h) { return h ? h->launch
 
 namespace {
 
-// The whole gradient pass.  With fused == nullptr the weight gradients dW1, dW2 are written to `grads`;
-// otherwise one persistent kernel (gemm_update_persistent: the tiles of W2, then of W1, two accumulators in
-// tensor memory) forms them and applies the engine's local step tile by tile (x, v and the bf16 copy of x are
-// updated in place, nothing is written to `grads`).
+// The whole gradient pass.  One persistent kernel (gemm_update_persistent: the tiles of W2, then of W1, two
+// accumulators in tensor memory) forms the weight gradients dW1, dW2: with fused == nullptr it writes them to
+// `grads`; otherwise it applies the engine's local step tile by tile (x, v and the bf16 copy of x are updated in
+// place, nothing is written to `grads`).
 int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labels, float *grads, float *loss,
              cudaStream_t s, const cocod_step_plan *fused)
 {
@@ -564,57 +555,35 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
         q.colsum_step.x_in += h->ob1; q.colsum_step.x_out += h->ob1; q.colsum_step.v += h->ob1;
         if (q.colsum_step.shadow) q.colsum_step.shadow += h->ob1;
     }
-    // dW2 = dz2^T h1, dW1 = dz1^T x: both operands read with their row index contiguous
-    Params r{};
-    r.error_flag = h->error_flag;
-    r.M = d_h; r.N = d_h; r.K = B; r.stages = stages_for(B);
-    // Replayed from a CUDA graph, the backward pass of the gradient call runs as two branches (the handle's own stream, forked from and
-    // joined to the caller's stream by events): measured 89.1 -> 82.8 us for the chain of the gradient call.
-    // Queued eagerly the same fork costs more in event calls than it gains (93.0 -> 94.2 us), so it is used under
-    // stream capture only.
-    const bool fork = (capturing != cudaStreamCaptureStatusNone);
-    if (fused) {
-        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, pdl)));
-        {
-            // one persistent kernel walks the tiles of W2 and then of W1 (loads of a tile under the update and the
-            // store drain of the tile before it); the batch of 128 is its whole reduction (two operand blocks)
-            static_assert(2 * BK == 128, "the update kernel holds the whole reduction in its two-stage ring");
-            UpdateProblem u2{}, u1{};
-            u2.a = h->mn_dz2; u2.b = h->mn_h1; u2.x_in = s_w2.x_in; u2.x_out = s_w2.x_out; u2.v = s_w2.v;
-            u2.shadow = s_w2.shadow; u2.has_shadow = fused->shadow != nullptr;
-            u2.M = d_h; u2.N = d_h; u2.tiles_m = (d_h + BM - 1) / BM; u2.tiles_n = (d_h + BN - 1) / BN;
-            u2.tiles = K * u2.tiles_m * u2.tiles_n;
-            u1.a = h->mn_dz1; u1.b = mn_x; u1.x_in = s_w1.x_in; u1.x_out = s_w1.x_out; u1.v = s_w1.v;
-            u1.shadow = s_w1.shadow; u1.has_shadow = fused->shadow != nullptr;
-            u1.M = d_h; u1.N = d_in; u1.tiles_m = (d_h + BM - 1) / BM; u1.tiles_n = (d_in + BN - 1) / BN;
-            u1.tiles = K * u1.tiles_m * u1.tiles_n;
-            UpdateParams uq{};
-            uq.K = B; uq.lr = fused->lr; uq.mu = fused->mu; uq.wd = fused->wd; uq.error_flag = h->error_flag;
-            const bool prof_upd = (capturing == cudaStreamCaptureStatusNone) && mlp_profile_open(h, h->prof_update, s);
-            if (h->profile != 0 && h->stamps && capturing == cudaStreamCaptureStatusNone && h->n_stamps < kMaxStamps)
-                uq.stamp = h->stamps + 2 * (size_t)(h->n_stamps++);
-            GEMM_OK(launch_update(u2, u1, uq, s, pdl && !prof_upd));
-            if (prof_upd) cudaEventRecord(h->prof_update.back().second, s);
+    // One persistent kernel walks the tiles of W2 and then of W1 (the batch of 128 is its whole reduction: two operand
+    // blocks): in the fused call it applies the local step to each tile as soon as its product is formed, in the gradient
+    // call it writes the product out.
+    static_assert(2 * BK == 128, "the update kernel holds the whole reduction in its two-stage ring");
+    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, pdl)));
+    {
+        UpdateProblem u2{}, u1{};
+        u2.a = h->mn_dz2; u2.b = h->mn_h1;
+        u2.M = d_h; u2.N = d_h; u2.tiles_m = (d_h + BM - 1) / BM; u2.tiles_n = (d_h + BN - 1) / BN;
+        u2.tiles = K * u2.tiles_m * u2.tiles_n;
+        u1.a = h->mn_dz1; u1.b = mn_x;
+        u1.M = d_h; u1.N = d_in; u1.tiles_m = (d_h + BM - 1) / BM; u1.tiles_n = (d_in + BN - 1) / BN;
+        u1.tiles = K * u1.tiles_m * u1.tiles_n;
+        UpdateParams uq{};
+        uq.K = B; uq.error_flag = h->error_flag;
+        if (fused) {
+            u2.x_in = s_w2.x_in; u2.x_out = s_w2.x_out; u2.v = s_w2.v; u2.shadow = s_w2.shadow; u2.has_shadow = fused->shadow != nullptr;
+            u1.x_in = s_w1.x_in; u1.x_out = s_w1.x_out; u1.v = s_w1.v; u1.shadow = s_w1.shadow; u1.has_shadow = fused->shadow != nullptr;
+            uq.lr = fused->lr; uq.mu = fused->mu; uq.wd = fused->wd;
+        } else {                      // the gradient tensors take the place of x_out; nothing else is touched
+            u2.x_out = c_w2; u1.x_out = c_w1;
+            u2.x_in = u2.v = c_w2; u1.x_in = u1.v = c_w1;      // (valid maps; never used)
+            uq.store_only = 1;
         }
-    } else if (fork) {
-        // dW2 needs only dz2 and h1: it runs beside dz1 -> dW1.  dz1 is queued first and keeps a ring of three
-        // stages here, so that a CTA of dW2 fits next to it on the same SM (2, 4 and 6 stages measured slower).
-        if (cudaEventRecord(h->ev_fork, s) != cudaSuccess) return COCOD_ERR_CUDA;
-        q.stages = std::min(q.stages, 3);
-        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, false)));
-        if (cudaStreamWaitEvent(h->side, h->ev_fork, 0) != cudaSuccess) return COCOD_ERR_CUDA;
-        r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, h->side, false)));
-        if (cudaEventRecord(h->ev_join, h->side) != cudaSuccess) return COCOD_ERR_CUDA;
-        r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, false)));
-        if (cudaStreamWaitEvent(s, h->ev_join, 0) != cudaSuccess) return COCOD_ERR_CUDA;
-    } else {
-        GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, pdl)));
-        r.c = grads + h->oW2; r.c_worker_stride = P; r.ldc = d_h; r.map_c_ok = 1;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz2, h->mn_h1, c_w2, r, K, s, pdl)));
-        r.N = d_in; r.c = grads + h->oW1; r.ldc = d_in;
-        GEMM_OK((launch_gemm<EPI_F32, true, true>(h->mn_dz1, mn_x, c_w1, r, K, s, pdl)));
+        const bool prof_upd = (capturing == cudaStreamCaptureStatusNone) && mlp_profile_open(h, h->prof_update, s);
+        if (h->profile != 0 && h->stamps && capturing == cudaStreamCaptureStatusNone && h->n_stamps < kMaxStamps)
+            uq.stamp = h->stamps + 2 * (size_t)(h->n_stamps++);
+        GEMM_OK(launch_update(u2, u1, uq, s, pdl && !prof_upd));
+        if (prof_upd) cudaEventRecord(h->prof_update.back().second, s);
     }
 #undef LAUNCH_OK
 #undef GEMM_OK

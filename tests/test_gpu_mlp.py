@@ -536,9 +536,9 @@ def test_fused_gradient_and_update_matches_the_oracle(M, E, K, dims, wd):
 
 @pytest.mark.parametrize("K,dims", [(3, (200, 256, 256, 7)), (16, I.MLP_DIMS)])
 def test_gradient_paths_replayed_from_a_cuda_graph_match_the_eager_calls(M, E, K, dims):
-    """Under stream capture the backward pass is queued as two branches on two streams (and without the
-    programmatic launch edges of the eager chain); replaying the graph must give the eager results bit for
-    bit, for the gradient call and for the fused gradient + update call, replay after replay."""
+    """Under stream capture the chain is queued without most of the programmatic launch edges of the eager chain;
+    replaying the graph must give the eager results bit for bit, for the gradient call and for the fused
+    gradient + update call, replay after replay."""
     rng = np.random.default_rng(100 + K)
     lr, mu, wd = 0.05, 0.9, 5e-4
     mg = M.MLPGrad(K, 128, dims[0], dims[1], dims[3])
