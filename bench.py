@@ -845,7 +845,8 @@ def measure_mlp(args, digest=False):
                                    "traffic": None, "peak_kind": peak_kind, "algorithmic_bytes_per_launch": 22 * K * P,
                                    "avg_launch_ms": round(avg_ms, 5), "bytes_per_parameter": 22,
                                    "measured_in": "a pass of its own with per-kernel CUDA events"}
-                out["gradient_pass_ms"] = {"whole_call": round(pass_ms, 5), "calls": calls}
+                out["gradient_pass_ms"] = {"whole_call": round(pass_ms, 5), "weight_gradient_kernel": round(upd_ms, 5),
+                                           "everything_else": round(pass_ms - upd_ms, 5), "calls": calls}
         torch.cuda.synchronize()
         n_done = min(step_no[0], n_rec) if not graphed else warm * k
         curve = loss_all[:n_done].double().mean(dim=1).cpu().numpy()
