@@ -76,9 +76,14 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
     uint8_t *xs = smem + UPD_RING, *vs = xs + BM * BN * 4;
     uint8_t *ss = vs + BM * BN * 4;           // bf16 staging: 64-column box b at b * 16 KB
     uint64_t *bars = reinterpret_cast<uint64_t *>(ss + UPD_SHADOW);
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 2), accf0 = smem_u32(bars + 4), acce0 = smem_u32(bars + 6);
-    const uint32_t xvf0 = smem_u32(bars + 8), xve0 = smem_u32(bars + 12);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 3), accf0 = smem_u32(bars + 6), acce0 = smem_u32(bars + 8);
+    const uint32_t xvf0 = smem_u32(bars + 10), xve0 = smem_u32(bars + 14);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 18);
+    // Operand ring: two stages of one reduction block each (one tile's operands) -- three in store_only mode, where the
+    // staging area of the bf16 copy is free: the first block of the next tile is then fetched while this tile's second
+    // block is still being multiplied.  Block number o = tile index * nkb + kb sits in stage o % n_stages.
+    const int n_stages = q.store_only ? 3 : 2;
+    auto stage_addr = [&](int st) { return st < 2 ? smem_u32(smem) + st * STAGE_BYTES : smem_u32(ss); };
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;          // stays 0: used by waits that must not be cut short
 
@@ -93,9 +98,11 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
         asm volatile("prefetch.tensormap [%0];" ::"l"(&p0.b) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&p0.x_in) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&p0.v) : "memory");
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < 3; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(accf0 + 8 * s, 1);
             mbar_init(acce0 + 8 * s, 8);      // one arrival per update warp
         }
@@ -134,22 +141,23 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
     int failed = 0;
     if (warp == 0 && lane == 0) {
         // ---- producer
-        int i = 0, issued_ops = 0, issued_xv = 0;      // tiles whose operand / x-v copies have been issued
+        int i = 0, issued_ops = 0, issued_xv = 0;      // operand blocks / tiles whose x-v copies have been issued
         for (int t = blockIdx.x; t < total && !failed && !q.debug_no_loads; t += gridDim.x, ++i) {
             const UpdateProblem *P; int wk, m0, n0;
             decode(t, P, wk, m0, n0);
             for (int kb = 0; kb < nkb; ++kb) {
-                if (i > 0 && !mbar_wait(empty0 + 8 * kb, (i - 1) & 1, abort, limit)) { failed = 1; break; }
-                const uint32_t bar = full0 + 8 * kb;
+                const int o = i * nkb + kb, st = o % n_stages, use = o / n_stages;
+                if (use > 0 && !mbar_wait(empty0 + 8 * st, (use - 1) & 1, abort, limit)) { failed = 1; break; }
+                const uint32_t bar = full0 + 8 * st;
                 mbar_expect_tx(bar, STAGE_BYTES);
-                const uint32_t dst_a = smem_base + kb * STAGE_BYTES, dst_b = dst_a + A_BYTES;
+                const uint32_t dst_a = stage_addr(st), dst_b = dst_a + A_BYTES;
                 tma_load_3d(dst_a, &P->a, bar, m0, kb * BK, wk);
                 tma_load_3d(dst_a + BK * 128, &P->a, bar, m0 + 64, kb * BK, wk);
                 tma_load_3d(dst_b, &P->b, bar, n0, kb * BK, wk);
                 tma_load_3d(dst_b + BK * 128, &P->b, bar, n0 + 64, kb * BK, wk);
+                issued_ops = o + 1;
             }
             if (failed) break;
-            issued_ops = i + 1;
             for (int cq = 0; cq < 4 && !q.store_only; ++cq) {
                 const int c = ((cq & 1) << 1) | (cq >> 1);      // 0, 2, 1, 3: each group's first chunk first
                 if (i > 0 && !mbar_wait(xve0 + 8 * c, (i - 1) & 1, abort, limit)) { failed = 1; break; }
@@ -162,8 +170,8 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
         }
         if (failed) {                 // let the copies of the last issued tile land before leaving
             abort[0] = 1;
-            if (issued_ops > 0)
-                for (int kb = 0; kb < nkb; ++kb) mbar_wait(full0 + 8 * kb, (issued_ops - 1) & 1, never, limit);
+            for (int o = (issued_ops > n_stages ? issued_ops - n_stages : 0); o < issued_ops; ++o)
+                mbar_wait(full0 + 8 * (o % n_stages), (o / n_stages) & 1, never, limit);
             if (issued_xv > 0)
                 for (int c = 0; c < 4; ++c) mbar_wait(xvf0 + 8 * c, (issued_xv - 1) & 1, never, limit);
         }
@@ -176,14 +184,15 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
             if (u > 0 && !mbar_wait(acce0 + 8 * a, (u - 1) & 1, abort, limit)) { failed = 2; break; }
             tc_fence_after();
             for (int kb = 0; kb < nkb; ++kb) {
-                if (!mbar_wait(full0 + 8 * kb, i & 1, abort, limit)) { failed = 2; break; }
+                const int o = i * nkb + kb, st = o % n_stages, use = o / n_stages;
+                if (!mbar_wait(full0 + 8 * st, use & 1, abort, limit)) { failed = 2; break; }
                 tc_fence_after();
-                const uint32_t a_addr = smem_base + kb * STAGE_BYTES, b_addr = a_addr + A_BYTES;
+                const uint32_t a_addr = stage_addr(st), b_addr = a_addr + A_BYTES;
 #pragma unroll
                 for (int k = 0; k < BK / UMMA_K; ++k)
                     umma_bf16(tmem_base + a * TMEM_COLS, smem_desc(a_addr + k * 2048u, true), smem_desc(b_addr + k * 2048u, true),
                               idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                umma_commit(empty0 + 8 * kb);     // frees the stage once these MMAs have read it
+                umma_commit(empty0 + 8 * st);     // frees the stage once these MMAs have read it
             }
             if (failed) break;
             umma_commit(accf0 + 8 * a);           // accumulator complete
