@@ -406,6 +406,50 @@ def measure_param_workload(args, wl, ctx, *, ring_n, do_e2e, cpu_seconds, do_gra
         eng.set_stream(compute)
         del g2
 
+    # ---- fusion variant of the round: the last local step and the merge in one pass (cocod_local_step_end)
+    def one_round_fused_end():
+        eng.comm_begin(side)
+        for j in range(k):
+            gbuf = ring[step_no[0] % len(ring)]
+            step_no[0] += 1
+            if j < k - 1:
+                eng.local_step(gbuf)
+            else:
+                eng.local_step_end(gbuf)
+
+    fusion = None
+    if do_schemes or do_graph is False:
+        for _ in range(3):
+            one_round_fused_end()
+        blocks = []
+        for rep in range(max(1, args.repeats)):
+            torch.cuda.synchronize()
+            ev0.record(compute)
+            for _ in range(steps):
+                one_round_fused_end()
+            ev1.record(compute)
+            torch.cuda.synchronize()
+            blocks.append(ev0.elapsed_time(ev1) / steps)
+        eng.set_option(E.OPT_PROFILE, 1)
+        eng.profile_reset()
+        for _ in range(min(steps, 20)):
+            one_round_fused_end()
+        byf = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+        eng.set_option(E.OPT_PROFILE, 0)
+        ms_f = median(blocks)
+        sm_bytes = (24.0 + 4.0 / K) * K * P
+        iv = byf.get("step_merge", [])
+        sm_ms = sum(b - a for a, b in iv) / max(1, len(iv))
+        fusion = {"last_step_and_merge_in_one_pass": {
+            "ms_per_step": ms_f, "ms_per_step_min": min(blocks), "ms_per_step_max": max(blocks),
+            "value": world * K * P * k / (ms_f * 1e-3), "speedup_over_the_three_kernels": (ms / steps) / ms_f,
+            "bytes_per_worker_parameter_per_round": 20 * (k - 1) + 24 + 4.0 / K + W.bytes_mean(K),
+            "kernel": {"name": "step_merge_vec8", "avg_ms": round(sm_ms, 5), "launches": len(iv),
+                       "algorithmic_bytes_per_launch": sm_bytes,
+                       "gbs": round(sm_bytes / (sm_ms * 1e-3) / 1e9, 1) if iv else None,
+                       "frac_of_peak": round(sm_bytes / (sm_ms * 1e-3) / 1e9 / hbm_peak, 4) if iv else None},
+            "note": "same values bit for bit; the headline value above is the explicit local step / mean / merge path"}}
+
     dom = "local_step"
     traffic = W.NCU_DRAM_BYTES_PER_WORKER_PARAM.get(dom)
     traffic = traffic * K * P if traffic is not None else None
@@ -488,7 +532,7 @@ def measure_param_workload(args, wl, ctx, *, ring_n, do_e2e, cpu_seconds, do_gra
         "overlap_fraction": overlap, "overlap_fraction_device_stamps": overlap_dev,
         "ms_per_round_overlapped": ms / steps, "ms_per_round_serial": ms_serial_plain,
         "ms_per_round_profiled": {"overlapped": ms_profiled, "serial": ms_serial},
-        "cuda_graph_replay": graph_extra, "ms_per_round_by_scheme": schemes,
+        "cuda_graph_replay": graph_extra, "ms_per_round_by_scheme": schemes, "fusion_variants": fusion,
         "hbm_gbs_whole_round": wl.bytes_per_round(args.snapshot == "copy") / (ms / steps * 1e-3) / 1e9,
     }
 
@@ -538,7 +582,7 @@ def run_ours(args, wl):
             other["vgg16"] = {key: v[key] for key in ("value", "steps", "ms_per_step", "timed_blocks", "config", "clocks",
                                                       "gpu_launches", "roofline", "cpu_baseline", "kernels_in_loop",
                                                       "kernels_isolated", "overlap_fraction", "overlap_fraction_device_stamps",
-                                                      "ms_per_round_serial", "hbm_gbs_whole_round")}
+                                                      "ms_per_round_serial", "hbm_gbs_whole_round", "fusion_variants")}
             other["vgg16"].update(metric=METRIC, unit=UNIT)
         except Exception as e:                              # e.g. a smaller GPU: say so instead of losing the headline
             other["vgg16"] = {"unavailable": f"{type(e).__name__}: {e}"}
@@ -677,9 +721,9 @@ def measure_mlp(args, digest=False):
     the same engine with its bf16 shadow switched on.  A step (round) = comm_begin, k = 4 x (batched gradients +
     local step), comm_end.  Every (worker, global step) has its own seeded minibatch (a pool of up to 2048 steps,
     generated on the device, labels from the teacher in fp64; a longer run goes through the pool again, like epochs
-    over a data set).  Three variants are timed, each from the common initial point: the two calls, the fused
-    gradient + update call, and the fused call replayed from CUDA graphs of two rounds each (one graph per pair of
-    rounds of the pool)."""
+    over a data set).  Four variants are timed, each from the common initial point: the two calls; the two calls with the
+    round's last local step and the merge in one pass (cocod_local_step_end); the fused gradient + update call; and the
+    fused call replayed from CUDA graphs of two rounds each (one graph per pair of rounds of the pool)."""
     import numpy as np
     import torch
     from paper_1906_12043_b200 import build, engine as E, inputs as I, mlp as M, workloads as W
@@ -711,7 +755,8 @@ def measure_mlp(args, digest=False):
     n_w12 = dims[1] * dims[0] + dims[2] * dims[1]                 # parameters the persistent kernel updates
 
     def run_variant(name):
-        fused, graphed = name != "two-call", name == "fused+graph"
+        fused, graphed = name in ("fused", "fused+graph"), name == "fused+graph"
+        fuse_end = name == "two-call+step_end"       # the round's last local step and the merge in one pass
         eng = E.Engine(K, P, lr, mu, wd)
         eng.set_option(E.OPT_BF16_SHADOW, 1)
         eng.set_params(x0)
@@ -729,8 +774,12 @@ def measure_mlp(args, digest=False):
                     mg.grad_step(eng, xs[first + j], ys[first + j], out)
                 else:
                     mg.grad(shadow, xs[first + j], ys[first + j], grads, out)
-                    eng.local_step(grads)
-            eng.comm_end()
+                    if fuse_end and j == k - 1:
+                        eng.local_step_end(grads)
+                    else:
+                        eng.local_step(grads)
+            if not fuse_end:
+                eng.comm_end()
 
         def eager_round():
             i = step_no[0]
@@ -857,7 +906,7 @@ def measure_mlp(args, digest=False):
     variants = {}
     curve2, snaps2 = None, None
     sampler = ClockSampler(0)
-    names = ["two-call", "fused", "fused+graph"]
+    names = ["two-call", "two-call+step_end", "fused", "fused+graph"]
     engines = {}
     for name in names:
         variants[name], engines[name], curve, snaps = run_variant(name)

@@ -70,7 +70,8 @@ enum {
 enum { COCOD_SNAPSHOT_COPY = 0, COCOD_SNAPSHOT_FLIP = 1 };
 
 /* Kernel kinds reported by cocod_profile_get. */
-enum { COCOD_KERNEL_LOCAL_STEP = 0, COCOD_KERNEL_SNAPSHOT = 1, COCOD_KERNEL_MEAN = 2, COCOD_KERNEL_MERGE = 3 };
+enum { COCOD_KERNEL_LOCAL_STEP = 0, COCOD_KERNEL_SNAPSHOT = 1, COCOD_KERNEL_MEAN = 2, COCOD_KERNEL_MERGE = 3,
+       COCOD_KERNEL_STEP_MERGE = 4 };
 
 /* ---------------------------------------------------------------------------------------------
  * Algorithm 1, "Input" / "Initialize": K workers, model size P, learning rate gamma = lr, and
@@ -106,6 +107,17 @@ int cocod_comm_begin(cocod_handle *h, cocod_stream_t side);
 /* Algorithm 1, line 6: once the mean is complete (stream-ordered wait, the host does not
  * block), x^i <- x_hat_t + (x^i - x_t^i) for every worker.  Errors: STATE without a begin. */
 int cocod_comm_end(cocod_handle *h);
+
+/* A fusion variant of the round: the LAST iteration of Step II of a round and line 6 in one call and one pass over the
+ * data.  Equal, bit for bit, to cocod_local_step(h, grads) followed by cocod_comm_end(h): the stepped model
+ * x' = x - lr v never goes to memory and line 6, x^i <- x_hat_t + (x' - x_t^i), is applied to it at once, so a round
+ * of k steps moves 20 (k - 1) + 24 + 4/K bytes per worker-parameter (plus the mean kernel's) instead of
+ * 20 k + 12 + 4/K.  The call waits (stream-ordered, not on the host) for the mean started by cocod_comm_begin, so with
+ * k = 1 nothing is left for the averaging to overlap with; with k >= 2 it still overlaps the first k - 1 steps.
+ * grads: device, K x P, borrowed.  Shapes the fused kernel does not take (P not a multiple of 8, misaligned gradient
+ * pointer) run the two kernels one after the other.  Errors: STATE without a begin (and, on a sharded engine, before
+ * cocod_comm_exchanged). */
+int cocod_local_step_end(cocod_handle *h, const float *grads);
 
 /* ---------------------------------------------------------------------------------------------
  * The two sequential schemes the paper compares against (Section 2 and Section 4.2, time-speedup

@@ -231,6 +231,31 @@ cudaError_t launch_merge(float *x, const float *snap, const float *mean, int K, 
     return cudaGetLastError();
 }
 
+// The fused last step + merge needs 8 columns per thread everywhere: returns false (nothing launched) when P or an
+// alignment does not allow it; the caller then runs the local step and the merge one after the other (same values).
+bool launch_step_merge(const float *x_in, float *x_out, float *v, const float *g, const float *snap, const float *mean,
+                       int K, int64_t P, float lr, float mu, float wd, __nv_bfloat16 *shadow, cudaStream_t s,
+                       cudaError_t *err)
+{
+    using namespace cocod;
+    *err = cudaSuccess;
+    if ((P % 8) != 0 || !aligned32(x_in) || !aligned32(x_out) || !aligned32(v) || !aligned32(g) || !aligned32(snap) ||
+        !aligned32(mean) || K > 4 * 65535 || (shadow != nullptr && !aligned16(shadow)))
+        return false;
+    const unsigned gx = grid_for(P / 8, kThreads);
+    if (K >= 4)                       // (four rows per thread: 0.673 ms on the ResNet18-sized workload, two rows: 0.698 ms)
+        step_merge_vec8<4><<<dim3(gx, (unsigned)((K + 3) / 4)), kThreads, 0, s>>>(x_in, x_out, v, g, snap, mean, K, P, lr, mu, wd,
+                                                                                shadow, g_stamp, g_backwards);
+    else if (K >= 2)
+        step_merge_vec8<2><<<dim3(gx, (unsigned)((K + 1) / 2)), kThreads, 0, s>>>(x_in, x_out, v, g, snap, mean, K, P, lr, mu, wd,
+                                                                                shadow, g_stamp, g_backwards);
+    else
+        step_merge_vec8<1><<<dim3(gx, 1), kThreads, 0, s>>>(x_in, x_out, v, g, snap, mean, K, P, lr, mu, wd, shadow, g_stamp,
+                                                          g_backwards);
+    *err = cudaGetLastError();
+    return true;
+}
+
 // ---------------------------------------------------------------- profiling brackets
 struct Bracket {
     cocod_engine *h;
@@ -246,6 +271,14 @@ struct Bracket {
         on = true;
         if (h->stamps) g_stamp = h->stamps + 2 * h->prof.size();      // this record's slot
         cudaEventRecord(a, s);
+    }
+    void cancel()                       // nothing was launched inside this bracket: keep no record
+    {
+        g_stamp = nullptr;
+        if (!on) return;
+        cudaEventDestroy(a);
+        cudaEventDestroy(b);
+        on = false;
     }
     ~Bracket()
     {
@@ -593,6 +626,39 @@ int cocod_comm_end(cocod_handle *h)
         CK(h, e);
     }
     h->launches += nl;
+    h->pending_flip = false;
+    h->snap = nullptr;
+    h->state = IDLE;
+    return COCOD_OK;
+}
+
+int cocod_local_step_end(cocod_handle *h, const float *grads)
+{
+    if (int rc = check_live(h)) return rc;
+    if (!grads) return COCOD_ERR_INVALID;
+    if (h->state != IN_FLIGHT) return COCOD_ERR_STATE;
+    if (h->K_global > 0 && !h->exchanged) return COCOD_ERR_STATE;      // the mean over the GPUs is not complete
+    if (h->side != h->compute) CK(h, cudaStreamWaitEvent(h->compute, h->ev_mean, 0));
+    const float *x_in = h->buf[h->cur];
+    float *x_out = h->pending_flip ? h->buf[1 - h->cur] : h->buf[h->cur];
+    bool fused = false;
+    {
+        Bracket br(h, h->compute, COCOD_KERNEL_STEP_MERGE);
+        if (h->sweep) h->dir ^= 1;
+        g_backwards = h->sweep ? h->dir : 0;
+        cudaError_t e = cudaSuccess;
+        fused = launch_step_merge(x_in, x_out, h->v, grads, h->snap, h->mean, h->K, h->P, h->lr, h->mu, h->wd, h->shadow,
+                                  h->compute, &e);
+        g_backwards = 0;
+        if (!fused) br.cancel();
+        CK(h, e);
+    }
+    if (!fused) {                    // shapes the fused kernel does not take: the two kernels, one after the other
+        if (int rc = cocod_local_step(h, grads)) return rc;
+        return cocod_comm_end(h);
+    }
+    ++h->launches;
+    finish_step(h);
     h->pending_flip = false;
     h->snap = nullptr;
     h->state = IDLE;

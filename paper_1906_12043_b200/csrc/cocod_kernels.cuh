@@ -457,6 +457,57 @@ merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, i
     stamp_end(stamp);
 }
 
+// Last local step of a round and line 6 in ONE pass (a fusion variant of the round; same values bit for bit as the
+// local step followed by the merge): d = fma(wd, x, g) ; v = fma(mu, v, d) ; x' = fma(-lr, v, x) ; x = mean + (x' - snap).
+// x' never goes to memory, the merge's re-read of x disappears: 24 + 4/K bytes per worker-parameter where the two
+// kernels move 20 + 12 + 4/K.  Same shape as merge_vec8: a thread owns 8 columns and RC rows, blockIdx.y picks the row
+// group.  x_in may alias snap (a round of one local step under the buffer flip) and x_in may equal x_out: every
+// element is read before it is written, by the same thread.
+template <int RC>
+__global__ void __launch_bounds__(kThreads)
+step_merge_vec8(const float *x_in, float *x_out, float *v, const float *__restrict__ g, const float *snap,
+                const float *__restrict__ mean, int K, int64_t P, float lr, float mu, float wd,
+                __nv_bfloat16 *__restrict__ shadow, unsigned long long *stamp, int backwards)
+{
+    stamp_begin(stamp);
+    const unsigned bx = backwards ? gridDim.x - 1u - blockIdx.x : blockIdx.x;
+    const unsigned by = backwards ? gridDim.y - 1u - blockIdx.y : blockIdx.y;
+    const int64_t c = ((int64_t)bx * kThreads + threadIdx.x) * 8;
+    if (c >= P) return;
+    const f32x8 m = ld256(mean + c);
+    const int i0 = by * RC;
+    f32x8 xr[RC], vr[RC], gr[RC], sr[RC];
+#pragma unroll
+    for (int j = 0; j < RC; ++j)
+        if (i0 + j < K) {
+            const int64_t e = (int64_t)(i0 + j) * P + c;
+            gr[j] = ld256(g + e);
+            xr[j] = ld256(x_in + e);
+            vr[j] = ld256(v + e);
+            sr[j] = ld256_stream(snap + e);
+        }
+#pragma unroll
+    for (int j = 0; j < RC; ++j)
+        if (i0 + j < K) {
+            const int64_t e = (int64_t)(i0 + j) * P + c;
+            f32x8 o, vn;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const float d = __fmaf_rn(wd, xr[j].a[q], gr[j].a[q]);
+                vn.a[q] = __fmaf_rn(mu, vr[j].a[q], d);
+                const float xs = __fmaf_rn(-lr, vn.a[q], xr[j].a[q]);
+                o.a[q] = __fadd_rn(m.a[q], __fsub_rn(xs, sr[j].a[q]));
+            }
+            st256(v + e, vn);
+            st256(x_out + e, o);
+            if (shadow != nullptr)
+                *reinterpret_cast<uint4 *>(shadow + e) =
+                    make_uint4(pack_bf16x2(o.a[0], o.a[1]), pack_bf16x2(o.a[2], o.a[3]),
+                               pack_bf16x2(o.a[4], o.a[5]), pack_bf16x2(o.a[6], o.a[7]));
+        }
+    stamp_end(stamp);
+}
+
 static __global__ void __launch_bounds__(kThreads)
 merge_scalar(float *x, const float *snap, const float *__restrict__ mean, int K, int64_t P,
              __nv_bfloat16 *__restrict__ shadow)

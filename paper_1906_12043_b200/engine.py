@@ -18,7 +18,7 @@ IPC_EXPORT_BYTES = 256
 OPT_SNAPSHOT, OPT_PROFILE, OPT_BF16_SHADOW, OPT_SWEEP = 1, 2, 3, 4
 SNAPSHOT_COPY, SNAPSHOT_FLIP = 0, 1
 KERNEL_LOCAL_STEP, KERNEL_SNAPSHOT, KERNEL_MEAN, KERNEL_MERGE = 0, 1, 2, 3
-KERNEL_NAMES = {0: "local_step", 1: "snapshot", 2: "mean", 3: "merge"}
+KERNEL_NAMES = {0: "local_step", 1: "snapshot", 2: "mean", 3: "merge", 4: "step_merge"}
 
 _vp, _i, _i64, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
 
@@ -30,6 +30,7 @@ SIGNATURES = {
     "cocod_local_step_host": (_i, [_vp, _vp]),
     "cocod_comm_begin": (_i, [_vp, _vp]),
     "cocod_comm_end": (_i, [_vp]),
+    "cocod_local_step_end": (_i, [_vp, _vp]),
     "cocod_local_sgd_average": (_i, [_vp]),
     "cocod_ssgd_step": (_i, [_vp, _vp]),
     "cocod_set_stream": (_i, [_vp, _vp]),
@@ -184,6 +185,12 @@ class Engine:
     def comm_begin(self, side_stream=None):
         """Step I: store x_t^i and start the averaging on ``side_stream``."""
         self._ck(self._lib.cocod_comm_begin(self._h, _stream(side_stream)), "cocod_comm_begin")
+
+    def local_step_end(self, grads):
+        """The round's last local step and the merge in one pass (bit-identical to local_step + comm_end)."""
+        if self._check_tensor(grads, self.K * self.P, "grads") != 0:
+            raise ValueError("grads must be a CUDA tensor")
+        self._ck(self._lib.cocod_local_step_end(self._h, _ptr(grads)), "cocod_local_step_end")
 
     def comm_end(self):
         """Line 6: x^i <- x_hat_t + (x^i - x_t^i)."""

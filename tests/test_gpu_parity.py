@@ -724,3 +724,62 @@ def test_alternating_sweep_and_device_time_stamps_change_no_value(E, K, P, shado
         assert all(comp[i][0] <= comp[i + 1][0] for i in range(len(comp) - 1))
     else:                                            # the flat local step still has a vectorised body; mean and merge do not
         assert len(stamps) == rounds * k and all(E.KERNEL_NAMES[kind] == "local_step" for kind, _, _ in stamps)
+
+
+# ----------------------------------------------------------------------------- fusion variant: last step + merge
+@pytest.mark.parametrize("K,P,k", [(16, 200_000, 2), (4, 100_000, 4), (5, 100_008, 1), (3, 1001, 2), (1, 4096, 3),
+                                   (64, 1032, 2), (2, 8, 1), (9, 8 * 1000, 3), (7, 262_144 + 12, 2)])
+@pytest.mark.parametrize("snapshot", [0, 1])
+def test_last_step_fused_with_the_merge_equals_the_two_calls_and_the_oracle(E, K, P, k, snapshot):
+    """cocod_local_step_end = the round's last iteration of Step II and line 6 in one pass.  Against the oracle (ref
+    at 1e-6 after one round / 1e-5 after the run, fp32 mirror bit for bit) and against an engine that makes the two
+    calls (bit for bit: x, v, average, bf16 copy), over rounds of k steps (k = 1: the stepped x aliases the stored copy
+    under the flip), unequal batch sizes, shapes that take the fused kernel and shapes that fall back to the two kernels."""
+    rounds, lr, mu, wd = 3, 0.1, 0.9, 5e-4
+    x0 = I.initial_point(P)
+    M = np.arange(1, K + 1, dtype=np.float64) if K in (5, 9) else None
+    fusedE, plainE = E.Engine(K, P, lr, mu, wd), E.Engine(K, P, lr, mu, wd)
+    ref = OracleEngine(K, P, lr, mu, wd, mode="ref", batch_sizes=M)
+    mir = OracleEngine(K, P, lr, mu, wd, mode="mirror", batch_sizes=M)
+    for eng in (fusedE, plainE):
+        eng.set_option(E.OPT_SNAPSHOT, snapshot)
+        eng.set_option(E.OPT_BF16_SHADOW, 1)
+        if M is not None:
+            eng.set_batch_sizes(M)
+        eng.set_params(torch.from_numpy(x0).cuda())
+    ref.set_params(x0)
+    mir.set_params(x0)
+    side = torch.cuda.Stream(priority=-1)
+    with pytest.raises(E.CocodError) as err:
+        fusedE.local_step_end(torch.zeros((K, P), dtype=torch.float32, device="cuda"))      # no round in flight
+    assert err.value.code == E.ERR_STATE
+    for r in range(rounds):
+        for eng in (fusedE, plainE):
+            eng.comm_begin(side)
+        ref.comm_begin()
+        mir.comm_begin()
+        for s in range(k):
+            g = I.gradients(K, P, r * k + s)
+            gd = torch.from_numpy(g).cuda()
+            if s < k - 1:
+                fusedE.local_step(gd)
+            else:
+                fusedE.local_step_end(gd)
+            plainE.local_step(gd)
+            ref.local_step(g)
+            mir.local_step(g)
+        plainE.comm_end()
+        ref.comm_end()
+        mir.comm_end()
+        what = f"round {r + 1}"
+        for got, want, name in ((fusedE.get_params(), plainE.get_params(), "x"), (fusedE.get_momentum(), plainE.get_momentum(), "v"),
+                                (fusedE.get_mean(), plainE.get_mean(), "average")):
+            assert torch.equal(got.view(torch.int32), want.view(torch.int32)), f"{name}, {what}"
+        assert torch.equal(fusedE.bf16_shadow().view(torch.int16), plainE.bf16_shadow().view(torch.int16)), f"bf16 copy, {what}"
+        assert_bit_equal(cpu(fusedE.get_params()), mir.x, f"x vs mirror, {what}")
+        assert_bit_equal(cpu(fusedE.get_momentum()), mir.v, f"v vs mirror, {what}")
+        rtol = 1e-6 if r == 0 else 1e-5
+        assert_close_scaled(cpu(fusedE.get_params()), ref.x, rtol, f"x vs ref, {what}")
+        assert_close_scaled(cpu(fusedE.get_momentum()), ref.v, rtol, f"v vs ref, {what}")
+    assert fusedE.step_count == plainE.step_count == rounds * k
+    np.testing.assert_array_equal(cpu(fusedE.bf16_shadow().float()), I.round_to_bf16(cpu(fusedE.get_params())))
