@@ -123,6 +123,10 @@ class WorkerShardedEngine:
         """Line 6 for this process's workers."""
         self.engine.comm_end()
 
+    def local_step_end(self, grads):
+        """The round's last local step and line 6 in one pass (equal to local_step + comm_end)."""
+        self.engine.local_step_end(grads)
+
     # -- around it
     def set_params(self, x0):
         self.engine.set_params(x0)

@@ -120,8 +120,9 @@ def virtual_ranks(E, K_global, G, P, M, attach):
     return engs
 
 
-def drive(E, engs, K_global, P, k, rounds, form, after_round=None):
-    """Algorithm 1 over all engines; everything is queued on one device in program order."""
+def drive(E, engs, K_global, P, k, rounds, form, after_round=None, fuse_end=False):
+    """Algorithm 1 over all engines; everything is queued on one device in program order.  fuse_end: the round's last
+    local step and line 6 through cocod_local_step_end instead of the two calls."""
     G = len(engs)
     sides = [torch.cuda.Stream() for _ in engs]
     bounds = [shard_workers(K_global, G, r) for r in range(G)]
@@ -148,9 +149,13 @@ def drive(E, engs, K_global, P, k, rounds, form, after_round=None):
             for e, (first, count) in zip(engs, bounds):
                 gd = torch.from_numpy(np.ascontiguousarray(g[first:first + count])).cuda()
                 keep.append(gd)
-                e.local_step(gd)
-        for e in engs:
-            e.comm_end()
+                if fuse_end and s == k - 1:
+                    e.local_step_end(gd)
+                else:
+                    e.local_step(gd)
+        if not fuse_end:
+            for e in engs:
+                e.comm_end()
         if after_round is not None:
             torch.cuda.synchronize()
             after_round(r, np.concatenate([cpu(e.get_params()) for e in engs], 0))
@@ -179,7 +184,7 @@ def test_gather_form_equals_the_single_engine_mirror_bit_for_bit(E, K_global, G,
     M = [32.0 * (1 + (i * 7) % 5) for i in range(K_global)] if weighted else None
     mir = oracle_run(K_global, P, k, rounds, M, "mirror")
     engs = virtual_ranks(E, K_global, G, P, M, attach=True)
-    x, v = drive(E, engs, K_global, P, k, rounds, "gather")
+    x, v = drive(E, engs, K_global, P, k, rounds, "gather", fuse_end=(G in (2, 4)))      # some spreads through the fused call
     assert_bit_equal(x, mir.x, "x")
     assert_bit_equal(v, mir.v, "v")
     assert_bit_equal(cpu(engs[-1].get_mean()), mir.mean, "average model")
