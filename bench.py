@@ -755,8 +755,9 @@ def measure_mlp(args, digest=False):
     n_w12 = dims[1] * dims[0] + dims[2] * dims[1]                 # parameters the persistent kernel updates
 
     def run_variant(name):
-        fused, graphed = name in ("fused", "fused+graph"), name == "fused+graph"
-        fuse_end = name == "two-call+step_end"       # the round's last local step and the merge in one pass
+        fused = name.startswith("fused")              # gradient + update in one call (all steps but, with step_end, the last)
+        graphed = name.endswith("+graph")
+        fuse_end = "+step_end" in name                # the round's last local step and the merge in one pass
         eng = E.Engine(K, P, lr, mu, wd)
         eng.set_option(E.OPT_BF16_SHADOW, 1)
         eng.set_params(x0)
@@ -770,7 +771,7 @@ def measure_mlp(args, digest=False):
             eng.comm_begin(side)
             for j in range(k):
                 out = loss_all[record_at + j] if (record_at is not None and record_at + k <= n_rec) else loss_all[n_rec]
-                if fused:
+                if fused and not (fuse_end and j == k - 1):
                     mg.grad_step(eng, xs[first + j], ys[first + j], out)
                 else:
                     mg.grad(shadow, xs[first + j], ys[first + j], grads, out)
@@ -906,7 +907,7 @@ def measure_mlp(args, digest=False):
     variants = {}
     curve2, snaps2 = None, None
     sampler = ClockSampler(0)
-    names = ["two-call", "two-call+step_end", "fused", "fused+graph"]
+    names = ["two-call", "two-call+step_end", "fused", "fused+graph", "fused+step_end", "fused+step_end+graph"]
     engines = {}
     for name in names:
         variants[name], engines[name], curve, snaps = run_variant(name)

@@ -783,3 +783,44 @@ def test_last_step_fused_with_the_merge_equals_the_two_calls_and_the_oracle(E, K
         assert_close_scaled(cpu(fusedE.get_momentum()), ref.v, rtol, f"v vs ref, {what}")
     assert fusedE.step_count == plainE.step_count == rounds * k
     np.testing.assert_array_equal(cpu(fusedE.bf16_shadow().float()), I.round_to_bf16(cpu(fusedE.get_params())))
+
+
+def test_rounds_ending_in_the_fused_call_replay_from_a_cuda_graph(E):
+    """Two rounds whose last step goes through cocod_local_step_end (which waits, on the stream, for the side stream's
+    mean) captured into a CUDA graph and replayed: equal to eagerly issued explicit rounds, bit for bit."""
+    K, P, k = 4, 100_000, 3
+    x0 = I.initial_point(P)
+    cap, side = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    static_g = [torch.from_numpy(I.gradients(K, P, t)).cuda() for t in range(2 * k)]
+    eager, graphed = E.Engine(K, P, 0.1, 0.9, 5e-4), E.Engine(K, P, 0.1, 0.9, 5e-4)
+    for eng in (eager, graphed):
+        eng.set_params(x0)
+    graphed.sync()
+    graphed.set_stream(cap)
+
+    def two_rounds(eng, fused_end):
+        for r in range(2):
+            eng.comm_begin(side)
+            for s in range(k):
+                if fused_end and s == k - 1:
+                    eng.local_step_end(static_g[r * k + s])
+                else:
+                    eng.local_step(static_g[r * k + s])
+            if not fused_end:
+                eng.comm_end()
+
+    with torch.cuda.stream(cap):
+        two_rounds(graphed, True)                    # warm-up on the capture stream
+    two_rounds(eager, False)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=cap):
+        two_rounds(graphed, True)
+    for _ in range(3):
+        graph.replay()
+        two_rounds(eager, False)
+        torch.cuda.synchronize()
+        assert_bit_equal(cpu(graphed.get_params()), cpu(eager.get_params()), "x")
+        assert_bit_equal(cpu(graphed.get_momentum()), cpu(eager.get_momentum()), "v")
+    graphed.sync()
+    graphed.set_stream(torch.cuda.current_stream())
