@@ -6,7 +6,9 @@
 A "step" is one communication round of Algorithm 1 over all K workers: comm_begin (stored copy +
 averaging on the side stream), k local momentum-SGD steps, comm_end (merge).  The metric is
 worker-parameter updates per second = K * P * k * rounds / time, whole job over all ranks.
-Prints ONE JSON line (rank 0).
+Prints ONE JSON line (rank 0).  The headline runs the three kernels the path is defined by; the same
+rounds with the last local step and the merge fused into one pass are reported under fusion_variants,
+the VGG16-sized and the end-to-end MLP workloads under other_workloads.
 
 N > 1 (torchrun): the path shards by parameter index with no exchange at all, so every rank
 runs the same per-GPU workload on its own column range (weak scaling); time is the max over
