@@ -1202,9 +1202,30 @@ def run_sweep(args):
                                  "gbs": {n: round(alg[n] / (sum(b - a for a, b in iv) / len(iv) * 1e-3) / 1e9, 1)
                                          for n, iv in by.items()},
                                  "overlap_fraction": overlap_fraction(by)}
+                # the same rounds with the last local step and the merge in one pass
+                def one_round_fused_end():
+                    eng.comm_begin(side)
+                    for j in range(k):
+                        if j < k - 1:
+                            eng.local_step(g)
+                        else:
+                            eng.local_step_end(g)
+
+                for _ in range(3):
+                    one_round_fused_end()
+                torch.cuda.synchronize()
+                ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                ev0.record(compute)
+                for _ in range(rounds):
+                    one_round_fused_end()
+                ev1.record(compute)
+                torch.cuda.synchronize()
+                ms_fe = ev0.elapsed_time(ev1) / rounds
                 ms = res["overlapped"]["ms_per_round"]
                 print(json.dumps({
                     "sweep": True, "K": K, "P": P, "k": k, "rounds": rounds,
+                    "ms_per_round_fused_end": ms_fe, "updates_per_s_fused_end": K * P * k / (ms_fe * 1e-3),
+                    "hbm_gbs_whole_round_fused_end": (wl.bytes_per_round() - 8 * K * P) / (ms_fe * 1e-3) / 1e9,
                     "updates_per_s": K * P * k / (ms * 1e-3),
                     "hbm_gbs_whole_round": wl.bytes_per_round() / (ms * 1e-3) / 1e9,
                     "ms_per_round": ms, "ms_per_round_serial": res["serial"]["ms_per_round"],
