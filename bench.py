@@ -605,6 +605,10 @@ def run_ours(args, wl):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         }
         line.update({key: res[key] for key in res if key not in ("value", "steps", "ms_per_step")})
+        fv = (res.get("fusion_variants") or {}).get("last_step_and_merge_in_one_pass")
+        if fv:                           # the fastest way through the library that ends on the same bits
+            line["best_value"] = {"value": fv["value"], "ms_per_step": fv["ms_per_step"],
+                                  "path": "cocod_local_step_end for the round's last step (fusion_variants)"}
         if other is not None:
             line["other_workloads"] = other
         print(json.dumps(line))

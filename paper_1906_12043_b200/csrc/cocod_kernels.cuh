@@ -14,6 +14,8 @@
 //                mean = s * (1/K) for equal weights, t_i = w_i * snap_i and mean = s otherwise.
 //                (Rounding error grows with log2(8) + K/8 additions instead of K.)
 //   merge      : x = mean + (x - snap)
+//   step+merge : the local step's three operations, then the merge's two, on the stepped x (same values as the two
+//                kernels one after the other)
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
