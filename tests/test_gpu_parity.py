@@ -188,7 +188,7 @@ def test_shapes_spanning_tiles_and_ragged_tails(E, K, P, snapshot):
     assert_close_scaled(v, ref.v, 1e-5, "v vs ref")
 
 
-@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("seed", range(40))
 def test_random_configurations_match_the_mirror_bit_for_bit(E, seed):
     """Randomised sweep over worker counts, sizes (aligned, ragged, tiny), periods, hyper-parameters,
     batch-size weights, snapshot modes, side-stream choices and the bf16 shadow: the fp32 mirror must
@@ -204,6 +204,8 @@ def test_random_configurations_match_the_mirror_bit_for_bit(E, seed):
     snapshot = int(rng.integers(0, 2))
     side = str(rng.choice(["own", "same", "high"]))
     shadow = bool(rng.random() < 0.3)
+    fuse_end = bool(rng.random() < 0.5)                 # the round's last step through cocod_local_step_end
+    sweep = bool(rng.random() < 0.3)                    # kernels walking in alternating directions
     x0 = (rng.standard_normal(P) * 0.05).astype(np.float32)
     G = (rng.standard_normal((k * rounds, K, P)) * 0.02).astype(np.float32)
 
@@ -213,6 +215,8 @@ def test_random_configurations_match_the_mirror_bit_for_bit(E, seed):
         eng.set_option(E.OPT_BF16_SHADOW, 1)
     if M is not None:
         eng.set_batch_sizes(M)
+    if sweep:
+        eng.set_option(E.OPT_SWEEP, 1)
     eng.set_params(x0)
     ref = OracleEngine(K, P, lr, mu, wd, mode="ref", batch_sizes=M)
     mir = OracleEngine(K, P, lr, mu, wd, mode="mirror", batch_sizes=M)
@@ -228,13 +232,18 @@ def test_random_configurations_match_the_mirror_bit_for_bit(E, seed):
         for s in range(k):
             g = G[r * k + s]
             keep.append(torch.from_numpy(g).cuda())
-            eng.local_step(keep[-1])
+            if fuse_end and s == k - 1:
+                eng.local_step_end(keep[-1])
+            else:
+                eng.local_step(keep[-1])
             ref.local_step(g)
             mir.local_step(g)
-        eng.comm_end()
+        if not fuse_end:
+            eng.comm_end()
         for o in (ref, mir):
             o.comm_end()
-    what = f"K={K} P={P} k={k} rounds={rounds} lr={lr} mu={mu} wd={wd} weighted={M is not None} snapshot={snapshot} side={side} shadow={shadow}"
+    what = (f"K={K} P={P} k={k} rounds={rounds} lr={lr} mu={mu} wd={wd} weighted={M is not None} snapshot={snapshot} side={side} "
+            f"shadow={shadow} fuse_end={fuse_end} sweep={sweep}")
     x, v = cpu(eng.get_params()), cpu(eng.get_momentum())
     assert_bit_equal(x, mir.x, "x vs mirror: " + what)
     assert_bit_equal(v, mir.v, "v vs mirror: " + what)
