@@ -590,6 +590,12 @@ def run_ours(args, wl):
             other["vgg16"] = {"unavailable": f"{type(e).__name__}: {e}"}
         finally:
             args.steps, args.repeats = saved
+        try:                                                # a digest of the scaling sweep: six of its 38 cells
+            digest = []
+            sweep_cells([(2, 1 << 24), (16, 1 << 24), (64, 1 << 24)], digest.append)
+            other["sweep_digest"] = {"cells": digest, "note": "timing only; the whole sweep is `bench.py --sweep`"}
+        except Exception as e:
+            other["sweep_digest"] = {"unavailable": f"{type(e).__name__}: {e}"}
         try:
             args.steps = max(2, min(saved[0], 20))
             other["mlp"] = measure_mlp(args, digest=True)
@@ -1155,90 +1161,97 @@ def run_worker_sharded(args, wl):
     dist.destroy_process_group()
 
 
-def run_sweep(args):
-    """Timing-only sweep over (P, K, k).  Values do not affect timing, so each cell reuses one
-    generated gradient buffer.  Cells whose four K x P buffers exceed 160 GB are skipped."""
+def sweep_cells(cells, emit):
+    """Timing-only measurement of (K, P) cells at k = 1 and k = 8.  Values do not affect timing, so each cell reuses
+    one generated gradient buffer.  `emit(record)` is called per (K, P, k)."""
     import torch
-    from paper_1906_12043_b200 import build, engine as E, inputs as I, workloads as W
-    build.build()
-    torch.cuda.set_device(0)
+    from paper_1906_12043_b200 import engine as E, inputs as I, workloads as W
     side = torch.cuda.Stream(priority=-1)
     compute = torch.cuda.current_stream()
-    for logP in [int(v) for v in args.sweep_logP.split(",")]:
-        for K in [int(v) for v in args.sweep_K.split(",")]:
-            P = 1 << logP
-            if K * P * 16 > 160e9:
-                continue
-            g = torch.empty((K, P), dtype=torch.float32, device="cuda")
-            I.device_gradients_into(g, 0)
-            x0 = torch.empty(P, dtype=torch.float32, device="cuda")
-            I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, 0, 0.01)
-            for k in (1, 8):
-                eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
-                eng.set_params(x0)
-                wl = W.Workload("sweep", K, P, k, 0, 0.1, 0.9, 5e-4)
-                rounds = max(3, min(200, int(0.25 / (wl.bytes_per_round() / 6.5e12))))
+    for K, P in cells:
+        g = torch.empty((K, P), dtype=torch.float32, device="cuda")
+        I.device_gradients_into(g, 0)
+        x0 = torch.empty(P, dtype=torch.float32, device="cuda")
+        I.device_gaussian_into(x0, I.X0_SEED, I.STREAM_X0, 0, 0, 0, 0.01)
+        for k in (1, 8):
+            eng = E.Engine(K, P, 0.1, 0.9, 5e-4)
+            eng.set_params(x0)
+            wl = W.Workload("sweep", K, P, k, 0, 0.1, 0.9, 5e-4)
+            rounds = max(3, min(200, int(0.25 / (wl.bytes_per_round() / 6.5e12))))
 
-                def one_round(s):
-                    eng.comm_begin(s)
-                    for _ in range(k):
-                        eng.local_step(g)
-                    eng.comm_end()
+            def one_round(s):
+                eng.comm_begin(s)
+                for _ in range(k):
+                    eng.local_step(g)
+                eng.comm_end()
 
-                res = {}
-                for mode, s in (("overlapped", side), ("serial", compute)):
-                    for _ in range(3):
-                        one_round(s)
-                    eng.set_option(E.OPT_PROFILE, 1)
-                    eng.profile_reset()
-                    torch.cuda.synchronize()
-                    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    ev0.record(compute)
-                    for _ in range(rounds):
-                        one_round(s)
-                    ev1.record(compute)
-                    torch.cuda.synchronize()
-                    by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
-                    eng.set_option(E.OPT_PROFILE, 0)
-                    alg = {"local_step": W.BYTES_LOCAL_STEP * K * P, "mean": W.bytes_mean(K) * K * P,
-                           "merge": W.bytes_merge(K) * K * P}
-                    res[mode] = {"ms_per_round": ev0.elapsed_time(ev1) / rounds,
-                                 "gbs": {n: round(alg[n] / (sum(b - a for a, b in iv) / len(iv) * 1e-3) / 1e9, 1)
-                                         for n, iv in by.items()},
-                                 "overlap_fraction": overlap_fraction(by)}
-                # the same rounds with the last local step and the merge in one pass
-                def one_round_fused_end():
-                    eng.comm_begin(side)
-                    for j in range(k):
-                        if j < k - 1:
-                            eng.local_step(g)
-                        else:
-                            eng.local_step_end(g)
-
+            res = {}
+            for mode, s in (("overlapped", side), ("serial", compute)):
                 for _ in range(3):
-                    one_round_fused_end()
+                    one_round(s)
+                eng.set_option(E.OPT_PROFILE, 1)
+                eng.profile_reset()
                 torch.cuda.synchronize()
                 ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 ev0.record(compute)
                 for _ in range(rounds):
-                    one_round_fused_end()
+                    one_round(s)
                 ev1.record(compute)
                 torch.cuda.synchronize()
-                ms_fe = ev0.elapsed_time(ev1) / rounds
-                ms = res["overlapped"]["ms_per_round"]
-                print(json.dumps({
-                    "sweep": True, "K": K, "P": P, "k": k, "rounds": rounds,
-                    "ms_per_round_fused_end": ms_fe, "updates_per_s_fused_end": K * P * k / (ms_fe * 1e-3),
-                    "hbm_gbs_whole_round_fused_end": (wl.bytes_per_round() - 8 * K * P) / (ms_fe * 1e-3) / 1e9,
-                    "updates_per_s": K * P * k / (ms * 1e-3),
-                    "hbm_gbs_whole_round": wl.bytes_per_round() / (ms * 1e-3) / 1e9,
-                    "ms_per_round": ms, "ms_per_round_serial": res["serial"]["ms_per_round"],
-                    "kernel_gbs_isolated": res["serial"]["gbs"], "kernel_gbs_overlapped": res["overlapped"]["gbs"],
-                    "overlap_fraction": res["overlapped"]["overlap_fraction"],
-                    "l2_resident": bool(K * P * 16 < 126e6)}), flush=True)
-                eng.destroy()
-            del g, x0
-            torch.cuda.empty_cache()
+                by = summarize_profile(eng.profile_records(), E.KERNEL_NAMES)
+                eng.set_option(E.OPT_PROFILE, 0)
+                alg = {"local_step": W.BYTES_LOCAL_STEP * K * P, "mean": W.bytes_mean(K) * K * P,
+                       "merge": W.bytes_merge(K) * K * P}
+                res[mode] = {"ms_per_round": ev0.elapsed_time(ev1) / rounds,
+                             "gbs": {n: round(alg[n] / (sum(b - a for a, b in iv) / len(iv) * 1e-3) / 1e9, 1)
+                                     for n, iv in by.items()},
+                             "overlap_fraction": overlap_fraction(by)}
+
+            # the same rounds with the last local step and the merge in one pass
+            def one_round_fused_end():
+                eng.comm_begin(side)
+                for j in range(k):
+                    if j < k - 1:
+                        eng.local_step(g)
+                    else:
+                        eng.local_step_end(g)
+
+            for _ in range(3):
+                one_round_fused_end()
+            torch.cuda.synchronize()
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ev0.record(compute)
+            for _ in range(rounds):
+                one_round_fused_end()
+            ev1.record(compute)
+            torch.cuda.synchronize()
+            ms_fe = ev0.elapsed_time(ev1) / rounds
+            ms = res["overlapped"]["ms_per_round"]
+            emit({
+                "sweep": True, "K": K, "P": P, "k": k, "rounds": rounds,
+                "ms_per_round_fused_end": ms_fe, "updates_per_s_fused_end": K * P * k / (ms_fe * 1e-3),
+                "hbm_gbs_whole_round_fused_end": (wl.bytes_per_round() - 8 * K * P) / (ms_fe * 1e-3) / 1e9,
+                "updates_per_s": K * P * k / (ms * 1e-3),
+                "hbm_gbs_whole_round": wl.bytes_per_round() / (ms * 1e-3) / 1e9,
+                "ms_per_round": ms, "ms_per_round_serial": res["serial"]["ms_per_round"],
+                "kernel_gbs_isolated": res["serial"]["gbs"], "kernel_gbs_overlapped": res["overlapped"]["gbs"],
+                "overlap_fraction": res["overlapped"]["overlap_fraction"],
+                "l2_resident": bool(K * P * 16 < 126e6)})
+            eng.destroy()
+        del g, x0
+        torch.cuda.empty_cache()
+
+
+def run_sweep(args):
+    """The scaling sweep over (P, K, k): one JSON line per cell.  Cells whose four K x P buffers exceed 160 GB are
+    skipped."""
+    import torch
+    from paper_1906_12043_b200 import build
+    build.build()
+    torch.cuda.set_device(0)
+    cells = [(K, 1 << logP) for logP in [int(v) for v in args.sweep_logP.split(",")]
+             for K in [int(v) for v in args.sweep_K.split(",")] if K * (1 << logP) * 16 <= 160e9]
+    sweep_cells(cells, lambda rec: print(json.dumps(rec), flush=True))
 
 
 def main():
