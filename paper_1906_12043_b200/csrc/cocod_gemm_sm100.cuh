@@ -101,6 +101,8 @@ struct Params {
     int *error_flag;
     unsigned long long wait_ns;        // time limit of every barrier wait (0 = WAIT_LIMIT_NS)
     int debug_no_loads;                // self-test: the producer issues nothing, so the waits run out
+    int b_keep;                        // 1: operand B (weights the next kernels of the chain read again) is fetched with the
+                                       //    L2 evict-last priority
 #ifdef COCOD_GEMM_TRACE
     unsigned long long *trace;         // tuning builds only: 8 timestamps per CTA
 #endif
@@ -161,6 +163,32 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t sr
 {
     asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                  ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+// L2 eviction priorities for bulk copies: data that is read or written once and not needed again soon leaves first,
+// data the next kernels of the chain come back to (the bf16 copy of the weights) leaves last.
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, int z,
+                                            uint64_t policy)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+                 "[%0], [%1, {%3, %4, %5}], [%2], %6;"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *map, uint32_t src, int x, int y, int z, uint64_t policy)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4}], [%1], %5;"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y), "r"(z), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void tma_store_wait_read()
@@ -294,7 +322,15 @@ gemm_bf16(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         } else {
             tma_load_3d(dst_a, &map_a, bar, kb * BK, m0, wk);
         }
-        if (B_MN) {
+        if (p.b_keep) {
+            const uint64_t pl = l2_policy_evict_last();
+            if (B_MN) {
+                tma_load_3d(dst_b, &map_b, bar, n0, kb * BK, wk, pl);
+                tma_load_3d(dst_b + BK * 128, &map_b, bar, n0 + 64, kb * BK, wk, pl);
+            } else {
+                tma_load_3d(dst_b, &map_b, bar, kb * BK, n0, wk, pl);
+            }
+        } else if (B_MN) {
             tma_load_3d(dst_b, &map_b, bar, n0, kb * BK, wk);
             tma_load_3d(dst_b + BK * 128, &map_b, bar, n0 + 64, kb * BK, wk);
         } else {

@@ -273,8 +273,10 @@ gemm_update_persistent(const __grid_constant__ UpdateProblem p0, const __grid_co
                         if (!q.store_only) tma_store_3d(&P->v, smem_u32(vs) + c * (BM * 128), n0 + c * 32, m0, wk);
                     }
                     // the group's 64-column box of the bf16 copy is complete after its second chunk
+                    // (evict-last: the 59 MB of bf16 weights are what the next step's forward and backward GEMMs read; x and v,
+                    //  ten times as much, pass through L2 with the normal priority.  Evict-first on the x / v loads cost 8 us.)
                     if (ok && cc == 1 && !q.store_only && P->has_shadow && n0 + group * 64 < P->N)
-                        tma_store_3d(&P->shadow, smem_u32(ss) + group * (BM * 128), n0 + group * 64, m0, wk);
+                        tma_store_3d(&P->shadow, smem_u32(ss) + group * (BM * 128), n0 + group * 64, m0, wk, l2_policy_evict_last());
                     tma_store_commit();
                 }
             }

@@ -66,9 +66,24 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b)
     const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);      // .x = a (low half), .y = b
     return *reinterpret_cast<const uint32_t *>(&h);
 }
+// The bf16 copy is what the gradient kernels of the next local step read (twice: forward and backward), a tenth of the
+// bytes that stream past it in between: it is stored with the L2 evict-last priority.
+__device__ __forceinline__ uint64_t l2_keep_policy()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 __device__ __forceinline__ void st_shadow4(__nv_bfloat16 *p, const float4 &x)
 {
-    *reinterpret_cast<uint2 *>(p) = make_uint2(pack_bf16x2(x.x, x.y), pack_bf16x2(x.z, x.w));
+    asm volatile("st.global.L2::cache_hint.v2.b32 [%0], {%1, %2}, %3;"
+                 :: "l"(p), "r"(pack_bf16x2(x.x, x.y)), "r"(pack_bf16x2(x.z, x.w)), "l"(l2_keep_policy()) : "memory");
+}
+__device__ __forceinline__ void st_shadow8(__nv_bfloat16 *p, const f32x8 &o)
+{
+    asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;"
+                 :: "l"(p), "r"(pack_bf16x2(o.a[0], o.a[1])), "r"(pack_bf16x2(o.a[2], o.a[3])),
+                    "r"(pack_bf16x2(o.a[4], o.a[5])), "r"(pack_bf16x2(o.a[6], o.a[7])), "l"(l2_keep_policy()) : "memory");
 }
 
 __device__ __forceinline__ void sgd_update(float4 &x, float4 &v, const float4 &g, float lr, float mu, float wd)
@@ -451,10 +466,7 @@ merge_vec8(float *x, const float *snap, const float *__restrict__ mean, int K, i
 #pragma unroll
             for (int q = 0; q < 8; ++q) o.a[q] = __fadd_rn(m.a[q], __fsub_rn(xr[j].a[q], sr[j].a[q]));
             st256(x + e, o);
-            if (shadow != nullptr)
-                *reinterpret_cast<uint4 *>(shadow + e) =
-                    make_uint4(pack_bf16x2(o.a[0], o.a[1]), pack_bf16x2(o.a[2], o.a[3]),
-                               pack_bf16x2(o.a[4], o.a[5]), pack_bf16x2(o.a[6], o.a[7]));
+            if (shadow != nullptr) st_shadow8(shadow + e, o);
         }
     stamp_end(stamp);
 }
@@ -502,10 +514,7 @@ step_merge_vec8(const float *x_in, float *x_out, float *v, const float *__restri
             }
             st256(v + e, vn);
             st256(x_out + e, o);
-            if (shadow != nullptr)
-                *reinterpret_cast<uint4 *>(shadow + e) =
-                    make_uint4(pack_bf16x2(o.a[0], o.a[1]), pack_bf16x2(o.a[2], o.a[3]),
-                               pack_bf16x2(o.a[4], o.a[5]), pack_bf16x2(o.a[6], o.a[7]));
+            if (shadow != nullptr) st_shadow8(shadow + e, o);
         }
     stamp_end(stamp);
 }

@@ -529,6 +529,7 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
         small.worker_stride = P; small.lr = fused->lr; small.mu = fused->mu; small.wd = fused->wd;
     }
     Params p{};
+    p.b_keep = 1;                      // the weights: read again by the backward pass and, rewritten in place, by the next step
     p.error_flag = h->error_flag;
     // h1 = relu(x W1^T + b1)
     p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
@@ -544,6 +545,7 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
                              h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out, small));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
     Params q{};
+    q.b_keep = 1;
     q.error_flag = h->error_flag;
     q.M = B; q.N = d_h; q.K = d_h; q.stages = stages_for(d_h);
     q.mask = h->h1; q.mask_worker_stride = (long long)B * d_h;
