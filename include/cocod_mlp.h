@@ -87,8 +87,13 @@ int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x
  * earliest start (after its wait for the predecessor) and the latest end of its thread blocks on the GPU's own clock,
  * so that its duration INSIDE the chain, with the programmatic overlap at both ends, can be read
  * (cocod_mlp_profile_get_device: number of stamped launches and their average milliseconds; also filled with
- * value 1).  The first non-zero setting allocates 64 KB on the device. */
-enum { COCOD_MLP_OPT_PROFILE = 1 };
+ * value 1).  The first non-zero setting allocates 64 KB on the device.
+ * COCOD_MLP_OPT_CHAIN = 1 (default) / 0: how the part of a gradient pass before the weight gradients (both hidden
+ * layers forward, the output layer, the hidden deltas) is launched: as ONE kernel in which the d_hidden / 128 thread
+ * blocks of a worker each own 128 columns of every hidden quantity and hand their tiles to one another through
+ * counters in global memory (every wait bounded; at most one block per SM per launch, all resident together, more
+ * workers than fit are split over several launches), or as one kernel per layer.  Both give the same bits. */
+enum { COCOD_MLP_OPT_PROFILE = 1, COCOD_MLP_OPT_CHAIN = 2 };
 int cocod_mlp_set_option(cocod_mlp_handle *h, int option, int value);
 int cocod_mlp_profile_get(cocod_mlp_handle *h, int *calls, float *pass_ms, float *update_ms);
 int cocod_mlp_profile_get_device(cocod_mlp_handle *h, int *calls, float *update_ms);
@@ -123,6 +128,13 @@ int cocod_gemm_wait_selftest(int wait_ms, cocod_stream_t stream);
  * tiles without touching memory (every barrier still sees all of its threads), tensor memory is
  * released, COCOD_ERR_TIMEOUT is returned and the context stays usable. */
 int cocod_gemm_update_wait_selftest(int wait_ms, cocod_stream_t stream);
+
+/* The same for the chain kernel (the part of the gradient pass before the weight gradients as one kernel whose CTAs wait
+ * for one another's tiles at counters in global memory): a small model of its own is run with a switch that keeps every
+ * CTA from reporting its first tile, so the wait for the worker's first hidden layer runs out after `wait_ms`
+ * (1 .. 2000); every CTA gives up, lets its copies land, frees its tensor memory and returns.  Returns COCOD_ERR_TIMEOUT
+ * (the expected outcome), COCOD_OK if nothing timed out, or a set-up error.  The context stays usable. */
+int cocod_mlp_chain_wait_selftest(int wait_ms, cocod_stream_t stream);
 
 #ifdef __cplusplus
 }

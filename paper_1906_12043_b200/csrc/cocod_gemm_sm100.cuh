@@ -75,6 +75,29 @@ __device__ __forceinline__ void step_element(const StepTarget &t, long long idx,
     if (t.shadow != nullptr) t.shadow[idx] = __float2bfloat16_rn(xn);
 }
 
+// The same for up to N elements at once: all loads first, so that their round trips overlap.
+template <int N>
+__device__ __forceinline__ void step_elements(const StepTarget &t, const long long (&idx)[N], const float (&g)[N], int n)
+{
+    float x[N], v[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i)
+        if (i < n) {
+            x[i] = t.x_in[idx[i]];
+            v[i] = t.v[idx[i]];
+        }
+#pragma unroll
+    for (int i = 0; i < N; ++i)
+        if (i < n) {
+            const float d = __fmaf_rn(t.wd, x[i], g[i]);
+            const float vn = __fmaf_rn(t.mu, v[i], d);
+            t.v[idx[i]] = vn;
+            const float xn = __fmaf_rn(-t.lr, vn, x[i]);
+            t.x_out[idx[i]] = xn;
+            if (t.shadow != nullptr) t.shadow[idx[i]] = __float2bfloat16_rn(xn);
+        }
+}
+
 struct Params {
     int M, N, K;                       // per-worker problem
     float *c;                          // EPI_F32

@@ -18,6 +18,7 @@
 #include "cocod_mlp.h"
 #include "cocod_gemm_sm100.cuh"
 #include "cocod_gemm_update_sm100.cuh"
+#include "cocod_mlp_chain_sm100.cuh"
 #include "cocod_internal.h"
 
 #include <algorithm>
@@ -156,6 +157,45 @@ cudaError_t launch_update(const UpdateProblem &p0, const UpdateProblem &p1, cons
     if (total <= 0) return cudaSuccess;
     return launch_dependent(pdl, gemm_update_persistent, dim3(std::min(total, sm_count[dev])), dim3(UPD_THREADS), (size_t)UPD_SMEM, s,
                             p0, p1, q);
+}
+
+// The gradient chain up to dz1 as one kernel: d_h / 128 CTAs per worker that wait for one another, so all CTAs of a
+// launch must be resident together: at most one CTA per SM per launch (a cooperative launch), the workers split over
+// several launches when there are more.
+template <int DOUT>
+cudaError_t launch_chain(const CUtensorMap &k_x, const CUtensorMap &k_w1, const CUtensorMap &k_h1, const CUtensorMap &k_w2,
+                         const CUtensorMap &k_w3, const CUtensorMap &k_dz2, const CUtensorMap &mn_w2, const CUtensorMap &st_dz1,
+                         ChainParams p, int tiles, int workers, cudaStream_t s, bool pdl, int *launches)
+{
+    static int sm_count[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    if (sm_count[dev] == 0) {
+        int sms = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(mlp_chain<DOUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, CH_SMEM);
+        if (e != cudaSuccess) return e;
+        sm_count[dev] = sms;
+    }
+    const int per_launch = sm_count[dev] / tiles;
+    if (per_launch < 1) return cudaErrorInvalidConfiguration;
+    for (int w0 = 0; w0 < workers; w0 += per_launch) {
+        const int n = std::min(per_launch, workers - w0);
+        p.w0 = w0;
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(tiles, 1, n); cfg.blockDim = dim3(CH_THREADS); cfg.dynamicSmemBytes = CH_SMEM; cfg.stream = s;
+        cudaLaunchAttribute at[2];
+        at[0].id = cudaLaunchAttributeCooperative;
+        at[0].val.cooperative = 1;
+        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = pdl ? 2 : 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, mlp_chain<DOUT>, k_x, k_w1, k_h1, k_w2, k_w3, k_dz2, mn_w2, st_dz1, p);
+        if (e != cudaSuccess) return e;
+        ++*launches;
+    }
+    return cudaSuccess;
 }
 
 inline int stages_for(int k) { return std::max(1, std::min(MAX_STAGES, (k + BK - 1) / BK)); }
@@ -364,6 +404,8 @@ struct cocod_mlp {
     CUtensorMap k_h1, k_dz2, mn_dz2, mn_h1, mn_dz1;
     CUtensorMap st_h2, st_dz1;          // store views (64 columns x 128 rows) of outputs that are not read that way
     long long launches = 0;
+    int *chain_sync = nullptr;          // [K][4] counters of the chain kernel (zero between launches)
+    int chain = 1;                      // COCOD_MLP_OPT_CHAIN: the four kernels before the weight gradients as one cluster kernel
     // COCOD_MLP_OPT_PROFILE: CUDA events around every gradient pass and around its gradient + update kernel
     int profile = 0;                    // 0 off, 1 events (+ stamps), 2 stamps only
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_pass, prof_update;
@@ -407,7 +449,7 @@ bool mlp_profile_open(cocod_mlp *h, std::vector<std::pair<cudaEvent_t, cudaEvent
 void mlp_free(cocod_mlp *h)
 {
     mlp_profile_clear(h);
-    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->logit_part, h->error_flag, h->stamps};
+    void *ptrs[] = {h->h1, h->h2, h->dz2, h->dz1, h->logit_part, h->error_flag, h->stamps, h->chain_sync};
     for (void *p : ptrs) if (p) cudaFree(p);
     delete h;
 }
@@ -442,7 +484,9 @@ int cocod_mlp_create(cocod_mlp_handle **out, int K, int batch, int d_in, int d_h
     alloc((void **)&h->dz1, act);
     alloc((void **)&h->logit_part, (size_t)K * (d_hidden / 128) * 128 * 16 * sizeof(float));
     alloc((void **)&h->error_flag, sizeof(int));
+    alloc((void **)&h->chain_sync, (size_t)K * 4 * sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(h->error_flag, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(h->chain_sync, 0, (size_t)K * 4 * sizeof(int));
     if (e != cudaSuccess) {
         cudaGetLastError();
         mlp_free(h);
@@ -528,21 +572,35 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
         small.x_in = fused->x_in; small.x_out = fused->x_out; small.v = fused->v; small.shadow = fused->shadow;
         small.worker_stride = P; small.lr = fused->lr; small.mu = fused->mu; small.wd = fused->wd;
     }
+    const bool chain = h->chain != 0;
+    if (chain) {
+        ChainParams c{};
+        c.d_in = d_in; c.d_h = d_h; c.d_out = d_out;
+        c.P = P; c.P_raw = h->P_raw; c.oW3 = h->oW3; c.ob1 = h->ob1; c.ob2 = h->ob2; c.ob3 = h->ob3;
+        c.params = prm; c.labels = labels; c.loss = loss; c.grads = grads; c.step = small; c.error_flag = h->error_flag;
+        c.logit_part = h->logit_part; c.sync = h->chain_sync;
+        int n = 0;
+        const cudaError_t e = (d_out == 10 ? launch_chain<10> : launch_chain<16>)(k_x, k_w1, h->k_h1, k_w2, k_w3, h->k_dz2, mn_w2,
+                                                                                 h->st_dz1, c, d_h / 128, K, s, pdl_fwd, &n);
+        h->launches += n;
+        if (e != cudaSuccess) { fprintf(stderr, "chain launch: %s\n", cudaGetErrorString(e)); return COCOD_ERR_CUDA; }
+    }
     Params p{};
     p.b_keep = 1;                      // the weights: read again by the backward pass and, rewritten in place, by the next step
     p.error_flag = h->error_flag;
     // h1 = relu(x W1^T + b1)
     p.M = B; p.N = d_h; p.K = d_in; p.stages = stages_for(d_in);
     p.bias = prm + h->ob1; p.bias_worker_stride = P;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, pdl_fwd)));
+    if (!chain) GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(k_x, k_w1, h->k_h1, p, K, s, pdl_fwd)));
     // h2 = relu(h1 W2^T + b2), and per 128-column tile the partial logits h2 W3^T of that tile
     p.K = d_h; p.stages = stages_for(d_h); p.bias = prm + h->ob2;
     p.logit_part = h->logit_part; p.b_next = prm + h->ob3; p.b_next_worker_stride = P; p.next_out = d_out;
-    GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, pdl_fwd, &k_w3)));
+    if (!chain) GEMM_OK((launch_gemm<EPI_BIAS_RELU, false, false>(h->k_h1, k_w2, h->st_h2, p, K, s, pdl_fwd, &k_w3)));
     // logits, loss, dz3; then dz2, dW3, db3, db2
-    GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
-                             dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->logit_part, d_h / 128, labels,
-                             h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out, small));
+    if (!chain)
+        GEMM_OK(launch_dependent(pdl, d_out == 10 ? head_backward<10, HEAD_NW> : head_backward<16, HEAD_NW>, dim3(d_h / 32 + 1, K),
+                                 dim3(32 * HEAD_NW), 0, s, h->h2, prm, (const float *)h->logit_part, d_h / 128, labels,
+                                 h->dz2, grads, loss, P, h->P_raw, h->oW3, h->ob2, h->ob3, B, d_h, d_out, small));
     // dz1 = (dz2 W2) * (h1 > 0): B operand is W2 itself, read with n contiguous
     Params q{};
     q.b_keep = 1;
@@ -561,7 +619,7 @@ int run_grad(cocod_mlp *h, const bf16 *prm, const bf16 *xin, const int32_t *labe
     // blocks): in the fused call it applies the local step to each tile as soon as its product is formed, in the gradient
     // call it writes the product out.
     static_assert(2 * BK == 128, "the update kernel holds the whole reduction in its two-stage ring");
-    GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, pdl)));
+    if (!chain) GEMM_OK((launch_gemm<EPI_MASK, false, true>(h->k_dz2, mn_w2, h->st_dz1, q, K, s, pdl)));
     {
         UpdateProblem u2{}, u1{};
         u2.a = h->mn_dz2; u2.b = h->mn_h1;
@@ -641,9 +699,21 @@ int cocod_mlp_grad_step(cocod_mlp_handle *h, cocod_handle *engine, const void *x
     return cocod_internal_finish_step(engine, 0);
 }
 
+#ifdef COCOD_CHAIN_TRACE
+int cocod_debug_chain_trace(unsigned long long *out, int n)
+{
+    return cudaMemcpyFromSymbol(out, cocod::gemm::g_chain_trace, (size_t)n * sizeof(unsigned long long)) == cudaSuccess ? 0 : 1;
+}
+#endif
+
 int cocod_mlp_set_option(cocod_mlp_handle *h, int option, int value)
 {
     if (!h) return COCOD_ERR_INVALID;
+    if (option == COCOD_MLP_OPT_CHAIN) {
+        if (value != 0 && value != 1) return COCOD_ERR_INVALID;
+        h->chain = value;
+        return COCOD_OK;
+    }
     if (option != COCOD_MLP_OPT_PROFILE) return COCOD_ERR_INVALID;
     if (value < 0 || value > 2) return COCOD_ERR_INVALID;
     if (cudaDeviceSynchronize() != cudaSuccess) return COCOD_ERR_CUDA;
@@ -704,6 +774,10 @@ int cocod_mlp_check(cocod_mlp_handle *h, cocod_stream_t stream)
     int flag = 0;
     if (cudaMemcpyAsync(&flag, h->error_flag, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess ||
         cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    // a chain kernel that gave up leaves its counters as they were: clear them once nothing of this handle runs any more
+    if (flag && (cudaDeviceSynchronize() != cudaSuccess ||
+                 cudaMemset(h->chain_sync, 0, (size_t)h->K * 4 * sizeof(int)) != cudaSuccess))
         return COCOD_ERR_CUDA;
     return flag ? COCOD_ERR_TIMEOUT : COCOD_OK;
 }
@@ -818,5 +892,46 @@ int cocod_gemm_update_wait_selftest(int wait_ms, cocod_stream_t stream)
     return f ? COCOD_ERR_TIMEOUT : COCOD_OK;
 }
 
+int cocod_mlp_chain_wait_selftest(int wait_ms, cocod_stream_t stream)
+{
+    if (wait_ms < 1 || wait_ms > 2000) return COCOD_ERR_INVALID;
+    // a small model of its own: 2 workers x 2 tiles, all inputs zero
+    cocod_mlp_handle *h = nullptr;
+    if (int rc = cocod_mlp_create(&h, 2, 128, 64, 256, 10)) return rc;
+    struct Guard { cocod_mlp_handle *h; ~Guard() { cocod_mlp_destroy(h); } } guard{h};
+    SelftestScratch sc;
+    const size_t n_state = (size_t)h->K * h->P;
+    bf16 *prm = static_cast<bf16 *>(sc.alloc(n_state * sizeof(bf16)));
+    bf16 *x = static_cast<bf16 *>(sc.alloc((size_t)h->K * 128 * 64 * sizeof(bf16)));
+    int32_t *labels = static_cast<int32_t *>(sc.alloc((size_t)h->K * 128 * sizeof(int32_t)));
+    float *out = static_cast<float *>(sc.alloc((n_state + h->K) * sizeof(float)));
+    if (!prm || !x || !labels || !out) return COCOD_ERR_OOM;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(prm, 0, n_state * sizeof(bf16), s) != cudaSuccess ||
+        cudaMemsetAsync(x, 0, (size_t)h->K * 128 * 64 * sizeof(bf16), s) != cudaSuccess ||
+        cudaMemsetAsync(labels, 0, (size_t)h->K * 128 * sizeof(int32_t), s) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    const uint64_t uK = h->K, uB = 128, uh = h->d_h, ui = h->d_in, uP = h->P;
+    CUtensorMap k_x, k_w1, k_w2, mn_w2, k_w3;
+    if (!make_map(&k_w3, prm + h->oW3, uh, 10, uK, uh, uP, NEXT_N) || !map_k(&k_x, x, ui, uB, uK, ui, uB * ui) ||
+        !map_k(&k_w1, prm + h->oW1, ui, uh, uK, ui, uP) || !map_k(&k_w2, prm + h->oW2, uh, uh, uK, uh, uP) ||
+        !map_mn(&mn_w2, prm + h->oW2, uh, uh, uK, uh, uP))
+        return COCOD_ERR_CUDA;
+    ChainParams c{};
+    c.d_in = h->d_in; c.d_h = h->d_h; c.d_out = h->d_out;
+    c.P = h->P; c.P_raw = h->P_raw; c.oW3 = h->oW3; c.ob1 = h->ob1; c.ob2 = h->ob2; c.ob3 = h->ob3;
+    c.params = prm; c.labels = labels; c.loss = out + n_state; c.grads = out; c.error_flag = h->error_flag;
+    c.logit_part = h->logit_part; c.sync = h->chain_sync;
+    c.wait_ns = (unsigned long long)wait_ms * 1000000ull;
+    c.debug_no_arrive = 1;
+    int n = 0;
+    if (launch_chain<10>(k_x, k_w1, h->k_h1, k_w2, k_w3, h->k_dz2, mn_w2, h->st_dz1, c, h->d_h / 128, h->K, s, false, &n) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    int f = 0;
+    if (cudaMemcpyAsync(&f, h->error_flag, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+        return COCOD_ERR_CUDA;
+    return f ? COCOD_ERR_TIMEOUT : COCOD_OK;
+}
 
 }  // extern "C"

@@ -25,10 +25,12 @@ SIGNATURES = {
     "cocod_mlp_launch_count": (_i64, [_vp]),
     "cocod_gemm_wait_selftest": (_i, [_i, _vp]),
     "cocod_gemm_update_wait_selftest": (_i, [_i, _vp]),
+    "cocod_mlp_chain_wait_selftest": (_i, [_i, _vp]),
     "cocod_gemm_bf16": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i64, _i64, _i64, _i64, _i64, _i64, _vp]),
 }
 
 OPT_PROFILE = 1
+OPT_CHAIN = 2
 _declared = False
 
 
@@ -106,6 +108,13 @@ class MLPGrad:
         if rc != _E.OK:
             raise _E.CocodError(rc, "cocod_mlp_set_option")
 
+    def set_chain(self, on):
+        """True (default): the four kernels before the weight gradients run as one cluster kernel (hidden widths up to
+        1024); False: one kernel per layer.  Both give the same bits."""
+        rc = self._lib.cocod_mlp_set_option(self._h, OPT_CHAIN, 1 if on else 0)
+        if rc != _E.OK:
+            raise _E.CocodError(rc, "cocod_mlp_set_option")
+
     def profile(self):
         """(recorded calls, average ms of a whole gradient pass, average ms of the gradient + update kernel)."""
         n, a, b = _i(), ctypes.c_float(), ctypes.c_float()
@@ -154,6 +163,11 @@ def gemm_bf16(A, B, C, a_rows_contiguous=False, b_rows_contiguous=False, stream=
 def gemm_update_wait_selftest(wait_ms: int = 50, stream=None) -> int:
     """The bounded-wait self-test of the persistent gradient + update kernel (ERR_TIMEOUT is the expected code)."""
     return int(load().cocod_gemm_update_wait_selftest(int(wait_ms), _cur_stream(stream)))
+
+
+def chain_wait_selftest(wait_ms: int = 50, stream=None) -> int:
+    """The bounded-wait self-test of the chain kernel (ERR_TIMEOUT is the expected code)."""
+    return int(load().cocod_mlp_chain_wait_selftest(int(wait_ms), _cur_stream(stream)))
 
 
 def gemm_wait_selftest(wait_ms: int = 50, stream=None) -> int:

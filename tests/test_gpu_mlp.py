@@ -364,6 +364,9 @@ def test_a_wait_that_nothing_satisfies_times_out_and_leaves_the_gpu_usable(M, E)
     # their remaining tiles without touching memory, and the fused path still works afterwards
     assert M.gemm_update_wait_selftest(50) == E.ERR_TIMEOUT
     assert M.gemm_update_wait_selftest(20) == E.ERR_TIMEOUT
+    # the chain kernel: no thread block reports its first tile, the others' wait for it runs out
+    assert M.chain_wait_selftest(50) == E.ERR_TIMEOUT
+    assert M.chain_wait_selftest(20) == E.ERR_TIMEOUT
     C.zero_()
     M.gemm_bf16(bf16_tensor(A), bf16_tensor(A), C)
     np.testing.assert_allclose(cpu(C)[0], A[0].astype(np.float64) @ A[0].astype(np.float64).T, rtol=0, atol=1e-4)
@@ -469,6 +472,46 @@ def test_fused_and_two_call_paths_stay_identical_over_long_uninterrupted_runs(M,
             assert torch.equal(sa.view(torch.int16), sb.view(torch.int16)), "bf16 copy, " + what
     again = run(False)
     assert all(torch.equal(a[0].view(torch.int32), b[0].view(torch.int32)) for a, b in zip(want, again)), "two calls, rerun"
+
+
+@pytest.mark.parametrize("K,dims", [(1, (64, 128, 128, 10)), (3, (200, 256, 256, 7)), (5, (72, 384, 384, 16)),
+                                    (20, (64, 1024, 1024, 10)), (16, I.MLP_DIMS)])
+def test_the_chain_kernel_and_the_per_layer_kernels_give_the_same_bits(M, E, K, dims):
+    """The part of the gradient pass before the weight gradients runs either as one kernel whose CTAs hand tiles to one
+    another through counters in global memory, or as one kernel per layer.  Gradients and losses (gradient call) and x, v,
+    the bf16 copy and the losses after three fused steps must agree bit for bit; K = 20 x 8 tiles needs two launches of
+    the chain kernel (more CTAs than SMs), 3 tiles and 16 classes take the other template paths."""
+    mg = M.MLPGrad(K, 128, dims[0], dims[1], dims[3])
+    P = mg.P
+    rng = np.random.default_rng(99 + K)
+    prm = np.zeros((K, P), np.float32)
+    prm[:, :mg.P_raw] = (rng.standard_normal((K, mg.P_raw)) * 0.05).astype(np.float32)
+    x0 = torch.from_numpy(prm).cuda()
+    shadow = x0.to(torch.bfloat16).contiguous()
+    X = torch.from_numpy(rng.standard_normal((3, K, 128, dims[0])).astype(np.float32)).cuda().to(torch.bfloat16)
+    y = torch.from_numpy(rng.integers(0, dims[3], (3, K, 128)).astype(np.int32)).cuda()
+    got = {}
+    for chain in (False, True):
+        mg.set_chain(chain)
+        g = torch.full((K, P), 7.0, dtype=torch.float32, device="cuda")
+        loss = torch.full((K,), 7.0, dtype=torch.float32, device="cuda")
+        mg.grad(shadow, X[0], y[0], g, loss)
+        eng = E.Engine(K, P, 0.05, 0.9, 5e-4)
+        eng.set_option(E.OPT_BF16_SHADOW, 1)
+        eng.set_params_all(x0)
+        losses = torch.empty((3, K), dtype=torch.float32, device="cuda")
+        for t in range(3):
+            mg.grad_step(eng, X[t], y[t], losses[t])
+        torch.cuda.synchronize()
+        mg.check()
+        got[chain] = (g, loss, eng.get_params().clone(), eng.get_momentum().clone(), eng.bf16_shadow().clone(), losses)
+        eng.destroy()
+    mg.set_chain(True)
+    for name, a, b in zip(("gradients", "loss", "x", "v", "bf16 copy", "losses of the fused steps"), got[False], got[True]):
+        ia = a.view(torch.int16 if a.dtype == torch.bfloat16 else torch.int32)
+        ib = b.view(torch.int16 if b.dtype == torch.bfloat16 else torch.int32)
+        assert torch.equal(ia, ib), f"{name}: {int((ia != ib).sum())} elements differ"
+    mg.destroy()
 
 
 @pytest.mark.parametrize("K,dims,wd", [(3, (200, 256, 256, 7), 5e-4), (16, I.MLP_DIMS, 0.0)])
