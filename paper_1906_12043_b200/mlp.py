@@ -109,8 +109,9 @@ class MLPGrad:
             raise _E.CocodError(rc, "cocod_mlp_set_option")
 
     def set_chain(self, on):
-        """True (default): the four kernels before the weight gradients run as one cluster kernel (hidden widths up to
-        1024); False: one kernel per layer.  Both give the same bits."""
+        """True (default): the part of a pass before the weight gradients (both hidden layers, the output layer, the
+        hidden deltas) runs as one kernel whose thread blocks hand tiles to one another through counters in global
+        memory; False: one kernel per layer.  Both give the same bits."""
         rc = self._lib.cocod_mlp_set_option(self._h, OPT_CHAIN, 1 if on else 0)
         if rc != _E.OK:
             raise _E.CocodError(rc, "cocod_mlp_set_option")
