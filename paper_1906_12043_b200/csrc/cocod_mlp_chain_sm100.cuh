@@ -19,7 +19,8 @@
 //
 // Roles in a CTA of 320 threads: warps 0..7 are the workers (epilogues, output layer), warp 8 (one lane) issues the TMA
 // loads, warp 9 (one lane) issues tcgen05.mma.  Shared memory: a 5-stage operand ring (32 KB per stage), one 128 x 128
-// bf16 tile buffer in the TMA / UMMA swizzle (h1, then h2, then dz2 in place of h2, then dz1), dz3, biases, barriers.
+// bf16 tile buffer in the TMA / UMMA swizzle (h1, then h2, then dz2 in place of h2, then dz1), dz3, biases, the output
+// layer's partial sums, barriers.
 // TMEM: two 128-column accumulators and 16 columns for the partial logits.
 //
 // The arithmetic, operation for operation, is that of the per-layer kernels (gemm_bf16 epilogues and head_backward), so
@@ -38,8 +39,10 @@ constexpr int CH_OFF_WN = CH_OFF_TILE + BM * BN * 2;
 constexpr int CH_OFF_DZ = CH_OFF_WN + 2 * NEXT_N * 128;
 constexpr int CH_OFF_BIAS = CH_OFF_DZ + BM * NEXT_N * 4;
 constexpr int CH_OFF_ROWLOSS = CH_OFF_BIAS + 2 * BN * 4;
-constexpr int CH_OFF_BARS = CH_OFF_ROWLOSS + BM * 4;
+constexpr int CH_OFF_RED = CH_OFF_ROWLOSS + BM * 4;             // partial sums of the output layer: [2][16][128] + [2][128] floats
+constexpr int CH_OFF_BARS = CH_OFF_RED + (2 * 16 + 2) * BN * 4;
 constexpr int CH_SMEM = CH_OFF_BARS + 256 + 1024;  // + alignment slack
+static_assert(CH_SMEM <= 227 * 1024, "shared memory of the chain kernel");
 
 struct ChainParams {
     int d_in, d_h, d_out;
@@ -118,10 +121,8 @@ mlp_chain(const __grid_constant__ CUtensorMap k_x, const __grid_constant__ CUten
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * CH_STAGES + 6);
     volatile int *abort = reinterpret_cast<volatile int *>(tmem_slot + 1);
     volatile int *never = abort + 1;
-    // scratch of the output-layer phase: the activation halves of ring stages 0 and 1 (idle then: the next layer's
-    // activation blocks are asked for only after every CTA of the worker has finished that phase)
-    float *red = reinterpret_cast<float *>(smem);                           // [2][16][128]
-    float *redsum = reinterpret_cast<float *>(smem + STAGE_BYTES);          // [2][128]
+    float *red = reinterpret_cast<float *>(smem + CH_OFF_RED);             // [2][16][128]
+    float *redsum = red + 2 * 16 * BN;                                      // [2][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rank = blockIdx.x, tiles = gridDim.x, w = p.w0 + blockIdx.z;
